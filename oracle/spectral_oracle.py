@@ -1,0 +1,340 @@
+"""fp64 CPU oracle for the spectral-correction optimizer step.
+
+THIS IS TEST INFRASTRUCTURE, NOT PRODUCT CODE.  Only the test-suite, the
+smoke check and the benchmark's CPU-baseline leg may import it.  It shares no
+code with the CUDA path and never imports it.
+
+Every function is the plain definition of one step of the method (Section 3.2
+"Anchor Priors and Spectral Correction", Eq. 1-3, Algorithm 1 lines 7-14 and
+the operator P_t of the convergence appendix), written in NumPy fp64 with no
+blocking, fusion or reordering.  A library routine (LAPACK SVD / QR / matmul)
+is used as a step where the paper just says "SVD".
+
+Two basis modes exist because the paper only says "SVD" while the GPU path
+uses a randomized subspace iteration:
+
+* EXACT  - full thin SVD of the anchor momentum, keep the leading r triplets
+           (the operator D_t = diag(d_1..d_r) of the appendix).
+* MIRROR - the documented randomized range finder written out in fp64:
+           Q = orth(M W); q x { Z = orth(M^T Q); Q = orth(M Z) };
+           B = Q^T M; thin SVD of B; U = Q U_B[:, :r], V = V_B[:, :r].
+           In exact arithmetic it depends only on (M, W, q, r), not on how
+           orth() is realised.
+
+Pins (tests/test_oracle_pins.py): hand-derived 2x2 worked example, brute-force
+one-sided Jacobi SVD, rank-1 / diagonal closed forms, Lemma 1 and Lemma 2,
+idempotence at tau_p = 0, the alpha / rank / keep limit cases, torch AdamW in
+fp64, the closed-form global norm, MIRROR == EXACT for rank(M) <= r.
+Parity unpinned: end-to-end MIRROR vs EXACT on inputs with no spectral gap at r
+(the cut is ill-posed there; it is reported, not gated).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------
+# Eq. 1 / Algorithm 1 line 8: anchor momentum
+# --------------------------------------------------------------------------
+def anchor_ema(M_anc: np.ndarray, G_anc: np.ndarray, beta_anc: float) -> np.ndarray:
+    """M <- beta_anc * M + (1 - beta_anc) * G_anc  (Eq. 1; zero init, no bias correction)."""
+    return beta_anc * np.asarray(M_anc, F64) + (1.0 - beta_anc) * np.asarray(G_anc, F64)
+
+
+# --------------------------------------------------------------------------
+# "M = U S V^T" (Section 3.2, "From momentum to a denoising operator")
+# --------------------------------------------------------------------------
+def svd_exact(M: np.ndarray):
+    """Thin SVD through LAPACK, singular values descending.  Returns (U, s, V) with M = U diag(s) V^T."""
+    U, s, Vt = np.linalg.svd(np.asarray(M, F64), full_matrices=False)
+    return U, s, Vt.T
+
+
+def svd_jacobi(M: np.ndarray, sweeps: int = 60, tol: float = 1e-15):
+    """Brute-force one-sided (Hestenes) Jacobi SVD, pure loops; for tiny matrices only.
+
+    Used to pin svd_exact to something that is not LAPACK.  Returns (U, s, V)
+    sorted by descending s.  Columns of U belonging to zero singular values are
+    left as zero vectors (callers compare only the non-null part).
+    """
+    A = np.array(M, F64)
+    transposed = A.shape[0] < A.shape[1]
+    if transposed:
+        A = A.T.copy()
+    m, n = A.shape
+    V = np.eye(n)
+    for _ in range(sweeps):
+        off = 0.0
+        for p in range(n - 1):
+            for q in range(p + 1, n):
+                a = A[:, p] @ A[:, p]
+                b = A[:, q] @ A[:, q]
+                c = A[:, p] @ A[:, q]
+                if abs(c) <= tol * np.sqrt(a * b) or c == 0.0:
+                    continue
+                off = max(off, abs(c) / np.sqrt(a * b))
+                zeta = (b - a) / (2.0 * c)
+                t = np.sign(zeta) / (abs(zeta) + np.sqrt(1.0 + zeta * zeta)) if zeta != 0 else 1.0
+                cs = 1.0 / np.sqrt(1.0 + t * t)
+                sn = cs * t
+                Ap = A[:, p].copy()
+                A[:, p] = cs * Ap - sn * A[:, q]
+                A[:, q] = sn * Ap + cs * A[:, q]
+                Vp = V[:, p].copy()
+                V[:, p] = cs * Vp - sn * V[:, q]
+                V[:, q] = sn * Vp + cs * V[:, q]
+        if off <= tol:
+            break
+    s = np.sqrt(np.sum(A * A, axis=0))
+    order = np.argsort(-s)
+    s = s[order]
+    A = A[:, order]
+    V = V[:, order]
+    U = np.zeros_like(A)
+    nz = s > 0
+    U[:, nz] = A[:, nz] / s[nz]
+    if transposed:
+        U, V = V, U
+    return U, s, V
+
+
+def truncate(U, s, V, r: int):
+    """Keep the leading r singular triplets (D_t = diag(d_1..d_r)); r = 0 gives an empty basis."""
+    r = int(r)
+    return U[:, :r], s[:r], V[:, :r]
+
+
+# --------------------------------------------------------------------------
+# Eq. 2: soft spectral filter
+# --------------------------------------------------------------------------
+def filter_weights(s: np.ndarray, tau_p: float) -> np.ndarray:
+    """d_i = s_i / (s_i + tau_p)  (Eq. 2).  0/0 (s_i = tau_p = 0) is taken as 0: an unsupported direction."""
+    s = np.asarray(s, F64)
+    den = s + tau_p
+    out = np.zeros_like(s)
+    np.divide(s, den, out=out, where=den > 0)
+    return out
+
+
+# --------------------------------------------------------------------------
+# "Two-sided application"
+# --------------------------------------------------------------------------
+def project(U, G, V):
+    """X = U^T G V."""
+    return U.T @ np.asarray(G, F64) @ V
+
+
+def filtered_gradient(U, d, G, V):
+    """G_filt = U diag(d) (U^T G V) diag(d) V^T  ==  P_t(G)."""
+    X = project(U, G, V)
+    X_filt = (d[:, None] * X) * d[None, :]
+    return U @ X_filt @ V.T
+
+
+def blend(G, G_filt, alpha: float):
+    """G_proj = alpha G + (1 - alpha) G_filt  (Eq. 3)."""
+    return alpha * np.asarray(G, F64) + (1.0 - alpha) * G_filt
+
+
+def corrected_gradient(U, s, V, G, alpha: float, tau_p: float, scale: float = 1.0):
+    """Eq. 2 + two-sided filter + Eq. 3 on g = scale * G (scale = 1/keep for un-rescaled inputs)."""
+    g = scale * np.asarray(G, F64)
+    d = filter_weights(s, tau_p)
+    return blend(g, filtered_gradient(U, d, g, V), alpha)
+
+
+# --------------------------------------------------------------------------
+# Diagnostics that the appendix defines
+# --------------------------------------------------------------------------
+def alignment_eta(U, G, V) -> float:
+    """eta_r = ||U^T g V||_F^2 / ||g||_F^2 (Alignment Trajectory appendix)."""
+    G = np.asarray(G, F64)
+    den = float(np.sum(G * G))
+    return float(np.sum(project(U, G, V) ** 2) / den) if den > 0 else 0.0
+
+
+def effective_rank(d) -> float:
+    """r_eff = ||D_t||_F^2 = sum_i d_i^2  (Lemma 2)."""
+    d = np.asarray(d, F64)
+    return float(np.sum(d * d))
+
+
+def gproj_sqnorm_closed_form(g_sqnorm: float, X, d, alpha: float) -> float:
+    """||G_proj||_F^2 from ||g||^2 and X = U^T g V only.
+
+    <g, U A V^T> = <U^T g V, A> and ||U A V^T||_F = ||A||_F for orthonormal U, V,
+    so with A = D X D:  ||alpha g + (1-alpha) U A V^T||^2
+      = alpha^2 ||g||^2 + 2 alpha (1-alpha) sum d_i d_j X_ij^2 + (1-alpha)^2 sum d_i^2 d_j^2 X_ij^2.
+    """
+    X = np.asarray(X, F64)
+    dd = np.outer(d, d)
+    return float(alpha * alpha * g_sqnorm
+                 + 2.0 * alpha * (1.0 - alpha) * np.sum(dd * X * X)
+                 + (1.0 - alpha) ** 2 * np.sum(dd * dd * X * X))
+
+
+def clip_factor(total_sqnorm: float, max_norm: float) -> float:
+    """Global-norm clipping factor min(1, c_max / ||G_proj||) over all matrices; max_norm <= 0 switches it off."""
+    if max_norm is None or max_norm <= 0.0:
+        return 1.0
+    nrm = float(np.sqrt(total_sqnorm))
+    return 1.0 if nrm <= max_norm else max_norm / nrm
+
+
+# --------------------------------------------------------------------------
+# Algorithm 1 line 13: AdamW with G_proj
+# --------------------------------------------------------------------------
+def adamw_step(W, m, v, g, t: int, lr: float, beta1: float, beta2: float, eps: float, weight_decay: float):
+    """One decoupled-weight-decay Adam step, step count t >= 1.
+
+    m <- b1 m + (1-b1) g ; v <- b2 v + (1-b2) g^2 ;
+    W <- W - lr*wd*W - lr * (m / (1-b1^t)) / (sqrt(v / (1-b2^t)) + eps).
+    Returns new (W, m, v).
+    """
+    W = np.asarray(W, F64)
+    g = np.asarray(g, F64)
+    m = beta1 * np.asarray(m, F64) + (1.0 - beta1) * g
+    v = beta2 * np.asarray(v, F64) + (1.0 - beta2) * g * g
+    m_hat = m / (1.0 - beta1 ** t)
+    v_hat = v / (1.0 - beta2 ** t)
+    W = W - lr * weight_decay * W - lr * m_hat / (np.sqrt(v_hat) + eps)
+    return W, m, v
+
+
+# --------------------------------------------------------------------------
+# Randomized range finder (MIRROR mode)
+# --------------------------------------------------------------------------
+_GOLDEN = np.uint64(0x9E3779B97F4A7C15)
+_MIX1 = np.uint64(0xBF58476D1CE4E5B9)
+_MIX2 = np.uint64(0x94D049BB133111EB)
+
+
+def mix64(x: np.ndarray) -> np.ndarray:
+    """The 64-bit finaliser of the SplitMix64 generator (wrap-around uint64 arithmetic)."""
+    x = np.asarray(x, np.uint64)
+    with np.errstate(over="ignore"):
+        x = (x ^ (x >> np.uint64(30))) * _MIX1
+        x = (x ^ (x >> np.uint64(27))) * _MIX2
+        x = x ^ (x >> np.uint64(31))
+    return x
+
+
+def rademacher_sketch(seed: int, mat_id: int, n: int, l: int) -> np.ndarray:
+    """Sketch matrix W in {-1,+1}^{n x l}, a pure function of (seed, mat_id, row j, column c).
+
+    counter = mat_id * 2^44 + j * 2^10 + c ; h = mix64(seed XOR (counter + 1) * golden) ;
+    W[j, c] = +1 if the top bit of h is 0 else -1.
+    """
+    j = np.arange(n, dtype=np.uint64)[:, None]
+    c = np.arange(l, dtype=np.uint64)[None, :]
+    with np.errstate(over="ignore"):
+        counter = np.uint64(mat_id) * np.uint64(1 << 44) + j * np.uint64(1 << 10) + c
+        h = mix64(np.uint64(seed) ^ ((counter + np.uint64(1)) * _GOLDEN))
+    return np.where((h >> np.uint64(63)) == 0, 1.0, -1.0).astype(F64)
+
+
+def _orth(Y):
+    """Orthonormal basis of range(Y) by Householder QR."""
+    Q, _ = np.linalg.qr(Y)
+    return Q
+
+
+def mirror_basis(M, Omega, q: int, r: int):
+    """Rank-r basis by randomized subspace iteration with sketch Omega (n x l), q power iterations."""
+    M = np.asarray(M, F64)
+    if r == 0:
+        return np.zeros((M.shape[0], 0)), np.zeros(0), np.zeros((M.shape[1], 0))
+    Q = _orth(M @ Omega)
+    for _ in range(int(q)):
+        Z = _orth(M.T @ Q)
+        Q = _orth(M @ Z)
+    B = Q.T @ M
+    Ub, s, Vbt = np.linalg.svd(B, full_matrices=False)
+    U = Q @ Ub
+    return U[:, :r], s[:r], Vbt.T[:, :r]
+
+
+def projector_distance(Ua, Ub) -> float:
+    """||Ua Ua^T - Ub Ub^T||_F / sqrt(2 r), via ||Pa-Pb||_F^2 = ra + rb - 2||Ua^T Ub||_F^2 (sign/rotation free)."""
+    ra, rb = Ua.shape[1], Ub.shape[1]
+    if ra == 0 and rb == 0:
+        return 0.0
+    d2 = ra + rb - 2.0 * float(np.sum((Ua.T @ Ub) ** 2))
+    return float(np.sqrt(max(d2, 0.0) / (ra + rb)))
+
+
+# --------------------------------------------------------------------------
+# Whole step for one matrix, and a small state holder (Algorithm 1 lines 7-14)
+# --------------------------------------------------------------------------
+@dataclass
+class Hyper:
+    alpha: float = 0.3
+    tau_p: float = 1e-3
+    beta_anc: float = 0.9
+    lr: float = 2e-5
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-8
+    weight_decay: float = 0.0
+    max_grad_norm: float = 0.0      # 0 = no clipping
+    grads_prescaled: bool = True    # False: the step multiplies the masked gradient by 1/keep
+    keep: float = 1.0
+
+
+@dataclass
+class MatrixState:
+    """Per-matrix oracle state: anchor momentum, cached basis, AdamW moments."""
+    M_anc: np.ndarray
+    U: np.ndarray = None
+    s: np.ndarray = None
+    V: np.ndarray = None
+    have_anchor: bool = False
+    extra: dict = field(default_factory=dict)
+
+
+def new_state(m: int, n: int) -> MatrixState:
+    return MatrixState(M_anc=np.zeros((m, n), F64), U=np.zeros((m, 0)), s=np.zeros(0), V=np.zeros((n, 0)))
+
+
+def anchor_update(state: MatrixState, G_anc, hp: Hyper, r: int, mode: str = "exact",
+                  Omega=None, q: int = 1) -> MatrixState:
+    """Anchor arrival: Eq. 1 then the rank-r basis of the new momentum (cached until the next arrival)."""
+    state.M_anc = anchor_ema(state.M_anc, G_anc, hp.beta_anc)
+    if mode == "exact":
+        state.U, state.s, state.V = truncate(*svd_exact(state.M_anc), r)
+    elif mode == "mirror":
+        state.U, state.s, state.V = mirror_basis(state.M_anc, Omega, q, r)
+    else:
+        raise ValueError(mode)
+    state.have_anchor = True
+    return state
+
+
+def correct(state: MatrixState, G_mask, hp: Hyper):
+    """G_proj for one matrix (before optional clipping).  Also returns X and ||g||^2 for the closed-form norm."""
+    scale = 1.0 if hp.grads_prescaled else 1.0 / hp.keep
+    g = scale * np.asarray(G_mask, F64)
+    d = filter_weights(state.s, hp.tau_p)
+    X = project(state.U, g, state.V)
+    G_proj = blend(g, state.U @ ((d[:, None] * X) * d[None, :]) @ state.V.T, hp.alpha)
+    return G_proj, X, float(np.sum(g * g)), d
+
+
+def correct_and_step(states, G_masks, Ws, ms, vs, t: int, hp: Hyper):
+    """One fast-circuit step over a list of matrices: correction, optional global clip, AdamW.
+
+    Returns (new Ws, new ms, new vs, list of G_proj after clipping).
+    """
+    projs = [correct(st, G, hp)[0] for st, G in zip(states, G_masks)]
+    total = sum(float(np.sum(P * P)) for P in projs)
+    c = clip_factor(total, hp.max_grad_norm)
+    outW, outm, outv, outg = [], [], [], []
+    for P, W, m, v in zip(projs, Ws, ms, vs):
+        g = c * P
+        W2, m2, v2 = adamw_step(W, m, v, g, t, hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay)
+        outW.append(W2); outm.append(m2); outv.append(v2); outg.append(g)
+    return outW, outm, outv, outg
