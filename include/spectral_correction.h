@@ -1,0 +1,192 @@
+/*
+ * spectral_correction.h - C ABI of the B200 (sm_100a) spectral-correction optimizer step.
+ *
+ * The library implements the per-matrix update of "Anchor Priors and Spectral Correction"
+ * (Section 3.2; Algorithm 1 lines 7-14):
+ *
+ *   on anchor arrival   M_anc <- beta_anc * M_anc + (1 - beta_anc) * G_anc            (Eq. 1)
+ *                       M_anc ~= U diag(s) V^T, leading `rank` triplets               (the SVD of Section 3.2)
+ *                       d_i = s_i / (s_i + tau_p)                                     (Eq. 2)
+ *   every step          X = U^T g V,  g = G_mask (times 1/keep_ratio unless prescaled)
+ *                       G_filt = U diag(d) X diag(d) V^T                              (two-sided application)
+ *                       G_proj = alpha * g + (1 - alpha) * G_filt                     (Eq. 3)
+ *                       AdamW(W, m, v; G_proj)                                        (Algorithm 1 line 13)
+ *
+ * Conventions
+ *   - A weight matrix W is rows x cols = out features x in features, row-major, contiguous.
+ *     Gradients, AdamW moments and the anchor momentum have the same shape and layout.
+ *   - "device" pointers are CUDA global-memory addresses of the current device; "host" pointers are
+ *     ordinary process memory.  Pointer ARRAYS (one entry per matrix) always live in host memory and
+ *     are read before the call returns; the buffers they point to are device memory unless a function
+ *     says otherwise, are owned by the caller, must be 16-byte aligned and must stay valid until the
+ *     work queued on the plan's stream has finished.
+ *   - All calls queue work on the stream given to sc_plan_create and return without waiting for it.
+ *   - Every function returns an sc_status; nothing throws or aborts across this boundary.
+ *     Conditions the device detects (a bounded wait that ran out, non-finite values) are latched in a
+ *     status word that sc_get_device_status reads back.
+ *   - The library never allocates device memory: the caller passes one workspace blob of at least
+ *     sc_plan_workspace_bytes() bytes (256-byte aligned), which holds the anchor momentum, the cached
+ *     basis and scratch.  The small host-side plan object (and pinned staging for pointer tables) is
+ *     allocated by sc_plan_create and freed by sc_plan_destroy.
+ */
+#ifndef SPECTRAL_CORRECTION_H_
+#define SPECTRAL_CORRECTION_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define SC_API
+#else
+#define SC_API __attribute__((visibility("default")))
+#endif
+
+typedef struct sc_plan sc_plan;
+
+typedef enum sc_status {
+  SC_OK = 0,
+  SC_WARN_NO_ANCHOR = 1,        /* step ran with an empty basis: G_proj = alpha * g (no anchor has arrived yet) */
+  SC_ERR_INVALID_ARG = -1,
+  SC_ERR_SHAPE = -2,
+  SC_ERR_DTYPE = -3,
+  SC_ERR_ALIGNMENT = -4,
+  SC_ERR_WORKSPACE = -5,
+  SC_ERR_STALE_TAG = -6,        /* anchor step tag older than the last one accepted */
+  SC_ERR_CUDA = -7,
+  SC_ERR_UNSUPPORTED_ARCH = -8, /* the current device is not sm_100 */
+  SC_ERR_TIMEOUT = -9,          /* a bounded device-side wait ran out */
+  SC_ERR_NONFINITE = -10,
+  SC_ERR_TOO_LARGE = -11
+} sc_status;
+
+typedef enum sc_dtype { SC_DTYPE_BF16 = 0, SC_DTYPE_FP32 = 1 } sc_dtype;
+
+/* Which kernels do the large contractions. AUTO: tcgen05 tensor-core kernels for bf16 gradients on
+ * shapes they support (cols % 8 == 0), plain fp32 CUDA-core kernels otherwise (fp32 gradients, odd shapes). */
+typedef enum sc_engine { SC_ENGINE_AUTO = 0, SC_ENGINE_SIMT = 1 } sc_engine;
+
+typedef struct sc_shape {
+  int64_t rows; /* m, out features */
+  int64_t cols; /* n, in features  */
+} sc_shape;
+
+/* Hyper-parameters (Algorithm 1 "Require" line, plus AdamW's and the basis iteration's). Plain data. */
+typedef struct sc_hparams {
+  float alpha;          /* blend weight of the raw masked gradient, Eq. 3 */
+  float tau_p;          /* spectral damping, Eq. 2 */
+  float beta_anc;       /* anchor EMA decay, Eq. 1 */
+  float lr;             /* AdamW */
+  float beta1;
+  float beta2;
+  float eps;
+  float weight_decay;   /* decoupled */
+  float max_grad_norm;  /* global-norm clip of G_proj over all matrices; <= 0 disables */
+  int32_t grads_prescaled; /* 1: masked gradients already carry the 1/keep_ratio rescale; 0: the step applies it */
+  int32_t grad_dtype;      /* sc_dtype of masked and anchor gradients */
+  int32_t sketch_width;    /* l: columns of the randomized range finder, rank <= l <= 256; 0 means l = rank */
+  int32_t power_iters;     /* q: subspace (power) iterations of the range finder, 0..16 */
+  int32_t engine;          /* sc_engine */
+  int32_t collect_stats;   /* 1: also accumulate ||g||^2 every step so that sc_get_stats can report eta_r and ||G_proj|| */
+  uint64_t seed;           /* key of the counter-based Rademacher sketch */
+} sc_hparams;
+
+/* AdamW state handed to sc_correct_and_step. Arrays of n_mats device pointers, held in host memory. */
+typedef struct sc_opt_state {
+  void* const* exp_avg;     /* m: fp32 rows x cols, updated in place */
+  void* const* exp_avg_sq;  /* v: fp32 rows x cols, updated in place */
+  void* const* params_bf16; /* optional bf16 copy of the updated weights (written only); NULL or NULL entries = none */
+} sc_opt_state;
+
+/* Per-matrix statistics of the last sc_correct_and_step (by-products of the projection). */
+typedef struct sc_mat_stats {
+  float g_sqnorm;     /* ||g||_F^2, g = rescaled masked gradient */
+  float x_sqnorm;     /* ||U^T g V||_F^2 ; eta_r = x_sqnorm / g_sqnorm (alignment diagnostic of the appendix) */
+  float gproj_sqnorm; /* ||G_proj||_F^2 before clipping, closed form from g_sqnorm and X */
+  float r_eff;        /* sum_i d_i^2 (Lemma 2's effective rank) */
+} sc_mat_stats;
+
+/* Fill *hp with defaults: alpha 0.3, tau_p 1e-3, beta_anc 0.9, lr 2e-5, betas (0.9, 0.999), eps 1e-8,
+ * weight_decay 0, no clipping, grads prescaled, bf16 gradients, l = rank, q = 1, engine AUTO, no stats, seed 0.
+ * (alpha, tau_p, lr, betas: the paper's defaults; the others are not given there.) */
+SC_API sc_status sc_hparams_default(sc_hparams* hp);
+
+/* Bytes of device workspace a plan for these shapes needs. Host-only, no CUDA calls. Returns 0 on invalid input. */
+SC_API size_t sc_plan_workspace_bytes(const sc_shape* shapes, int n_mats, int rank, const sc_hparams* hp);
+
+/* sc_plan_create - validate, lay out the workspace, zero the anchor momentum (Algorithm 1 line 2: M_anc <- 0).
+ *   out            host: receives the plan handle
+ *   shapes         host: n_mats entries
+ *   rank           r >= 0, r <= min(rows, cols) of every matrix, r <= 256; 0 = no basis (G_proj = alpha g)
+ *   keep_ratio     in (0, 1]; 1 - p_mask. Used for the 1/keep rescale when hp->grads_prescaled == 0.
+ *   workspace      device: caller-owned blob, 256-byte aligned, kept alive until sc_plan_destroy
+ *   stream         a cudaStream_t (as void*), NULL = default stream; all later calls queue work on it
+ * Errors: INVALID_ARG, SHAPE, DTYPE, ALIGNMENT, WORKSPACE (too small), UNSUPPORTED_ARCH, CUDA. */
+SC_API sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int rank, float keep_ratio,
+                                const sc_hparams* hp, void* workspace, size_t workspace_bytes, void* stream);
+
+SC_API sc_status sc_plan_destroy(sc_plan* plan);
+
+/* sc_anchor_update - an anchor gradient has arrived (Algorithm 1 lines 7-9 and the SVD of line 11).
+ *   anchor_grads   host array of n_mats device pointers (grad_dtype, rows x cols); a NULL entry means no anchor
+ *                  gradient arrived for that matrix: its momentum and basis are left as they are.
+ *   step_tag       fast-circuit step at which the anchor's weight snapshot was taken; must not decrease.
+ *                  It does not enter the arithmetic (the paper applies no staleness weighting); it is
+ *                  recorded so that staleness = step - tag can be reported.
+ * For each arrived matrix: Eq. 1, then the rank-r basis of the new momentum by randomized subspace iteration
+ * (sketch width l, q power iterations), then Eq. 2. The basis is cached until the next arrival. */
+SC_API sc_status sc_anchor_update(sc_plan* plan, const void* const* anchor_grads, int64_t step_tag);
+
+/* sc_correct_and_step - one fast-circuit optimizer step over all matrices (Algorithm 1 lines 10-13).
+ *   masked_grads   host array of n_mats device pointers (grad_dtype, rows x cols), read only
+ *   params         host array of n_mats device pointers, fp32 master weights, updated in place
+ *   state          AdamW moments (updated in place) and the optional bf16 weight copy
+ *   step           optimizer step count t >= 1 (AdamW bias correction; staleness report)
+ * Returns SC_WARN_NO_ANCHOR (still a completed step) when no anchor has arrived yet. */
+SC_API sc_status sc_correct_and_step(sc_plan* plan, const void* const* masked_grads, void* const* params,
+                                     const sc_opt_state* state, int64_t step);
+
+/* ---- inspection / test hooks ------------------------------------------------------------------------- */
+
+/* Copy matrix `mat`'s cached basis into caller device buffers (any may be NULL):
+ * U rows x rank fp32 row-major, s rank fp32, V cols x rank fp32 row-major. Queued on the plan's stream. */
+SC_API sc_status sc_export_basis(sc_plan* plan, int mat, void* U_dev, void* s_dev, void* V_dev);
+
+/* Replace matrix `mat`'s cached basis (same layouts; columns must be orthonormal, s descending) and
+ * recompute Eq. 2 and the operand copies the step kernels read. Marks the matrix as having an anchor. */
+SC_API sc_status sc_import_basis(sc_plan* plan, int mat, const void* U_dev, const void* s_dev, const void* V_dev);
+
+/* Copy the anchor momentum (rows x cols fp32) to / from a caller device buffer. */
+SC_API sc_status sc_export_anchor_momentum(sc_plan* plan, int mat, void* M_dev);
+SC_API sc_status sc_import_anchor_momentum(sc_plan* plan, int mat, const void* M_dev);
+
+/* Copy the first rows x width block of the Rademacher sketch (fp32, row-major, entries +-1) to a device buffer. */
+SC_API sc_status sc_export_sketch(sc_plan* plan, int64_t rows, int width, void* Omega_dev);
+
+/* Ask the next steps to also write G_proj (after clipping, fp32 rows x cols) for each matrix.
+ * gproj_out: host array of n_mats device pointers (NULL entries skipped), or NULL to switch it off. */
+SC_API sc_status sc_set_debug_gproj_out(sc_plan* plan, void* const* gproj_out);
+
+/* Wait for the plan's stream, then copy the per-matrix statistics of the last step into stats[n_mats] (host)
+ * and the clip factor applied into *clip (host, may be NULL). */
+SC_API sc_status sc_get_stats(sc_plan* plan, sc_mat_stats* stats, float* clip);
+
+/* Wait for the plan's stream and return the latched device status (SC_OK, SC_ERR_TIMEOUT, SC_ERR_NONFINITE), then clear it. */
+SC_API sc_status sc_get_device_status(sc_plan* plan);
+
+/* Step tag of the last accepted anchor (-1 if none) and number of matrices that have a basis. */
+SC_API sc_status sc_get_anchor_info(sc_plan* plan, int64_t* last_tag, int* n_with_basis);
+
+/* 1 if the tensor-core (tcgen05) kernels serve this plan, 0 if the fp32 CUDA-core kernels do. */
+SC_API int sc_plan_uses_tensor_cores(const sc_plan* plan);
+
+SC_API const char* sc_status_string(sc_status s);
+SC_API int sc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECTRAL_CORRECTION_H_ */

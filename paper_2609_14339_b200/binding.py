@@ -1,0 +1,248 @@
+"""ctypes binding of libspectral_correction.so: same names as the C ABI, argument marshalling only.
+
+PyTorch is used for device memory and streams; every arithmetic step of the path runs in the library's
+kernels.  There is no CPU fallback: if the library is missing or cannot be loaded, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_NAME = "libspectral_correction.so"
+
+SC_OK = 0
+SC_WARN_NO_ANCHOR = 1
+SC_DTYPE_BF16, SC_DTYPE_FP32 = 0, 1
+SC_ENGINE_AUTO, SC_ENGINE_SIMT = 0, 1
+
+
+class SCError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (%d)" % (where, status_string(status), status))
+
+
+class Shape(C.Structure):
+    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64)]
+
+
+class Hparams(C.Structure):
+    """Mirror of sc_hparams."""
+    _fields_ = [("alpha", C.c_float), ("tau_p", C.c_float), ("beta_anc", C.c_float), ("lr", C.c_float),
+                ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float), ("weight_decay", C.c_float),
+                ("max_grad_norm", C.c_float), ("grads_prescaled", C.c_int32), ("grad_dtype", C.c_int32),
+                ("sketch_width", C.c_int32), ("power_iters", C.c_int32), ("engine", C.c_int32),
+                ("collect_stats", C.c_int32), ("seed", C.c_uint64)]
+
+    @classmethod
+    def default(cls, **kw) -> "Hparams":
+        hp = cls()
+        _check(load_library().sc_hparams_default(C.byref(hp)), "sc_hparams_default")
+        for k, v in kw.items():
+            if not hasattr(hp, k):
+                raise AttributeError(k)
+            setattr(hp, k, v)
+        return hp
+
+
+class OptState(C.Structure):
+    _fields_ = [("exp_avg", C.POINTER(C.c_void_p)), ("exp_avg_sq", C.POINTER(C.c_void_p)),
+                ("params_bf16", C.POINTER(C.c_void_p))]
+
+
+class MatStats(C.Structure):
+    _fields_ = [("g_sqnorm", C.c_float), ("x_sqnorm", C.c_float), ("gproj_sqnorm", C.c_float), ("r_eff", C.c_float)]
+
+
+# every symbol include/spectral_correction.h declares: name -> (restype, argtypes)
+_VP, _VPP = C.c_void_p, C.POINTER(C.c_void_p)
+EXPORTS = {
+    "sc_hparams_default": (C.c_int, [C.POINTER(Hparams)]),
+    "sc_plan_workspace_bytes": (C.c_size_t, [C.POINTER(Shape), C.c_int, C.c_int, C.POINTER(Hparams)]),
+    "sc_plan_create": (C.c_int, [C.POINTER(_VP), C.POINTER(Shape), C.c_int, C.c_int, C.c_float, C.POINTER(Hparams),
+                                 _VP, C.c_size_t, _VP]),
+    "sc_plan_destroy": (C.c_int, [_VP]),
+    "sc_anchor_update": (C.c_int, [_VP, _VPP, C.c_int64]),
+    "sc_correct_and_step": (C.c_int, [_VP, _VPP, _VPP, C.POINTER(OptState), C.c_int64]),
+    "sc_export_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
+    "sc_import_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
+    "sc_export_anchor_momentum": (C.c_int, [_VP, C.c_int, _VP]),
+    "sc_import_anchor_momentum": (C.c_int, [_VP, C.c_int, _VP]),
+    "sc_export_sketch": (C.c_int, [_VP, C.c_int64, C.c_int, _VP]),
+    "sc_set_debug_gproj_out": (C.c_int, [_VP, _VPP]),
+    "sc_get_stats": (C.c_int, [_VP, C.POINTER(MatStats), C.POINTER(C.c_float)]),
+    "sc_get_device_status": (C.c_int, [_VP]),
+    "sc_get_anchor_info": (C.c_int, [_VP, C.POINTER(C.c_int64), C.POINTER(C.c_int)]),
+    "sc_plan_uses_tensor_cores": (C.c_int, [_VP]),
+    "sc_status_string": (C.c_char_p, [C.c_int]),
+    "sc_version": (C.c_int, []),
+}
+
+_lib = None
+
+
+def lib_path() -> str:
+    return os.path.join(_HERE, _LIB_NAME)
+
+
+def load_library():
+    """dlopen the in-tree library and declare prototypes. Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = lib_path()
+    if not os.path.exists(path):
+        raise RuntimeError("%s is missing: run `python -m paper_2609_14339_b200.build` "
+                           "(there is no CPU fallback)" % path)
+    lib = C.CDLL(path)
+    for name, (res, args) in EXPORTS.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().sc_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str, allow=(SC_OK,)) -> int:
+    if status not in allow:
+        raise SCError(status, where)
+    return status
+
+
+def _ptr_array(tensors: Optional[Sequence], n: int, allow_none: bool):
+    if tensors is None:
+        return None
+    if len(tensors) != n:
+        raise ValueError("expected %d tensors, got %d" % (n, len(tensors)))
+    arr = (C.c_void_p * n)()
+    for i, t in enumerate(tensors):
+        if t is None:
+            if not allow_none:
+                raise ValueError("tensor %d is None" % i)
+            arr[i] = None
+        else:
+            if not t.is_cuda or not t.is_contiguous():
+                raise ValueError("tensor %d must be a contiguous CUDA tensor" % i)
+            arr[i] = t.data_ptr()
+    return arr
+
+
+class Plan:
+    """Owns a workspace tensor and an sc_plan handle; methods mirror the C entry points one to one."""
+
+    def __init__(self, shapes, rank: int, keep_ratio: float, hp: Optional[Hparams] = None, stream=None, device="cuda:0"):
+        import torch
+        self._torch = torch
+        self.lib = load_library()
+        self.hp = hp if hp is not None else Hparams.default()
+        self.shapes = [(int(m), int(n)) for m, n in shapes]
+        self.n_mats = len(self.shapes)
+        self.rank = int(rank)
+        self.device = torch.device(device)
+        arr = (Shape * self.n_mats)(*[Shape(m, n) for m, n in self.shapes])
+        need = self.lib.sc_plan_workspace_bytes(arr, self.n_mats, self.rank, C.byref(self.hp))
+        if need == 0:
+            raise SCError(-1, "sc_plan_workspace_bytes")
+        self.workspace_bytes = int(need)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
+            base = (self.workspace.data_ptr() + 255) // 256 * 256
+            self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+            handle = C.c_void_p()
+            _check(self.lib.sc_plan_create(C.byref(handle), arr, self.n_mats, self.rank, float(keep_ratio),
+                                           C.byref(self.hp), base, need, self.stream.cuda_stream), "sc_plan_create")
+        self.handle = handle
+        self._keep = []
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.sc_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- the three calls of the method -------------------------------------------------------------
+    def anchor_update(self, anchor_grads: Sequence, step_tag: int) -> int:
+        arr = _ptr_array(anchor_grads, self.n_mats, True)
+        return _check(self.lib.sc_anchor_update(self.handle, arr, int(step_tag)), "sc_anchor_update")
+
+    def correct_and_step(self, masked_grads, params, exp_avg, exp_avg_sq, step: int, params_bf16=None) -> int:
+        n = self.n_mats
+        st = OptState(_ptr_array(exp_avg, n, False), _ptr_array(exp_avg_sq, n, False),
+                      _ptr_array(params_bf16, n, True) if params_bf16 is not None else None)
+        return _check(self.lib.sc_correct_and_step(self.handle, _ptr_array(masked_grads, n, False),
+                                                   _ptr_array(params, n, False), C.byref(st), int(step)),
+                      "sc_correct_and_step", allow=(SC_OK, SC_WARN_NO_ANCHOR))
+
+    # ---- inspection --------------------------------------------------------------------------------
+    def export_basis(self, mat: int):
+        t = self._torch
+        m, n = self.shapes[mat]
+        r = self.rank
+        U = t.empty((m, r), dtype=t.float32, device=self.device)
+        s = t.empty((r,), dtype=t.float32, device=self.device)
+        V = t.empty((n, r), dtype=t.float32, device=self.device)
+        if r > 0:
+            _check(self.lib.sc_export_basis(self.handle, mat, U.data_ptr(), s.data_ptr(), V.data_ptr()), "sc_export_basis")
+        return U, s, V
+
+    def import_basis(self, mat: int, U, s, V):
+        t = self._torch
+        U = U.to(self.device, t.float32).contiguous(); s = s.to(self.device, t.float32).contiguous()
+        V = V.to(self.device, t.float32).contiguous()
+        m, n = self.shapes[mat]
+        assert U.shape == (m, self.rank) and V.shape == (n, self.rank) and s.shape == (self.rank,)
+        _check(self.lib.sc_import_basis(self.handle, mat, U.data_ptr(), s.data_ptr(), V.data_ptr()), "sc_import_basis")
+        self._torch.cuda.current_stream(self.device).wait_stream(self.stream)
+        self.stream.synchronize()
+
+    def export_anchor_momentum(self, mat: int):
+        t = self._torch
+        M = t.empty(self.shapes[mat], dtype=t.float32, device=self.device)
+        _check(self.lib.sc_export_anchor_momentum(self.handle, mat, M.data_ptr()), "sc_export_anchor_momentum")
+        return M
+
+    def import_anchor_momentum(self, mat: int, M):
+        M = M.to(self.device, self._torch.float32).contiguous()
+        assert tuple(M.shape) == self.shapes[mat]
+        _check(self.lib.sc_import_anchor_momentum(self.handle, mat, M.data_ptr()), "sc_import_anchor_momentum")
+        self.stream.synchronize()
+
+    def export_sketch(self, rows: int, width: int):
+        t = self._torch
+        Om = t.empty((rows, width), dtype=t.float32, device=self.device)
+        _check(self.lib.sc_export_sketch(self.handle, rows, width, Om.data_ptr()), "sc_export_sketch")
+        return Om
+
+    def set_debug_gproj_out(self, tensors):
+        self._keep = list(tensors) if tensors is not None else []
+        arr = _ptr_array(tensors, self.n_mats, True) if tensors is not None else None
+        _check(self.lib.sc_set_debug_gproj_out(self.handle, arr), "sc_set_debug_gproj_out")
+
+    def get_stats(self):
+        arr = (MatStats * self.n_mats)()
+        clip = C.c_float()
+        _check(self.lib.sc_get_stats(self.handle, arr, C.byref(clip)), "sc_get_stats")
+        return [dict(g_sqnorm=a.g_sqnorm, x_sqnorm=a.x_sqnorm, gproj_sqnorm=a.gproj_sqnorm, r_eff=a.r_eff)
+                for a in arr], clip.value
+
+    def get_device_status(self) -> int:
+        return int(self.lib.sc_get_device_status(self.handle))
+
+    def get_anchor_info(self):
+        tag, k = C.c_int64(), C.c_int()
+        _check(self.lib.sc_get_anchor_info(self.handle, C.byref(tag), C.byref(k)), "sc_get_anchor_info")
+        return tag.value, k.value
+
+    def uses_tensor_cores(self) -> bool:
+        return bool(self.lib.sc_plan_uses_tensor_cores(self.handle))

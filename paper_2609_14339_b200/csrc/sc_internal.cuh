@@ -1,0 +1,170 @@
+// Internal declarations shared by the translation units of the spectral-correction library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "spectral_correction.h"
+
+namespace sc {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kMaxRank = 256;
+constexpr int kStatsFloats = 8;        // per-matrix statistics slot
+constexpr int kSqnormBlocks = 128;     // partial sums of ||G||^2 per matrix (fixed-order reduction)
+constexpr int kStagingSlots = 4;       // ring of pinned upload buffers for the per-call pointer table
+
+// Device status word bits (latched, read by sc_get_device_status).
+constexpr unsigned kDevTimeout = 1u;
+constexpr unsigned kDevNonfinite = 2u;
+
+// One record per weight matrix, resident in device memory (the "table"). The first block of fields is
+// fixed at plan creation (addresses inside the workspace); the second block is rewritten by every call.
+struct MatDev {
+  // cached basis and anchor momentum (persistent)
+  float* Manc;   // m x n       anchor momentum, Eq. 1
+  float* U;      // m x rp      left basis, fp32, columns >= rank are zero
+  float* V;      // n x rp      right basis
+  float* sv;     // rp          singular values
+  float* d;      // rp          filter weights, Eq. 2
+  bf16* Uhi;     // m x rp      bf16 split of U  (U ~= Uhi + Ulo), K-major MMA operand
+  bf16* Ulo;
+  bf16* Vthi;    // rp x n      bf16 split of V^T, K-major MMA operand
+  bf16* Vtlo;
+  // per-step scratch (slot shared by matrices of different shape classes)
+  float* T;      // ksplit x m x rp   T = G V (partials)
+  float* X;      // rp x rp     X = U^T G V (unscaled)
+  float* Xs;     // rp x rp     (1-alpha) * scale * D X D
+  float* Ct;     // n x rp      C^T = V Xs^T, fp32
+  bf16* Cthi;    // n x rp      bf16 split of C^T
+  bf16* Ctlo;
+  float* sqpart; // kSqnormBlocks partial sums of ||G||^2
+  float* stats;  // kStatsFloats
+  // anchor-update scratch (slot)
+  float* Y;      // m x lp
+  float* Y2;     // m x lp
+  float* Z;      // n x lp
+  float* Z2;     // n x lp
+  float* gram;   // lp x lp
+  float* rmat;   // lp x lp   Cholesky factor (upper), first pass
+  float* rmat2;  // lp x lp   second pass
+  float* rinv;   // lp x lp   inverse of the factor
+  float* racc;   // lp x lp   rmat2 * rmat
+  float* jk;     // lp x lp   Jacobi work: columns being orthogonalised
+  float* jv;     // lp x lp   accumulated rotations
+  float* ub;     // lp x rp   left singular vectors of the small factor (selected, sorted)
+  float* wb;     // lp x rp   right singular vectors
+  const float* omega_t;  // lp x n  Rademacher sketch, transposed (shared by a shape class)
+  // per call
+  const void* G;      // masked gradient
+  const void* Ganc;   // anchor gradient
+  float* W;           // fp32 master weights
+  float* m1;          // AdamW first moment
+  float* m2;          // AdamW second moment
+  bf16* Wb;           // optional bf16 weight copy
+  float* gproj_dbg;   // optional G_proj output
+  int m, n;
+  int pad0, pad1;
+};
+
+// All matrices of one shape; kernels are launched once per class with blockIdx.z = instance.
+struct ShapeClass {
+  int64_t m = 0, n = 0;
+  std::vector<int> mats;   // matrix ids, in plan order
+  float* omega_t = nullptr;
+  int* idx_all = nullptr;  // device: mats[]
+  int* idx_dyn = nullptr;  // device: subset list written per call (anchor arrivals)
+  bool tensor = false;     // served by the tcgen05 kernels
+  int ksplit = 1;
+  void* tmaps = nullptr;   // device: per-instance tensor maps (tensor engine only)
+};
+
+struct StepScalars {       // scalars of one step, passed by value to kernels
+  float alpha_s;           // alpha * scale
+  float beta1, beta2, one_m_beta1, one_m_beta2;
+  float step_size;         // lr / (1 - beta1^t)
+  float inv_sqrt_bc2;      // 1 / sqrt(1 - beta2^t)
+  float eps;
+  float decay;             // 1 - lr * weight_decay
+};
+
+}  // namespace sc
+
+struct sc_plan {
+  int n_mats = 0, rank = 0, rp = 0, l = 0, lp = 0, q = 0;
+  float keep = 1.f;
+  sc_hparams hp{};
+  cudaStream_t stream = nullptr;
+  std::vector<sc_shape> shapes;
+  std::vector<sc::ShapeClass> classes;
+  std::vector<int> class_of;       // matrix -> class
+  std::vector<int> inst_of;        // matrix -> instance index inside its class
+  std::vector<sc::MatDev> host_tab;   // host mirror of the device table
+  std::vector<sc::MatDev> last_uploaded;
+  sc::MatDev* dev_tab = nullptr;
+  char* staging = nullptr;            // pinned, kStagingSlots * staging_bytes
+  size_t staging_bytes = 0;
+  cudaEvent_t staging_ev[sc::kStagingSlots]{};
+  int staging_next = 0;
+  float* clip_dev = nullptr;          // clip factor applied to G_proj
+  unsigned* status_dev = nullptr;     // latched device status bits
+  float* stats_dev = nullptr;         // n_mats * kStatsFloats
+  char* ws = nullptr;
+  size_t ws_bytes = 0;
+  int64_t last_tag = -1;
+  std::vector<char> has_basis;
+  std::vector<void*> dbg_out;
+  bool table_dirty = true;
+  bool tensor_any = false;
+};
+
+namespace sc {
+
+// ---- host helpers (sc_plan.cu) -------------------------------------------------------------------------
+sc_status upload_table(sc_plan* p);
+sc_status cuda_ok(cudaError_t e);
+
+// ---- CUDA-core kernels (sc_simt.cu) ----------------------------------------------------------------------
+struct GemmArgs {
+  const MatDev* tab;
+  const int* idx;
+  int offA, offB, offC;    // byte offsets of the pointer fields inside MatDev
+  int M, N, K;
+  int lda, ldb, ldc;
+  int transA, transB;
+  int a_bf16;              // A holds bf16 (gradients) instead of fp32
+  float alpha;
+};
+void launch_gemm(const GemmArgs& a, int count, cudaStream_t s);
+void launch_epilogue_simt(const MatDev* tab, const int* idx, int count, int m, int n, int rp, int g_bf16,
+                          const StepScalars& sc, const float* clip, cudaStream_t s);
+void launch_ema(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, float beta, cudaStream_t s);
+void launch_sketch(float* omega_t, int lp, int l, int64_t n, uint64_t seed, cudaStream_t s);
+void launch_sketch_rowmajor(float* omega, int64_t rows, int width, uint64_t seed, cudaStream_t s);
+void launch_chol(const MatDev* tab, const int* idx, int count, int lp, int offR, cudaStream_t s);
+void launch_jacobi(const MatDev* tab, const int* idx, int count, int lp, int rp, int rank, float tau_p, cudaStream_t s);
+void launch_filter_weights(const MatDev* tab, const int* idx, int count, int rp, int rank, float tau_p, cudaStream_t s);
+void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int n, int rp, cudaStream_t s);
+void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, cudaStream_t s);
+void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, float coef, float scale, float alpha,
+               cudaStream_t s);
+void launch_split_ct(const MatDev* tab, const int* idx, int count, int n, int rp, cudaStream_t s);
+void launch_clip(const MatDev* tab, int n_mats, float max_norm, float* clip, cudaStream_t s);
+void launch_pad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, int cols_dst, cudaStream_t s);
+void launch_unpad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, cudaStream_t s);
+void launch_reduce_partials(const MatDev* tab, const int* idx, int count, int64_t numel, int ksplit, cudaStream_t s);
+
+// ---- tensor-core kernels (sc_tc.cu) -----------------------------------------------------------------------
+bool tc_shape_supported(int64_t m, int64_t n, int rp);
+size_t tc_tmaps_bytes(int count);
+sc_status tc_init();   // resolves the driver entry point for tensor-map encoding
+sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_call_part);
+sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count);   // T = G V
+sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc);
+
+}  // namespace sc

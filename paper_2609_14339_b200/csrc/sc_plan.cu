@@ -1,0 +1,617 @@
+// Host side of the spectral-correction library: the C ABI, argument checks, workspace layout and the
+// order in which the kernels of one anchor arrival / one optimizer step are queued.
+#include <math.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "sc_internal.cuh"
+
+using namespace sc;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+inline int round_up_int(int x, int a) { return (x + a - 1) / a * a; }
+
+// Bump allocator over the workspace; with base == nullptr it only measures.
+struct Carver {
+  char* base;
+  size_t off = 0;
+  explicit Carver(char* b) : base(b) {}
+  template <typename T>
+  T* take(size_t count) {
+    off = align_up(off);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+struct Dims {
+  int rp, l, lp, q;
+};
+
+bool derive_dims(int rank, const sc_hparams* hp, Dims* d) {
+  if (rank < 0 || rank > kMaxRank) return false;
+  int l = hp->sketch_width > 0 ? hp->sketch_width : rank;
+  if (l < rank || l > kMaxRank) return false;
+  if (hp->power_iters < 0 || hp->power_iters > 16) return false;
+  d->rp = rank > 0 ? round_up_int(rank, 16) : 0;
+  d->l = l;
+  d->lp = rank > 0 ? round_up_int(l, 16) : 0;
+  d->q = hp->power_iters;
+  return true;
+}
+
+bool valid_hparams(const sc_hparams* hp) {
+  if (!hp) return false;
+  if (!(hp->alpha >= 0.f && hp->alpha <= 1.f)) return false;
+  if (!(hp->tau_p >= 0.f)) return false;
+  if (!(hp->beta_anc >= 0.f && hp->beta_anc < 1.f)) return false;
+  if (!(hp->beta1 >= 0.f && hp->beta1 < 1.f) || !(hp->beta2 >= 0.f && hp->beta2 < 1.f)) return false;
+  if (!(hp->eps >= 0.f) || !isfinite(hp->lr) || !(hp->weight_decay >= 0.f)) return false;
+  return true;
+}
+
+struct ClassKey {
+  int64_t m, n;
+};
+
+// Groups matrices by shape, in order of first appearance.
+void build_classes(const sc_shape* shapes, int n_mats, std::vector<ShapeClass>& classes, std::vector<int>& class_of,
+                   std::vector<int>& inst_of) {
+  class_of.assign(n_mats, -1);
+  inst_of.assign(n_mats, -1);
+  for (int i = 0; i < n_mats; ++i) {
+    int c = -1;
+    for (size_t k = 0; k < classes.size(); ++k)
+      if (classes[k].m == shapes[i].rows && classes[k].n == shapes[i].cols) { c = (int)k; break; }
+    if (c < 0) {
+      classes.emplace_back();
+      c = (int)classes.size() - 1;
+      classes[c].m = shapes[i].rows;
+      classes[c].n = shapes[i].cols;
+    }
+    class_of[i] = c;
+    inst_of[i] = (int)classes[c].mats.size();
+    classes[c].mats.push_back(i);
+  }
+}
+
+int choose_ksplit(const ShapeClass& c) {
+  const int64_t tiles = (c.m + 127) / 128 * (int64_t)c.mats.size();
+  int ks = 1;
+  while (ks < 8 && tiles * ks < 148 * 2 && c.n / (ks * 2) >= 1024) ks *= 2;
+  return ks;
+}
+
+// Lays the whole workspace out. With p->ws == nullptr nothing is dereferenced: it only measures.
+size_t layout(sc_plan* p, bool assign) {
+  Carver cv(assign ? p->ws : nullptr);
+  const int n_mats = p->n_mats, rp = p->rp, lp = p->lp;
+  MatDev* tab = cv.take<MatDev>(n_mats);
+  float* clip = cv.take<float>(1);
+  unsigned* status = cv.take<unsigned>(1);
+  float* stats = cv.take<float>((size_t)n_mats * kStatsFloats);
+  if (assign) { p->dev_tab = tab; p->clip_dev = clip; p->status_dev = status; p->stats_dev = stats; }
+  for (auto& c : p->classes) {
+    int* a = cv.take<int>(c.mats.size());
+    int* b = cv.take<int>(c.mats.size());
+    float* om = cv.take<float>((size_t)lp * c.n);
+    void* tm = c.tensor ? (void*)cv.take<char>(tc_tmaps_bytes((int)c.mats.size())) : nullptr;
+    if (assign) { c.idx_all = a; c.idx_dyn = b; c.omega_t = om; c.tmaps = tm; }
+  }
+  // persistent + per-step scratch, per matrix
+  for (int i = 0; i < n_mats; ++i) {
+    const size_t m = (size_t)p->shapes[i].rows, n = (size_t)p->shapes[i].cols;
+    const ShapeClass& c = p->classes[p->class_of[i]];
+    MatDev md;
+    memset(&md, 0, sizeof(md));
+    md.m = (int)m; md.n = (int)n;
+    md.Manc = cv.take<float>(m * n);
+    md.U = cv.take<float>(m * rp);
+    md.V = cv.take<float>(n * rp);
+    md.sv = cv.take<float>(rp);
+    md.d = cv.take<float>(rp);
+    md.X = cv.take<float>((size_t)rp * rp);
+    md.Xs = cv.take<float>((size_t)rp * rp);
+    md.T = cv.take<float>((size_t)c.ksplit * m * rp);
+    md.Ct = cv.take<float>(n * rp);
+    md.sqpart = cv.take<float>(kSqnormBlocks);
+    if (c.tensor) {
+      md.Uhi = cv.take<bf16>(m * rp); md.Ulo = cv.take<bf16>(m * rp);
+      md.Vthi = cv.take<bf16>(n * rp); md.Vtlo = cv.take<bf16>(n * rp);
+      md.Cthi = cv.take<bf16>(n * rp); md.Ctlo = cv.take<bf16>(n * rp);
+    }
+    md.stats = assign ? p->stats_dev + (size_t)i * kStatsFloats : nullptr;
+    md.omega_t = c.omega_t;
+    if (assign) p->host_tab[i] = md;
+  }
+  // anchor-update scratch: one region, reused by the classes in turn (slot = instance index)
+  cv.off = align_up(cv.off);
+  const size_t slot_base = cv.off;
+  size_t slot_max = 0;
+  for (auto& c : p->classes) {
+    Carver sv(assign ? p->ws + slot_base : nullptr);
+    for (size_t k = 0; k < c.mats.size(); ++k) {
+      const size_t m = (size_t)c.m, n = (size_t)c.n;
+      float* Y = sv.take<float>(m * lp); float* Y2 = sv.take<float>(m * lp);
+      float* Z = sv.take<float>(n * lp); float* Z2 = sv.take<float>(n * lp);
+      float* gram = sv.take<float>((size_t)lp * lp); float* rmat = sv.take<float>((size_t)lp * lp);
+      float* rmat2 = sv.take<float>((size_t)lp * lp); float* rinv = sv.take<float>((size_t)lp * lp);
+      float* racc = sv.take<float>((size_t)lp * lp); float* jk = sv.take<float>((size_t)lp * lp);
+      float* jv = sv.take<float>((size_t)lp * lp);
+      float* ub = sv.take<float>((size_t)lp * rp); float* wb = sv.take<float>((size_t)lp * rp);
+      if (assign) {
+        MatDev& md = p->host_tab[c.mats[k]];
+        md.Y = Y; md.Y2 = Y2; md.Z = Z; md.Z2 = Z2; md.gram = gram; md.rmat = rmat; md.rmat2 = rmat2;
+        md.rinv = rinv; md.racc = racc; md.jk = jk; md.jv = jv; md.ub = ub; md.wb = wb;
+      }
+    }
+    slot_max = std::max(slot_max, align_up(sv.off));
+  }
+  cv.off = slot_base + slot_max;
+  return align_up(cv.off);
+}
+
+void fill_plan_basics(sc_plan* p, const sc_shape* shapes, int n_mats, int rank, const sc_hparams* hp, const Dims& d) {
+  p->n_mats = n_mats; p->rank = rank; p->rp = d.rp; p->l = d.l; p->lp = d.lp; p->q = d.q;
+  p->hp = *hp;
+  p->shapes.assign(shapes, shapes + n_mats);
+  build_classes(shapes, n_mats, p->classes, p->class_of, p->inst_of);
+  for (auto& c : p->classes) {
+    c.tensor = hp->engine == SC_ENGINE_AUTO && hp->grad_dtype == SC_DTYPE_BF16 && rank > 0 &&
+               tc_shape_supported(c.m, c.n, d.rp);
+    c.ksplit = c.tensor ? choose_ksplit(c) : 1;
+    p->tensor_any = p->tensor_any || c.tensor;
+  }
+}
+
+sc_status check_shapes(const sc_shape* shapes, int n_mats, int rank) {
+  if (!shapes || n_mats <= 0 || n_mats > (1 << 20)) return SC_ERR_INVALID_ARG;
+  for (int i = 0; i < n_mats; ++i) {
+    if (shapes[i].rows <= 0 || shapes[i].cols <= 0) return SC_ERR_SHAPE;
+    if (shapes[i].rows > (1 << 24) || shapes[i].cols > (1 << 24)) return SC_ERR_TOO_LARGE;
+    if (rank > shapes[i].rows || rank > shapes[i].cols) return SC_ERR_SHAPE;
+  }
+  return SC_OK;
+}
+
+GemmArgs gemm(sc_plan* p, const int* idx, int offA, int offB, int offC, int M, int N, int K, int lda, int ldb, int ldc,
+              int tA, int tB, int a_bf16 = 0) {
+  GemmArgs a{};
+  a.tab = p->dev_tab; a.idx = idx; a.offA = offA; a.offB = offB; a.offC = offC;
+  a.M = M; a.N = N; a.K = K; a.lda = lda; a.ldb = ldb; a.ldc = ldc; a.transA = tA; a.transB = tB;
+  a.a_bf16 = a_bf16; a.alpha = 1.f;
+  return a;
+}
+
+#define OFF(f) ((int)offsetof(MatDev, f))
+
+// Q <- orth(Y) by two rounds of Cholesky QR; Y (rows x lp) is overwritten, tmp is scratch of the same size.
+// keepR: leave the two factors in rmat / rmat2 (and their product in racc) for the caller.
+void cholqr2(sc_plan* p, const int* idx, int cnt, int offY, int offTmp, int rows, bool keepR) {
+  const int lp = p->lp;
+  cudaStream_t s = p->stream;
+  launch_gemm(gemm(p, idx, offY, offY, OFF(gram), lp, lp, rows, lp, lp, lp, 1, 0), cnt, s);
+  launch_chol(p->dev_tab, idx, cnt, lp, OFF(rmat), s);
+  launch_gemm(gemm(p, idx, offY, OFF(rinv), offTmp, rows, lp, lp, lp, lp, lp, 0, 0), cnt, s);
+  launch_gemm(gemm(p, idx, offTmp, offTmp, OFF(gram), lp, lp, rows, lp, lp, lp, 1, 0), cnt, s);
+  launch_chol(p->dev_tab, idx, cnt, lp, OFF(rmat2), s);
+  launch_gemm(gemm(p, idx, offTmp, OFF(rinv), offY, rows, lp, lp, lp, lp, lp, 0, 0), cnt, s);
+  if (keepR) launch_gemm(gemm(p, idx, OFF(rmat2), OFF(rmat), OFF(racc), lp, lp, lp, lp, lp, lp, 0, 0), cnt, s);
+}
+
+// Rebuild d (Eq. 2) and the bf16 operand copies of one matrix list after its U, s, V changed.
+void refresh_operands(sc_plan* p, const ShapeClass& c, const int* idx, int cnt) {
+  if (c.tensor) launch_split_basis(p->dev_tab, idx, cnt, (int)c.m, (int)c.n, p->rp, p->stream);
+}
+
+sc_status check_ptr_array(const void* const* arr, int n, bool allow_null_entries) {
+  if (!arr) return SC_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    if (!arr[i]) { if (allow_null_entries) continue; return SC_ERR_INVALID_ARG; }
+    if (reinterpret_cast<uintptr_t>(arr[i]) & 15u) return SC_ERR_ALIGNMENT;
+  }
+  return SC_OK;
+}
+
+}  // namespace
+
+namespace sc {
+
+sc_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? SC_OK : SC_ERR_CUDA; }
+
+// Copies the host mirror of the table to the device if it changed since the last upload. The copy goes
+// through a ring of pinned buffers so that a later call never overwrites bytes an earlier, still queued
+// copy has yet to read.
+sc_status upload_table(sc_plan* p) {
+  const size_t bytes = (size_t)p->n_mats * sizeof(MatDev);
+  if (!p->table_dirty && p->last_uploaded.size() == p->host_tab.size() &&
+      memcmp(p->last_uploaded.data(), p->host_tab.data(), bytes) == 0)
+    return SC_OK;
+  const int slot = p->staging_next;
+  p->staging_next = (slot + 1) % kStagingSlots;
+  if (cudaEventSynchronize(p->staging_ev[slot]) != cudaSuccess) return SC_ERR_CUDA;
+  char* buf = p->staging + (size_t)slot * p->staging_bytes;
+  memcpy(buf, p->host_tab.data(), bytes);
+  if (cudaMemcpyAsync(p->dev_tab, buf, bytes, cudaMemcpyHostToDevice, p->stream) != cudaSuccess) return SC_ERR_CUDA;
+  if (cudaEventRecord(p->staging_ev[slot], p->stream) != cudaSuccess) return SC_ERR_CUDA;
+  p->last_uploaded = p->host_tab;
+  p->table_dirty = false;
+  return SC_OK;
+}
+
+}  // namespace sc
+
+// ============================================================================================ ABI
+
+extern "C" {
+
+sc_status sc_hparams_default(sc_hparams* hp) {
+  if (!hp) return SC_ERR_INVALID_ARG;
+  memset(hp, 0, sizeof(*hp));
+  hp->alpha = 0.3f; hp->tau_p = 1e-3f; hp->beta_anc = 0.9f;
+  hp->lr = 2e-5f; hp->beta1 = 0.9f; hp->beta2 = 0.999f; hp->eps = 1e-8f; hp->weight_decay = 0.f;
+  hp->max_grad_norm = 0.f; hp->grads_prescaled = 1; hp->grad_dtype = SC_DTYPE_BF16;
+  hp->sketch_width = 0; hp->power_iters = 1; hp->engine = SC_ENGINE_AUTO; hp->collect_stats = 0; hp->seed = 0;
+  return SC_OK;
+}
+
+size_t sc_plan_workspace_bytes(const sc_shape* shapes, int n_mats, int rank, const sc_hparams* hp) {
+  Dims d;
+  if (!valid_hparams(hp) || check_shapes(shapes, n_mats, rank) != SC_OK || !derive_dims(rank, hp, &d)) return 0;
+  sc_plan tmp;
+  fill_plan_basics(&tmp, shapes, n_mats, rank, hp, d);
+  tmp.ws = nullptr;
+  return layout(&tmp, false);
+}
+
+sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int rank, float keep_ratio,
+                         const sc_hparams* hp, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!out) return SC_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!valid_hparams(hp)) return SC_ERR_INVALID_ARG;
+  if (!(keep_ratio > 0.f && keep_ratio <= 1.f)) return SC_ERR_INVALID_ARG;
+  if (hp->grad_dtype != SC_DTYPE_BF16 && hp->grad_dtype != SC_DTYPE_FP32) return SC_ERR_DTYPE;
+  if (hp->engine != SC_ENGINE_AUTO && hp->engine != SC_ENGINE_SIMT) return SC_ERR_INVALID_ARG;
+  sc_status st = check_shapes(shapes, n_mats, rank);
+  if (st != SC_OK) return st;
+  Dims d;
+  if (!derive_dims(rank, hp, &d)) return SC_ERR_INVALID_ARG;
+  if (!workspace) return SC_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) return SC_ERR_ALIGNMENT;
+
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SC_ERR_CUDA;
+  if (prop.major != 10) return SC_ERR_UNSUPPORTED_ARCH;
+
+  sc_plan* p = new (std::nothrow) sc_plan();
+  if (!p) return SC_ERR_INVALID_ARG;
+  fill_plan_basics(p, shapes, n_mats, rank, hp, d);
+  p->keep = keep_ratio;
+  p->stream = reinterpret_cast<cudaStream_t>(stream);
+  p->ws = nullptr;
+  const size_t need = layout(p, false);
+  if (workspace_bytes < need) { delete p; return SC_ERR_WORKSPACE; }
+  p->ws = static_cast<char*>(workspace);
+  p->ws_bytes = need;
+  p->host_tab.resize(n_mats);
+  p->has_basis.assign(n_mats, 0);
+  p->dbg_out.assign(n_mats, nullptr);
+  layout(p, true);
+  for (auto& c : p->classes)
+    for (int id : c.mats) p->host_tab[id].omega_t = c.omega_t;
+
+  if (p->tensor_any && tc_init() != SC_OK) { delete p; return SC_ERR_CUDA; }
+
+  cudaStream_t s = p->stream;
+  bool ok = cudaMemsetAsync(p->ws, 0, need, s) == cudaSuccess;
+  p->staging_bytes = align_up((size_t)n_mats * sizeof(MatDev));
+  ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&p->staging), p->staging_bytes * kStagingSlots,
+                           cudaHostAllocDefault) == cudaSuccess;
+  for (int i = 0; ok && i < kStagingSlots; ++i)
+    ok = cudaEventCreateWithFlags(&p->staging_ev[i], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) { sc_plan_destroy(p); return SC_ERR_CUDA; }
+  const float one = 1.f;
+  ok = cudaMemcpyAsync(p->clip_dev, &one, sizeof(float), cudaMemcpyHostToDevice, s) == cudaSuccess;
+  for (auto& c : p->classes) {
+    ok = ok && cudaMemcpyAsync(c.idx_all, c.mats.data(), c.mats.size() * sizeof(int), cudaMemcpyHostToDevice, s) ==
+                   cudaSuccess;
+    if (p->lp > 0) launch_sketch(c.omega_t, p->lp, p->l, c.n, p->hp.seed, s);
+    if (c.tensor && ok) ok = tc_encode_class(p, c, true, false) == SC_OK;
+  }
+  p->table_dirty = true;
+  ok = ok && upload_table(p) == SC_OK;
+  // The small host-to-device copies above read host memory that lives only in this call.
+  ok = ok && cudaStreamSynchronize(s) == cudaSuccess && cudaGetLastError() == cudaSuccess;
+  if (!ok) { sc_plan_destroy(p); return SC_ERR_CUDA; }
+  *out = p;
+  return SC_OK;
+}
+
+sc_status sc_plan_destroy(sc_plan* p) {
+  if (!p) return SC_ERR_INVALID_ARG;
+  cudaStreamSynchronize(p->stream);
+  for (int i = 0; i < kStagingSlots; ++i)
+    if (p->staging_ev[i]) cudaEventDestroy(p->staging_ev[i]);
+  if (p->staging) cudaFreeHost(p->staging);
+  delete p;
+  return SC_OK;
+}
+
+sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t step_tag) {
+  if (!p) return SC_ERR_INVALID_ARG;
+  sc_status st = check_ptr_array(anchor_grads, p->n_mats, true);
+  if (st != SC_OK) return st;
+  if (step_tag < p->last_tag) return SC_ERR_STALE_TAG;
+  cudaStream_t s = p->stream;
+  const int lp = p->lp, rp = p->rp;
+  const int g_bf16 = p->hp.grad_dtype == SC_DTYPE_BF16;
+  for (int i = 0; i < p->n_mats; ++i) p->host_tab[i].Ganc = anchor_grads[i];
+  if ((st = upload_table(p)) != SC_OK) return st;
+  for (auto& c : p->classes) {
+    std::vector<int> act;
+    for (int id : c.mats)
+      if (anchor_grads[id]) act.push_back(id);
+    const int cnt = (int)act.size();
+    if (!cnt) continue;
+    const int* idx = c.idx_all;
+    if (cnt != (int)c.mats.size()) {
+      // pageable source: the runtime has taken its copy of `act` when this returns
+      if (cudaMemcpyAsync(c.idx_dyn, act.data(), cnt * sizeof(int), cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return SC_ERR_CUDA;
+      idx = c.idx_dyn;
+    }
+    const int m = (int)c.m, n = (int)c.n;
+    launch_ema(p->dev_tab, idx, cnt, (int64_t)m * n, g_bf16, p->hp.beta_anc, s);                        // Eq. 1
+    if (p->rank > 0) {
+      // range finder: Y = M Omega, Q = orth(Y)
+      launch_gemm(gemm(p, idx, OFF(Manc), OFF(omega_t), OFF(Y), m, lp, n, n, n, lp, 0, 1), cnt, s);
+      cholqr2(p, idx, cnt, OFF(Y), OFF(Y2), m, false);
+      for (int it = 0; it < p->q; ++it) {
+        launch_gemm(gemm(p, idx, OFF(Manc), OFF(Y), OFF(Z), n, lp, m, n, lp, lp, 1, 0), cnt, s);   // Z = M^T Q
+        cholqr2(p, idx, cnt, OFF(Z), OFF(Z2), n, false);
+        launch_gemm(gemm(p, idx, OFF(Manc), OFF(Z), OFF(Y), m, lp, n, n, lp, lp, 0, 0), cnt, s);   // Y = M Z
+        cholqr2(p, idx, cnt, OFF(Y), OFF(Y2), m, false);
+      }
+      // B^T = M^T Q = Qb R ; SVD of the small factor ; U = Q Ub, V = Qb Wb
+      launch_gemm(gemm(p, idx, OFF(Manc), OFF(Y), OFF(Z), n, lp, m, n, lp, lp, 1, 0), cnt, s);
+      cholqr2(p, idx, cnt, OFF(Z), OFF(Z2), n, true);
+      launch_jacobi(p->dev_tab, idx, cnt, lp, rp, p->rank, p->hp.tau_p, s);                           // + Eq. 2
+      launch_gemm(gemm(p, idx, OFF(Y), OFF(ub), OFF(U), m, rp, lp, lp, rp, rp, 0, 0), cnt, s);
+      launch_gemm(gemm(p, idx, OFF(Z), OFF(wb), OFF(V), n, rp, lp, lp, rp, rp, 0, 0), cnt, s);
+      refresh_operands(p, c, idx, cnt);
+    }
+    for (int id : act) p->has_basis[id] = 1;
+  }
+  p->last_tag = step_tag;
+  return cuda_ok(cudaGetLastError());
+}
+
+sc_status sc_correct_and_step(sc_plan* p, const void* const* masked_grads, void* const* params,
+                              const sc_opt_state* state, int64_t step) {
+  if (!p || !state || step < 1) return SC_ERR_INVALID_ARG;
+  sc_status st;
+  if ((st = check_ptr_array(masked_grads, p->n_mats, false)) != SC_OK) return st;
+  if ((st = check_ptr_array(reinterpret_cast<const void* const*>(params), p->n_mats, false)) != SC_OK) return st;
+  if ((st = check_ptr_array(reinterpret_cast<const void* const*>(state->exp_avg), p->n_mats, false)) != SC_OK) return st;
+  if ((st = check_ptr_array(reinterpret_cast<const void* const*>(state->exp_avg_sq), p->n_mats, false)) != SC_OK) return st;
+  if (state->params_bf16 &&
+      (st = check_ptr_array(reinterpret_cast<const void* const*>(state->params_bf16), p->n_mats, true)) != SC_OK)
+    return st;
+  cudaStream_t s = p->stream;
+  const sc_hparams& hp = p->hp;
+  const int rp = p->rp;
+  const int g_bf16 = hp.grad_dtype == SC_DTYPE_BF16;
+  bool g_changed = false;
+  for (int i = 0; i < p->n_mats; ++i) {
+    MatDev& md = p->host_tab[i];
+    g_changed = g_changed || md.G != masked_grads[i];
+    md.G = masked_grads[i];
+    md.W = static_cast<float*>(params[i]);
+    md.m1 = static_cast<float*>(state->exp_avg[i]);
+    md.m2 = static_cast<float*>(state->exp_avg_sq[i]);
+    md.Wb = state->params_bf16 ? static_cast<bf16*>(state->params_bf16[i]) : nullptr;
+    md.gproj_dbg = static_cast<float*>(p->dbg_out[i]);
+  }
+  if ((st = upload_table(p)) != SC_OK) return st;
+  if (g_changed)
+    for (auto& c : p->classes)
+      if (c.tensor && (st = tc_encode_class(p, c, false, true)) != SC_OK) return st;
+
+  const float scale = hp.grads_prescaled ? 1.f : 1.f / p->keep;
+  const double bc1 = 1.0 - pow((double)hp.beta1, (double)step), bc2 = 1.0 - pow((double)hp.beta2, (double)step);
+  StepScalars sc{};
+  sc.alpha_s = hp.alpha * scale;
+  sc.beta1 = hp.beta1; sc.beta2 = hp.beta2; sc.one_m_beta1 = 1.f - hp.beta1; sc.one_m_beta2 = 1.f - hp.beta2;
+  sc.step_size = (float)((double)hp.lr / bc1);
+  sc.inv_sqrt_bc2 = (float)(1.0 / sqrt(bc2));
+  sc.eps = hp.eps;
+  sc.decay = 1.f - hp.lr * hp.weight_decay;
+  const bool clip_on = hp.max_grad_norm > 0.f;
+  const bool want_norm = clip_on || hp.collect_stats;
+
+  auto project = [&](ShapeClass& c) -> sc_status {
+    const int cnt = (int)c.mats.size(), m = (int)c.m, n = (int)c.n;
+    const int* idx = c.idx_all;
+    if (rp > 0) {
+      if (c.tensor) {
+        sc_status e = tc_launch_project(p, c, idx, cnt);                                                  // T = G V
+        if (e != SC_OK) return e;
+        launch_reduce_partials(p->dev_tab, idx, cnt, (int64_t)m * rp, c.ksplit, s);
+      } else {
+        launch_gemm(gemm(p, idx, OFF(G), OFF(V), OFF(T), m, rp, n, n, rp, rp, 0, 0, g_bf16), cnt, s);
+      }
+      launch_gemm(gemm(p, idx, OFF(U), OFF(T), OFF(X), rp, rp, m, rp, rp, rp, 1, 0), cnt, s);        // X = U^T T
+    }
+    if (want_norm) launch_sqnorm(p->dev_tab, idx, cnt, (int64_t)m * n, g_bf16, s);
+    launch_xs(p->dev_tab, idx, cnt, rp, p->rank, 0.f, scale, hp.alpha, s);                             // D X D
+    if (rp > 0) {
+      launch_gemm(gemm(p, idx, OFF(V), OFF(Xs), OFF(Ct), n, rp, rp, rp, rp, rp, 0, 1), cnt, s);      // C^T = V Xs^T
+      if (c.tensor) launch_split_ct(p->dev_tab, idx, cnt, n, rp, s);
+    }
+    return SC_OK;
+  };
+  auto update = [&](ShapeClass& c) -> sc_status {
+    const int cnt = (int)c.mats.size(), m = (int)c.m, n = (int)c.n;
+    if (c.tensor) return tc_launch_epilogue(p, c, c.idx_all, cnt, sc);
+    launch_epilogue_simt(p->dev_tab, c.idx_all, cnt, m, n, rp, g_bf16, sc, p->clip_dev, s);
+    return SC_OK;
+  };
+
+  if (clip_on) {
+    for (auto& c : p->classes) if ((st = project(c)) != SC_OK) return st;
+    launch_clip(p->dev_tab, p->n_mats, hp.max_grad_norm, p->clip_dev, s);
+    for (auto& c : p->classes) if ((st = update(c)) != SC_OK) return st;
+  } else {
+    for (auto& c : p->classes) {
+      if ((st = project(c)) != SC_OK) return st;
+      if ((st = update(c)) != SC_OK) return st;
+    }
+  }
+  if (cudaGetLastError() != cudaSuccess) return SC_ERR_CUDA;
+  bool any = false;
+  for (char h : p->has_basis) any = any || h;
+  return (p->rank > 0 && !any) ? SC_WARN_NO_ANCHOR : SC_OK;
+}
+
+// -------------------------------------------------------------------------------------- inspection
+
+static sc_status check_mat(sc_plan* p, int mat) {
+  if (!p || mat < 0 || mat >= p->n_mats) return SC_ERR_INVALID_ARG;
+  return SC_OK;
+}
+
+sc_status sc_export_basis(sc_plan* p, int mat, void* U_dev, void* s_dev, void* V_dev) {
+  sc_status st = check_mat(p, mat);
+  if (st != SC_OK) return st;
+  const MatDev& md = p->host_tab[mat];
+  const int r = p->rank, rp = p->rp;
+  if (r == 0) return SC_OK;
+  if (U_dev) launch_unpad_copy(static_cast<float*>(U_dev), r, md.U, rp, md.m, r, p->stream);
+  if (V_dev) launch_unpad_copy(static_cast<float*>(V_dev), r, md.V, rp, md.n, r, p->stream);
+  if (s_dev && cudaMemcpyAsync(s_dev, md.sv, r * sizeof(float), cudaMemcpyDeviceToDevice, p->stream) != cudaSuccess)
+    return SC_ERR_CUDA;
+  return cuda_ok(cudaGetLastError());
+}
+
+sc_status sc_import_basis(sc_plan* p, int mat, const void* U_dev, const void* s_dev, const void* V_dev) {
+  sc_status st = check_mat(p, mat);
+  if (st != SC_OK) return st;
+  if (!U_dev || !s_dev || !V_dev) return SC_ERR_INVALID_ARG;
+  const MatDev& md = p->host_tab[mat];
+  const int r = p->rank, rp = p->rp;
+  if (r == 0) return SC_OK;
+  cudaStream_t s = p->stream;
+  if ((st = upload_table(p)) != SC_OK) return st;
+  launch_pad_copy(md.U, rp, static_cast<const float*>(U_dev), r, md.m, r, rp, s);
+  launch_pad_copy(md.V, rp, static_cast<const float*>(V_dev), r, md.n, r, rp, s);
+  launch_pad_copy(md.sv, rp, static_cast<const float*>(s_dev), r, 1, r, rp, s);
+  ShapeClass& c = p->classes[p->class_of[mat]];
+  const int* idx = c.idx_all + p->inst_of[mat];
+  launch_filter_weights(p->dev_tab, idx, 1, rp, r, p->hp.tau_p, s);
+  refresh_operands(p, c, idx, 1);
+  p->has_basis[mat] = 1;
+  return cuda_ok(cudaGetLastError());
+}
+
+sc_status sc_export_anchor_momentum(sc_plan* p, int mat, void* M_dev) {
+  sc_status st = check_mat(p, mat);
+  if (st != SC_OK) return st;
+  if (!M_dev) return SC_ERR_INVALID_ARG;
+  const MatDev& md = p->host_tab[mat];
+  return cuda_ok(cudaMemcpyAsync(M_dev, md.Manc, (size_t)md.m * md.n * sizeof(float), cudaMemcpyDeviceToDevice,
+                                 p->stream));
+}
+
+sc_status sc_import_anchor_momentum(sc_plan* p, int mat, const void* M_dev) {
+  sc_status st = check_mat(p, mat);
+  if (st != SC_OK) return st;
+  if (!M_dev) return SC_ERR_INVALID_ARG;
+  const MatDev& md = p->host_tab[mat];
+  return cuda_ok(cudaMemcpyAsync(md.Manc, M_dev, (size_t)md.m * md.n * sizeof(float), cudaMemcpyDeviceToDevice,
+                                 p->stream));
+}
+
+sc_status sc_export_sketch(sc_plan* p, int64_t rows, int width, void* Omega_dev) {
+  if (!p || !Omega_dev || rows <= 0 || width <= 0 || width > 1024) return SC_ERR_INVALID_ARG;
+  launch_sketch_rowmajor(static_cast<float*>(Omega_dev), rows, width, p->hp.seed, p->stream);
+  return cuda_ok(cudaGetLastError());
+}
+
+sc_status sc_set_debug_gproj_out(sc_plan* p, void* const* gproj_out) {
+  if (!p) return SC_ERR_INVALID_ARG;
+  for (int i = 0; i < p->n_mats; ++i) p->dbg_out[i] = gproj_out ? gproj_out[i] : nullptr;
+  return SC_OK;
+}
+
+sc_status sc_get_stats(sc_plan* p, sc_mat_stats* stats, float* clip) {
+  if (!p || !stats) return SC_ERR_INVALID_ARG;
+  std::vector<float> h((size_t)p->n_mats * kStatsFloats);
+  if (cudaMemcpyAsync(h.data(), p->stats_dev, h.size() * sizeof(float), cudaMemcpyDeviceToHost, p->stream) !=
+      cudaSuccess)
+    return SC_ERR_CUDA;
+  float c = 1.f;
+  if (cudaMemcpyAsync(&c, p->clip_dev, sizeof(float), cudaMemcpyDeviceToHost, p->stream) != cudaSuccess)
+    return SC_ERR_CUDA;
+  if (cudaStreamSynchronize(p->stream) != cudaSuccess) return SC_ERR_CUDA;
+  for (int i = 0; i < p->n_mats; ++i) {
+    const float* f = &h[(size_t)i * kStatsFloats];
+    stats[i].g_sqnorm = f[0]; stats[i].x_sqnorm = f[1]; stats[i].gproj_sqnorm = f[2]; stats[i].r_eff = f[3];
+  }
+  if (clip) *clip = c;
+  return SC_OK;
+}
+
+sc_status sc_get_device_status(sc_plan* p) {
+  if (!p) return SC_ERR_INVALID_ARG;
+  unsigned w = 0;
+  if (cudaMemcpyAsync(&w, p->status_dev, sizeof(w), cudaMemcpyDeviceToHost, p->stream) != cudaSuccess ||
+      cudaStreamSynchronize(p->stream) != cudaSuccess)
+    return SC_ERR_CUDA;
+  if (w) cudaMemsetAsync(p->status_dev, 0, sizeof(w), p->stream);
+  if (w & kDevTimeout) return SC_ERR_TIMEOUT;
+  if (w & kDevNonfinite) return SC_ERR_NONFINITE;
+  return SC_OK;
+}
+
+sc_status sc_get_anchor_info(sc_plan* p, int64_t* last_tag, int* n_with_basis) {
+  if (!p) return SC_ERR_INVALID_ARG;
+  if (last_tag) *last_tag = p->last_tag;
+  if (n_with_basis) {
+    int k = 0;
+    for (char h : p->has_basis) k += h ? 1 : 0;
+    *n_with_basis = k;
+  }
+  return SC_OK;
+}
+
+int sc_plan_uses_tensor_cores(const sc_plan* p) { return p && p->tensor_any ? 1 : 0; }
+
+const char* sc_status_string(sc_status s) {
+  switch (s) {
+    case SC_OK: return "ok";
+    case SC_WARN_NO_ANCHOR: return "no anchor gradient has arrived yet (empty basis)";
+    case SC_ERR_INVALID_ARG: return "invalid argument";
+    case SC_ERR_SHAPE: return "invalid shape or rank larger than a matrix dimension";
+    case SC_ERR_DTYPE: return "unsupported dtype";
+    case SC_ERR_ALIGNMENT: return "pointer not sufficiently aligned";
+    case SC_ERR_WORKSPACE: return "workspace too small";
+    case SC_ERR_STALE_TAG: return "anchor step tag older than the last accepted one";
+    case SC_ERR_CUDA: return "CUDA error";
+    case SC_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+    case SC_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case SC_ERR_NONFINITE: return "non-finite value encountered";
+    case SC_ERR_TOO_LARGE: return "dimension too large";
+  }
+  return "unknown status";
+}
+
+int sc_version(void) { return 100; }
+
+}  // extern "C"

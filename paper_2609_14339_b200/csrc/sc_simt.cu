@@ -1,0 +1,559 @@
+// CUDA-core (fp32) kernels of the spectral-correction step.
+//
+// These serve (a) every small, latency-bound piece of the method (Cholesky and Jacobi factorisations of
+// l x l matrices, the r x r filter, norms) for all plans and (b) the large contractions too when the plan
+// runs on the fp32 engine (fp32 gradients, shapes the tensor-core kernels do not take).
+// Kernels are launched once per shape class; blockIdx.z selects the matrix through idx[] and the table.
+#include "sc_internal.cuh"
+
+namespace sc {
+
+template <typename T>
+__device__ __forceinline__ T* field(const MatDev& md, int off) {
+  return *reinterpret_cast<T* const*>(reinterpret_cast<const char*>(&md) + off);
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// =====================================================================================================
+// Batched tiled GEMM  C = alpha * op(A) * op(B), fp32 accumulate, with an optional fused AdamW epilogue.
+// =====================================================================================================
+constexpr int BM = 64, BN = 64, BK = 16;
+
+struct EpiStore {};
+struct EpiAdamW {
+  StepScalars sc;
+  const float* clip;
+  int g_bf16;
+};
+
+template <bool kAdamW>
+__global__ void __launch_bounds__(256) gemm_kernel(GemmArgs a, EpiAdamW epi) {
+  __shared__ float As[BK][BM + 1];
+  __shared__ float Bs[BK][BN + 1];
+  const MatDev& md = a.tab[a.idx[blockIdx.z]];
+  const float* A = field<const float>(md, a.offA);
+  const bf16* Ab = reinterpret_cast<const bf16*>(A);
+  const float* B = field<const float>(md, a.offB);
+  const int row0 = blockIdx.y * BM, col0 = blockIdx.x * BN;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  float acc[4][4] = {};
+  for (int k0 = 0; k0 < a.K; k0 += BK) {
+    for (int e = tid; e < BM * BK; e += 256) {
+      int r, k;
+      if (!a.transA) { r = e / BK; k = e % BK; } else { k = e / BM; r = e % BM; }
+      const int gr = row0 + r, gk = k0 + k;
+      float v = 0.f;
+      if (gr < a.M && gk < a.K) {
+        const size_t off = a.transA ? (size_t)gk * a.lda + gr : (size_t)gr * a.lda + gk;
+        v = a.a_bf16 ? __bfloat162float(Ab[off]) : A[off];
+      }
+      As[k][r] = v;
+    }
+    for (int e = tid; e < BN * BK; e += 256) {
+      int c, k;
+      if (!a.transB) { k = e / BN; c = e % BN; } else { c = e / BK; k = e % BK; }
+      const int gc = col0 + c, gk = k0 + k;
+      float v = 0.f;
+      if (gc < a.N && gk < a.K) v = a.transB ? B[(size_t)gc * a.ldb + gk] : B[(size_t)gk * a.ldb + gc];
+      Bs[k][c] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < BK; ++k) {
+      float av[4], bv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) av[i] = As[k][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) bv[j] = Bs[k][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  if (!kAdamW) {
+    float* C = field<float>(md, a.offC);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int gr = row0 + ty * 4 + i;
+      if (gr >= a.M) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int gc = col0 + tx * 4 + j;
+        if (gc < a.N) C[(size_t)gr * a.ldc + gc] = a.alpha * acc[i][j];
+      }
+    }
+  } else {
+    // acc = (U C)[i][j], the low-rank part (already carrying (1-alpha)*scale); blend, clip, AdamW.
+    const float clip = *epi.clip;
+    const StepScalars& s = epi.sc;
+    const float* Gf = reinterpret_cast<const float*>(md.G);
+    const bf16* Gb = reinterpret_cast<const bf16*>(md.G);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int gr = row0 + ty * 4 + i;
+      if (gr >= a.M) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int gc = col0 + tx * 4 + j;
+        if (gc >= a.N) continue;
+        const size_t o = (size_t)gr * a.N + gc;
+        const float graw = epi.g_bf16 ? __bfloat162float(Gb[o]) : Gf[o];
+        const float g = clip * fmaf(s.alpha_s, graw, acc[i][j]);
+        const float mo = fmaf(s.beta1, md.m1[o], s.one_m_beta1 * g);
+        const float vo = fmaf(s.beta2, md.m2[o], s.one_m_beta2 * g * g);
+        const float den = fmaf(sqrtf(vo), s.inv_sqrt_bc2, s.eps);
+        const float w = fmaf(-s.step_size, mo / den, md.W[o] * s.decay);
+        md.m1[o] = mo;
+        md.m2[o] = vo;
+        md.W[o] = w;
+        if (md.Wb) md.Wb[o] = __float2bfloat16_rn(w);
+        if (md.gproj_dbg) md.gproj_dbg[o] = g;
+      }
+    }
+  }
+}
+
+void launch_gemm(const GemmArgs& a, int count, cudaStream_t s) {
+  if (count <= 0 || a.M <= 0 || a.N <= 0) return;
+  dim3 grid((a.N + BN - 1) / BN, (a.M + BM - 1) / BM, count);
+  gemm_kernel<false><<<grid, 256, 0, s>>>(a, EpiAdamW{});
+}
+
+void launch_epilogue_simt(const MatDev* tab, const int* idx, int count, int m, int n, int rp, int g_bf16,
+                          const StepScalars& sc, const float* clip, cudaStream_t s) {
+  if (count <= 0) return;
+  GemmArgs a{};
+  a.tab = tab; a.idx = idx;
+  a.offA = offsetof(MatDev, U); a.offB = offsetof(MatDev, Ct); a.offC = 0;
+  a.M = m; a.N = n; a.K = rp;
+  a.lda = rp; a.ldb = rp; a.ldc = n;
+  a.transA = 0; a.transB = 1; a.a_bf16 = 0; a.alpha = 1.f;
+  EpiAdamW e{sc, clip, g_bf16};
+  dim3 grid((n + BN - 1) / BN, (m + BM - 1) / BM, count);
+  gemm_kernel<true><<<grid, 256, 0, s>>>(a, e);
+}
+
+// =====================================================================================================
+// Eq. 1: anchor momentum  M <- beta M + (1 - beta) G_anc
+// =====================================================================================================
+__global__ void __launch_bounds__(256) ema_kernel(const MatDev* tab, const int* idx, int64_t numel, int g_bf16,
+                                                  float beta) {
+  const MatDev& md = tab[idx[blockIdx.z]];
+  float* M = md.Manc;
+  const float omb = 1.f - beta;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if ((numel & 3) == 0) {
+    const int64_t n4 = numel >> 2;
+    float4* M4 = reinterpret_cast<float4*>(M);
+    for (int64_t i = t0; i < n4; i += stride) {
+      float4 mv = M4[i];
+      float g0, g1, g2, g3;
+      if (g_bf16) {
+        const uint2 raw = reinterpret_cast<const uint2*>(md.Ganc)[i];
+        const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162*>(&raw.x);
+        const __nv_bfloat162 b = *reinterpret_cast<const __nv_bfloat162*>(&raw.y);
+        g0 = __low2float(a); g1 = __high2float(a); g2 = __low2float(b); g3 = __high2float(b);
+      } else {
+        const float4 gv = reinterpret_cast<const float4*>(md.Ganc)[i];
+        g0 = gv.x; g1 = gv.y; g2 = gv.z; g3 = gv.w;
+      }
+      mv.x = fmaf(beta, mv.x, omb * g0); mv.y = fmaf(beta, mv.y, omb * g1);
+      mv.z = fmaf(beta, mv.z, omb * g2); mv.w = fmaf(beta, mv.w, omb * g3);
+      M4[i] = mv;
+    }
+  } else {
+    for (int64_t i = t0; i < numel; i += stride) {
+      const float g = g_bf16 ? __bfloat162float(reinterpret_cast<const bf16*>(md.Ganc)[i])
+                             : reinterpret_cast<const float*>(md.Ganc)[i];
+      M[i] = fmaf(beta, M[i], omb * g);
+    }
+  }
+}
+
+void launch_ema(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, float beta, cudaStream_t s) {
+  if (count <= 0) return;
+  int64_t blocks = (numel / 4 + 255) / 256;
+  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (blocks < 1) blocks = 1;
+  ema_kernel<<<dim3((unsigned)blocks, 1, count), 256, 0, s>>>(tab, idx, numel, g_bf16, beta);
+}
+
+// =====================================================================================================
+// Counter-based Rademacher sketch: Omega[j][c] = +1 / -1 from the top bit of a 64-bit hash of (seed, j, c).
+//   counter = j * 2^10 + c ; h = mix(seed ^ ((counter + 1) * 0x9E3779B97F4A7C15)), mix = SplitMix64 finaliser.
+// =====================================================================================================
+__device__ __forceinline__ float sketch_entry(uint64_t seed, uint64_t j, uint64_t c) {
+  uint64_t x = seed ^ (((j << 10) + c + 1ull) * 0x9E3779B97F4A7C15ull);
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  x = x ^ (x >> 31);
+  return (x >> 63) ? -1.f : 1.f;
+}
+
+__global__ void sketch_t_kernel(float* omega_t, int lp, int l, int64_t n, uint64_t seed) {
+  const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int c = blockIdx.y;
+  if (j >= n || c >= lp) return;
+  omega_t[(size_t)c * n + j] = c < l ? sketch_entry(seed, (uint64_t)j, (uint64_t)c) : 0.f;
+}
+
+void launch_sketch(float* omega_t, int lp, int l, int64_t n, uint64_t seed, cudaStream_t s) {
+  if (lp <= 0) return;
+  sketch_t_kernel<<<dim3((unsigned)((n + 255) / 256), lp), 256, 0, s>>>(omega_t, lp, l, n, seed);
+}
+
+__global__ void sketch_rm_kernel(float* omega, int64_t rows, int width, uint64_t seed) {
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= rows * width) return;
+  omega[e] = sketch_entry(seed, (uint64_t)(e / width), (uint64_t)(e % width));
+}
+
+void launch_sketch_rowmajor(float* omega, int64_t rows, int width, uint64_t seed, cudaStream_t s) {
+  const int64_t tot = rows * width;
+  if (tot <= 0) return;
+  sketch_rm_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, s>>>(omega, rows, width, seed);
+}
+
+// =====================================================================================================
+// Cholesky factor of the Gram matrix (gram = R^T R, R upper) and its inverse, one block per matrix.
+// A pivot that has cancelled to (numerically) nothing marks a column that lies in the span of the earlier
+// ones: that direction is dropped (its column of R^-1 is zero) instead of dividing by ~0.
+// =====================================================================================================
+__global__ void __launch_bounds__(256) chol_kernel(const MatDev* tab, const int* idx, int lp, int offR) {
+  __shared__ float invd[kMaxRank];
+  __shared__ float piv_inv;
+  const MatDev& md = tab[idx[blockIdx.x]];
+  const float* G = md.gram;
+  float* R = field<float>(md, offR);
+  float* Ri = md.rinv;
+  const int t = threadIdx.x;
+  for (int j = 0; j < lp; ++j) {
+    const int i = t;
+    double s = 0.0;
+    if (i >= j && i < lp) {
+      s = (double)G[(size_t)j * lp + i];
+      for (int k = 0; k < j; ++k) s -= (double)R[(size_t)k * lp + j] * (double)R[(size_t)k * lp + i];
+    }
+    if (i == j) {
+      const double gjj = (double)G[(size_t)j * lp + j];
+      const bool ok = (s > 1e-6 * gjj) && (gjj > 0.0);
+      const float rjj = ok ? (float)sqrt(s) : 0.f;
+      piv_inv = ok ? 1.f / rjj : 0.f;
+      invd[j] = piv_inv;
+      R[(size_t)j * lp + j] = rjj;
+    }
+    __syncthreads();
+    if (i > j && i < lp) R[(size_t)j * lp + i] = (float)s * piv_inv;
+    if (i < j) R[(size_t)j * lp + i] = 0.f;
+    __syncthreads();
+  }
+  // inverse of the upper-triangular factor, one column per thread
+  const int c = t;
+  if (c < lp) {
+    for (int i = lp - 1; i > c; --i) Ri[(size_t)i * lp + c] = 0.f;
+    Ri[(size_t)c * lp + c] = invd[c];
+    for (int i = c - 1; i >= 0; --i) {
+      double s = 0.0;
+      for (int k = i + 1; k <= c; ++k) s += (double)R[(size_t)i * lp + k] * (double)Ri[(size_t)k * lp + c];
+      Ri[(size_t)i * lp + c] = (float)(-s) * invd[i];
+    }
+  }
+}
+
+void launch_chol(const MatDev* tab, const int* idx, int count, int lp, int offR, cudaStream_t s) {
+  if (count <= 0 || lp <= 0) return;
+  chol_kernel<<<count, 256, 0, s>>>(tab, idx, lp, offR);
+}
+
+// =====================================================================================================
+// One-sided Jacobi SVD of the small factor, one block per matrix.
+//   racc = R (lp x lp) with B^T = Qb R, hence B = R^T Qb^T. Row j of R is column j of K = R^T, so the
+//   buffer is read as lp contiguous columns. Right rotations J orthogonalise the columns: K J = Ub S.
+//   Output (sorted by descending singular value, leading `rank` kept, padded to rp with zeros):
+//     sv, d (Eq. 2), ub = Ub (lp x rp), wb = J (lp x rp).
+// =====================================================================================================
+constexpr int kJacobiThreads = 512;
+
+__global__ void __launch_bounds__(kJacobiThreads) jacobi_kernel(const MatDev* tab, const int* idx, int lp, int rp,
+                                                                int rank, float tau_p) {
+  __shared__ float nrm[kMaxRank];
+  __shared__ int order[kMaxRank];
+  __shared__ int rotated;
+  const MatDev& md = tab[idx[blockIdx.x]];
+  float* Kc = md.jk;
+  float* Jc = md.jv;
+  const float* R = md.racc;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kJacobiThreads / 32;
+  for (int e = tid; e < lp * lp; e += kJacobiThreads) {
+    Kc[e] = R[e];
+    Jc[e] = (e / lp == e % lp) ? 1.f : 0.f;
+  }
+  __syncthreads();
+  const int half = lp / 2;
+  for (int sweep = 0; sweep < 24; ++sweep) {
+    if (tid == 0) rotated = 0;
+    __syncthreads();
+    for (int rd = 0; rd < lp - 1; ++rd) {
+      for (int pi = warp; pi < half; pi += nwarp) {
+        int p, q;
+        if (pi == 0) { p = lp - 1; q = rd; }
+        else { p = (rd + pi) % (lp - 1); q = (rd - pi + (lp - 1)) % (lp - 1); }
+        float* kp = Kc + (size_t)p * lp; float* kq = Kc + (size_t)q * lp;
+        float a = 0.f, b = 0.f, c = 0.f;
+        for (int i = lane; i < lp; i += 32) {
+          const float x = kp[i], y = kq[i];
+          a = fmaf(x, x, a); b = fmaf(y, y, b); c = fmaf(x, y, c);
+        }
+        a = warp_sum(a); b = warp_sum(b); c = warp_sum(c);
+        const float lim = sqrtf(a) * sqrtf(b);
+        if (!(fabsf(c) > 1e-7f * lim) || lim == 0.f) continue;
+        if (fabsf(c) > 2e-6f * lim && lane == 0) rotated = 1;
+        const float zeta = (b - a) / (2.f * c);
+        const float tt = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
+        const float cs = rsqrtf(1.f + tt * tt), sn = cs * tt;
+        float* jp = Jc + (size_t)p * lp; float* jq = Jc + (size_t)q * lp;
+        for (int i = lane; i < lp; i += 32) {
+          const float x = kp[i], y = kq[i];
+          kp[i] = cs * x - sn * y; kq[i] = sn * x + cs * y;
+          const float u = jp[i], w = jq[i];
+          jp[i] = cs * u - sn * w; jq[i] = sn * u + cs * w;
+        }
+      }
+      __syncthreads();
+    }
+    if (!rotated) break;
+    __syncthreads();
+  }
+  // column norms = singular values
+  for (int j = warp; j < lp; j += nwarp) {
+    float a = 0.f;
+    for (int i = lane; i < lp; i += 32) { const float x = Kc[(size_t)j * lp + i]; a = fmaf(x, x, a); }
+    a = warp_sum(a);
+    if (lane == 0) nrm[j] = sqrtf(a);
+  }
+  __syncthreads();
+  // rank of each column by counting (stable for ties)
+  for (int j = tid; j < lp; j += kJacobiThreads) {
+    int rk = 0;
+    const float sj = nrm[j];
+    for (int k = 0; k < lp; ++k) rk += (nrm[k] > sj) || (nrm[k] == sj && k < j);
+    order[rk] = j;
+  }
+  __syncthreads();
+  const float smax = nrm[order[0]];
+  for (int k = tid; k < rp; k += kJacobiThreads) {
+    float s = (k < rank && k < lp) ? nrm[order[k]] : 0.f;
+    if (!(s > 1e-7f * smax)) s = 0.f;
+    md.sv[k] = s;
+    md.d[k] = (s + tau_p > 0.f) ? s / (s + tau_p) : 0.f;
+  }
+  for (int e = tid; e < lp * rp; e += kJacobiThreads) {
+    const int i = e / rp, k = e % rp;
+    float u = 0.f, w = 0.f;
+    if (k < rank && k < lp) {
+      const int j = order[k];
+      const float s = nrm[j];
+      if (s > 1e-7f * smax) { u = Kc[(size_t)j * lp + i] / s; w = Jc[(size_t)j * lp + i]; }
+    }
+    md.ub[e] = u;
+    md.wb[e] = w;
+  }
+}
+
+void launch_jacobi(const MatDev* tab, const int* idx, int count, int lp, int rp, int rank, float tau_p,
+                   cudaStream_t s) {
+  if (count <= 0 || lp <= 0 || rp <= 0) return;
+  jacobi_kernel<<<count, kJacobiThreads, 0, s>>>(tab, idx, lp, rp, rank, tau_p);
+}
+
+// Eq. 2 from stored singular values (used after a basis import).
+__global__ void filter_weights_kernel(const MatDev* tab, const int* idx, int rp, int rank, float tau_p) {
+  const MatDev& md = tab[idx[blockIdx.x]];
+  for (int k = threadIdx.x; k < rp; k += blockDim.x) {
+    const float s = k < rank ? md.sv[k] : 0.f;
+    md.d[k] = (s + tau_p > 0.f) ? s / (s + tau_p) : 0.f;
+  }
+}
+
+void launch_filter_weights(const MatDev* tab, const int* idx, int count, int rp, int rank, float tau_p,
+                           cudaStream_t s) {
+  if (count <= 0 || rp <= 0) return;
+  filter_weights_kernel<<<count, 256, 0, s>>>(tab, idx, rp, rank, tau_p);
+}
+
+// =====================================================================================================
+// bf16 hi/lo splits of the basis: U ~= Uhi + Ulo (m x rp), V^T ~= Vthi + Vtlo (rp x n, transposed).
+// =====================================================================================================
+__device__ __forceinline__ void split2(float x, bf16& hi, bf16& lo) {
+  hi = __float2bfloat16_rn(x);
+  lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
+__global__ void __launch_bounds__(256) split_basis_kernel(const MatDev* tab, const int* idx, int m, int n, int rp) {
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t nu = (int64_t)m * rp, nv = (int64_t)n * rp;
+  for (int64_t e = t0; e < nu; e += stride) split2(md.U[e], md.Uhi[e], md.Ulo[e]);
+  // V is n x rp; write the transpose rp x n (threads run along n for coalesced stores)
+  for (int64_t e = t0; e < nv; e += stride) {
+    const int64_t k = e / n, j = e % n;
+    split2(md.V[(size_t)j * rp + k], md.Vthi[e], md.Vtlo[e]);
+  }
+}
+
+void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int n, int rp, cudaStream_t s) {
+  if (count <= 0 || rp <= 0) return;
+  int64_t tot = (int64_t)(m > n ? m : n) * rp;
+  int blocks = (int)((tot + 255) / 256 < 1184 ? (tot + 255) / 256 : 1184);
+  split_basis_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, m, n, rp);
+}
+
+__global__ void __launch_bounds__(256) split_ct_kernel(const MatDev* tab, const int* idx, int64_t numel) {
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < numel; e += stride)
+    split2(md.Ct[e], md.Cthi[e], md.Ctlo[e]);
+}
+
+void launch_split_ct(const MatDev* tab, const int* idx, int count, int n, int rp, cudaStream_t s) {
+  if (count <= 0 || rp <= 0) return;
+  const int64_t tot = (int64_t)n * rp;
+  int blocks = (int)((tot + 255) / 256 < 296 ? (tot + 255) / 256 : 296);
+  split_ct_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, tot);
+}
+
+// =====================================================================================================
+// ||G||_F^2 in two fixed-order stages (no float atomics): kSqnormBlocks partials per matrix.
+// =====================================================================================================
+__global__ void __launch_bounds__(256) sqnorm_kernel(const MatDev* tab, const int* idx, int64_t numel, int g_bf16) {
+  __shared__ float red[8];
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const int64_t per = (numel + kSqnormBlocks - 1) / kSqnormBlocks;
+  const int64_t lo = per * blockIdx.x, hi = (lo + per < numel) ? lo + per : numel;
+  float acc = 0.f;
+  for (int64_t i = lo + threadIdx.x; i < hi; i += 256) {
+    const float g = g_bf16 ? __bfloat162float(reinterpret_cast<const bf16*>(md.G)[i])
+                           : reinterpret_cast<const float*>(md.G)[i];
+    acc = fmaf(g, g, acc);
+  }
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int w = 0; w < 8; ++w) t += red[w];
+    md.sqpart[blockIdx.x] = t;
+  }
+}
+
+void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, cudaStream_t s) {
+  if (count <= 0) return;
+  sqnorm_kernel<<<dim3(kSqnormBlocks, 1, count), 256, 0, s>>>(tab, idx, numel, g_bf16);
+}
+
+// =====================================================================================================
+// The r x r filter: Xs = coef * D X D (coef = (1-alpha)*scale), and the per-matrix statistics.
+//   stats[0] = ||g||^2, stats[1] = ||X||^2 (scaled), stats[2] = ||G_proj||^2 (closed form), stats[3] = sum d^2
+// =====================================================================================================
+__global__ void __launch_bounds__(256) xs_kernel(const MatDev* tab, const int* idx, int rp, int rank, float coef,
+                                                 float scale, float alpha) {
+  __shared__ float red[3][8];
+  const MatDev& md = tab[idx[blockIdx.x]];
+  float sx = 0.f, s1 = 0.f, s2 = 0.f;
+  for (int e = threadIdx.x; e < rp * rp; e += 256) {
+    const int i = e / rp, j = e % rp;
+    const float x = md.X[e] * scale;
+    const float dd = (i < rank && j < rank) ? md.d[i] * md.d[j] : 0.f;
+    md.Xs[e] = (1.f - alpha) * dd * x;
+    sx = fmaf(x, x, sx);
+    s1 = fmaf(dd * x, x, s1);
+    s2 = fmaf(dd * dd * x, x, s2);
+  }
+  (void)coef;
+  sx = warp_sum(sx); s1 = warp_sum(s1); s2 = warp_sum(s2);
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = sx; red[1][threadIdx.x >> 5] = s1; red[2][threadIdx.x >> 5] = s2; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tx = 0.f, t1 = 0.f, t2 = 0.f, gg = 0.f, re = 0.f;
+    for (int w = 0; w < 8; ++w) { tx += red[0][w]; t1 += red[1][w]; t2 += red[2][w]; }
+    for (int b = 0; b < kSqnormBlocks; ++b) gg += md.sqpart[b];
+    gg *= scale * scale;
+    for (int k = 0; k < rank; ++k) re = fmaf(md.d[k], md.d[k], re);
+    md.stats[0] = gg;
+    md.stats[1] = tx;
+    md.stats[2] = alpha * alpha * gg + 2.f * alpha * (1.f - alpha) * t1 + (1.f - alpha) * (1.f - alpha) * t2;
+    md.stats[3] = re;
+  }
+}
+
+void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, float coef, float scale, float alpha,
+               cudaStream_t s) {
+  if (count <= 0) return;
+  xs_kernel<<<count, 256, 0, s>>>(tab, idx, rp, rank, coef, scale, alpha);
+}
+
+// Global-norm clip factor over all matrices, summed in matrix order by one thread block.
+__global__ void clip_kernel(const MatDev* tab, int n_mats, float max_norm, float* clip) {
+  __shared__ float red[256];
+  float acc = 0.f;
+  for (int i = threadIdx.x; i < n_mats; i += 256) acc += tab[i].stats[2];
+  red[threadIdx.x] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int i = 0; i < 256; ++i) t += red[i];
+    const float nrm = sqrtf(t);
+    *clip = (max_norm > 0.f && nrm > max_norm) ? max_norm / nrm : 1.f;
+  }
+}
+
+void launch_clip(const MatDev* tab, int n_mats, float max_norm, float* clip, cudaStream_t s) {
+  clip_kernel<<<1, 256, 0, s>>>(tab, n_mats, max_norm, clip);
+}
+
+// Copies between a dense rows x cols matrix and its zero-padded rows x cols_dst copy (basis import/export).
+__global__ void pad_copy_kernel(float* dst, int ldd, const float* src, int lds, int rows, int cols, int cols_dst) {
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (int64_t)rows * cols_dst) return;
+  const int i = (int)(e / cols_dst), j = (int)(e % cols_dst);
+  dst[(size_t)i * ldd + j] = j < cols ? src[(size_t)i * lds + j] : 0.f;
+}
+
+void launch_pad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, int cols_dst,
+                     cudaStream_t s) {
+  const int64_t tot = (int64_t)rows * cols_dst;
+  if (tot <= 0) return;
+  pad_copy_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, s>>>(dst, ldd, src, lds, rows, cols, cols_dst);
+}
+
+void launch_unpad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, cudaStream_t s) {
+  launch_pad_copy(dst, ldd, src, lds, rows, cols, cols, s);
+}
+
+// Sum of split-K partials of T (fixed order): T[0] <- sum_s T[s].
+__global__ void reduce_partials_kernel(const MatDev* tab, const int* idx, int64_t numel, int ksplit) {
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < numel; e += stride) {
+    float t = md.T[e];
+    for (int s = 1; s < ksplit; ++s) t += md.T[(size_t)s * numel + e];
+    md.T[e] = t;
+  }
+}
+
+void launch_reduce_partials(const MatDev* tab, const int* idx, int count, int64_t numel, int ksplit, cudaStream_t s) {
+  if (count <= 0 || ksplit <= 1) return;
+  int blocks = (int)((numel + 255) / 256 < 592 ? (numel + 255) / 256 : 592);
+  reduce_partials_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, numel, ksplit);
+}
+
+}  // namespace sc
