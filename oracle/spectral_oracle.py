@@ -259,12 +259,22 @@ def mirror_basis(M, Omega, q: int, r: int):
 
 
 def projector_distance(Ua, Ub) -> float:
-    """||Ua Ua^T - Ub Ub^T||_F / sqrt(2 r), via ||Pa-Pb||_F^2 = ra + rb - 2||Ua^T Ub||_F^2 (sign/rotation free)."""
+    """||Pa - Pb||_F / sqrt(2 r) for the orthogonal projectors onto span(Ua), span(Ub) (sign/rotation free).
+
+    For equal ranks ||Pa - Pb||_F^2 = 2 ||(I - Pa) Qb||_F^2 with Qb an orthonormal basis of span(Ub); the
+    residual form is used because 2r - 2||Ua^T Ub||_F^2 cancels catastrophically (it cannot resolve
+    distances below ~sqrt(machine eps of the inputs)).  Inputs are re-orthonormalised first, so
+    a slightly non-unit column norm of an fp32 basis does not register as a subspace error.
+    """
     ra, rb = Ua.shape[1], Ub.shape[1]
     if ra == 0 and rb == 0:
         return 0.0
-    d2 = ra + rb - 2.0 * float(np.sum((Ua.T @ Ub) ** 2))
-    return float(np.sqrt(max(d2, 0.0) / (ra + rb)))
+    if ra != rb:
+        return 1.0
+    Qa, _ = np.linalg.qr(np.asarray(Ua, F64))
+    Qb, _ = np.linalg.qr(np.asarray(Ub, F64))
+    res = Qb - Qa @ (Qa.T @ Qb)
+    return float(np.linalg.norm(res) / np.sqrt(ra))
 
 
 # --------------------------------------------------------------------------

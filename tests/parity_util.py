@@ -60,9 +60,12 @@ def make_inputs(case: Case):
 
 
 def oracle_hyper(case: Case) -> so.Hyper:
-    return so.Hyper(alpha=case.alpha, tau_p=case.tau_p, beta_anc=case.beta_anc, lr=case.lr, eps=case.eps,
-                    weight_decay=case.weight_decay, max_grad_norm=case.max_grad_norm,
-                    grads_prescaled=case.prescaled, keep=case.keep)
+    """The hyper-parameters as the C ABI receives them: the ABI's fields are C floats, so both sides get the
+    fp32-rounded values (0.999 as a float is 0.99900001287..., which moves 1 - beta2 by 1.3e-5 relative)."""
+    f = lambda x: float(np.float32(x))
+    return so.Hyper(alpha=f(case.alpha), tau_p=f(case.tau_p), beta_anc=f(case.beta_anc), lr=f(case.lr), eps=f(case.eps),
+                    weight_decay=f(case.weight_decay), max_grad_norm=f(case.max_grad_norm),
+                    beta1=f(0.9), beta2=f(0.999), grads_prescaled=case.prescaled, keep=f(case.keep))
 
 
 def to_dev(arr, dtype: str, torch, device):
@@ -173,12 +176,14 @@ def compare_step(g: GpuRun, o: OracleRun, mask_small_g=False):
 
 
 def compare_basis(g: GpuRun, o: OracleRun):
-    errs = dict(M=0.0, PU=0.0, PV=0.0, s=0.0)
+    errs = dict(M=0.0, PU=0.0, PV=0.0, s=0.0, orth=0.0)
     for i, st in enumerate(o.states):
         errs["M"] = max(errs["M"], rel(g.M_anc[i], st.M_anc))
         U, s, V = g.basis[i]
         if st.U.shape[1] == 0:
             continue
+        r = U.shape[1]
+        errs["orth"] = max(errs["orth"], float(np.abs(U.T @ U - np.eye(r)).max()), float(np.abs(V.T @ V - np.eye(r)).max()))
         errs["PU"] = max(errs["PU"], so.projector_distance(U, st.U))
         errs["PV"] = max(errs["PV"], so.projector_distance(V, st.V))
         errs["s"] = max(errs["s"], rel(s, st.s))

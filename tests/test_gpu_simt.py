@@ -35,7 +35,7 @@ def test_c1_single_256_fp32_mirror_and_exact(torch):
     assert g.dev_status == 0 and g.step_status == 0 and not g.uses_tc
     o = OracleRun(case, inp, "mirror")
     eb = compare_basis(g, o)
-    assert eb["M"] < 1e-6 and eb["PU"] < TOL32 and eb["PV"] < TOL32 and eb["s"] < TOL32, eb
+    assert eb["M"] < 1e-6 and eb["PU"] < TOL32 and eb["PV"] < TOL32 and eb["s"] < TOL32 and eb["orth"] < 1e-5, eb
     es = compare_step(g, o, mask_small_g=True)
     assert es["gproj"] < TOL32 and es["m"] < TOL32 and es["v"] < TOL32 and es["dW"] < TOL32, es
     # rule parity on the oracle's exact basis (imported)

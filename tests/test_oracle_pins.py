@@ -336,3 +336,16 @@ def test_planted_component_has_requested_snr():
     G = gen.dense_gradient(spec, 1)
     inside = np.linalg.norm(Py.T @ G @ Px) ** 2 / np.linalg.norm(G) ** 2
     assert 0.2 < inside < 0.9       # planted energy comparable to the noise energy at SNR 1
+
+
+def test_projector_distance_matches_explicit_projectors():
+    A, _ = np.linalg.qr(RNG.standard_normal((40, 6)))
+    for th in (1e-7, 1e-3, 0.3):
+        x = RNG.standard_normal(40); x -= A @ (A.T @ x); x /= np.linalg.norm(x)
+        B = A.copy(); B[:, 2] = np.cos(th) * A[:, 2] + np.sin(th) * x
+        explicit = np.sin(th) / np.sqrt(6)           # ||Pa-Pb||_F = sqrt(2) sin(theta) for one rotated direction
+        assert abs(so.projector_distance(A, B) - explicit) < 1e-12 + 1e-9 * explicit
+        assert abs(so.projector_distance(A, B @ np.diag([1, -1, 2, 1, 1, 0.5])) - explicit) < 1e-12 + 1e-9 * explicit
+    if True:
+        Pa, Pb = A @ A.T, B @ B.T
+        assert abs(so.projector_distance(A, B) - np.linalg.norm(Pa - Pb) / np.sqrt(12)) < 1e-12
