@@ -159,6 +159,10 @@ SC_API sc_status sc_export_basis(sc_plan* plan, int mat, void* U_dev, void* s_de
  * recompute Eq. 2 and the operand copies the step kernels read. Marks the matrix as having an anchor. */
 SC_API sc_status sc_import_basis(sc_plan* plan, int mat, const void* U_dev, const void* s_dev, const void* V_dev);
 
+/* Copy the projections of the last step for matrix `mat` (either may be NULL): T = G V (rows x rank fp32,
+ * row-major, on the raw masked gradient) and X = U^T G V (rank x rank fp32, row-major). */
+SC_API sc_status sc_export_projection(sc_plan* plan, int mat, void* T_dev, void* X_dev);
+
 /* Copy the anchor momentum (rows x cols fp32) to / from a caller device buffer. */
 SC_API sc_status sc_export_anchor_momentum(sc_plan* plan, int mat, void* M_dev);
 SC_API sc_status sc_import_anchor_momentum(sc_plan* plan, int mat, const void* M_dev);

@@ -68,6 +68,7 @@ EXPORTS = {
     "sc_correct_and_step": (C.c_int, [_VP, _VPP, _VPP, C.POINTER(OptState), C.c_int64]),
     "sc_export_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
     "sc_import_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
+    "sc_export_projection": (C.c_int, [_VP, C.c_int, _VP, _VP]),
     "sc_export_anchor_momentum": (C.c_int, [_VP, C.c_int, _VP]),
     "sc_import_anchor_momentum": (C.c_int, [_VP, C.c_int, _VP]),
     "sc_export_sketch": (C.c_int, [_VP, C.c_int64, C.c_int, _VP]),
@@ -205,6 +206,15 @@ class Plan:
         _check(self.lib.sc_import_basis(self.handle, mat, U.data_ptr(), s.data_ptr(), V.data_ptr()), "sc_import_basis")
         self._torch.cuda.current_stream(self.device).wait_stream(self.stream)
         self.stream.synchronize()
+
+    def export_projection(self, mat: int):
+        t = self._torch
+        m, n = self.shapes[mat]
+        T = t.empty((m, self.rank), dtype=t.float32, device=self.device)
+        X = t.empty((self.rank, self.rank), dtype=t.float32, device=self.device)
+        if self.rank > 0:
+            _check(self.lib.sc_export_projection(self.handle, mat, T.data_ptr(), X.data_ptr()), "sc_export_projection")
+        return T, X
 
     def export_anchor_momentum(self, mat: int):
         t = self._torch

@@ -32,7 +32,7 @@ struct MatDev {
   float* V;      // n x rp      right basis
   float* sv;     // rp          singular values
   float* d;      // rp          filter weights, Eq. 2
-  bf16* Uhi;     // m x rp      bf16 split of U  (U ~= Uhi + Ulo), K-major MMA operand
+  bf16* Uhi;     // m x rk      bf16 split of U  (U ~= Uhi + Ulo), K-major MMA operand, rk = rp rounded up to 64
   bf16* Ulo;
   bf16* Vthi;    // rp x n      bf16 split of V^T, K-major MMA operand
   bf16* Vtlo;
@@ -41,7 +41,7 @@ struct MatDev {
   float* X;      // rp x rp     X = U^T G V (unscaled)
   float* Xs;     // rp x rp     (1-alpha) * scale * D X D
   float* Ct;     // n x rp      C^T = V Xs^T, fp32
-  bf16* Cthi;    // n x rp      bf16 split of C^T
+  bf16* Cthi;    // n x rk      bf16 split of C^T
   bf16* Ctlo;
   float* sqpart; // kSqnormBlocks partial sums of ||G||^2
   float* stats;  // kStatsFloats
@@ -96,7 +96,7 @@ struct StepScalars {       // scalars of one step, passed by value to kernels
 }  // namespace sc
 
 struct sc_plan {
-  int n_mats = 0, rank = 0, rp = 0, l = 0, lp = 0, q = 0;
+  int n_mats = 0, rank = 0, rp = 0, rk = 0, l = 0, lp = 0, q = 0;   // rk: row stride of the bf16 K-operand copies
   float keep = 1.f;
   sc_hparams hp{};
   cudaStream_t stream = nullptr;
@@ -149,11 +149,11 @@ void launch_sketch_rowmajor(float* omega, int64_t rows, int width, uint64_t seed
 void launch_chol(const MatDev* tab, const int* idx, int count, int lp, int offR, cudaStream_t s);
 void launch_jacobi(const MatDev* tab, const int* idx, int count, int lp, int rp, int rank, float tau_p, cudaStream_t s);
 void launch_filter_weights(const MatDev* tab, const int* idx, int count, int rp, int rank, float tau_p, cudaStream_t s);
-void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int n, int rp, cudaStream_t s);
+void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int n, int rp, int rk, cudaStream_t s);
 void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, cudaStream_t s);
 void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, float coef, float scale, float alpha,
                cudaStream_t s);
-void launch_split_ct(const MatDev* tab, const int* idx, int count, int n, int rp, cudaStream_t s);
+void launch_split_ct(const MatDev* tab, const int* idx, int count, int n, int rp, int rk, cudaStream_t s);
 void launch_clip(const MatDev* tab, int n_mats, float max_norm, float* clip, cudaStream_t s);
 void launch_pad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, int cols_dst, cudaStream_t s);
 void launch_unpad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, cudaStream_t s);

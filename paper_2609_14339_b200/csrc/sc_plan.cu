@@ -31,7 +31,7 @@ struct Carver {
 };
 
 struct Dims {
-  int rp, l, lp, q;
+  int rp, rk, l, lp, q;
 };
 
 bool derive_dims(int rank, const sc_hparams* hp, Dims* d) {
@@ -40,6 +40,7 @@ bool derive_dims(int rank, const sc_hparams* hp, Dims* d) {
   if (l < rank || l > kMaxRank) return false;
   if (hp->power_iters < 0 || hp->power_iters > 16) return false;
   d->rp = rank > 0 ? round_up_int(rank, 16) : 0;
+  d->rk = round_up_int(d->rp, 64);
   d->l = l;
   d->lp = rank > 0 ? round_up_int(l, 16) : 0;
   d->q = hp->power_iters;
@@ -83,7 +84,7 @@ void build_classes(const sc_shape* shapes, int n_mats, std::vector<ShapeClass>& 
 
 int choose_ksplit(const ShapeClass& c) {
   const int64_t tiles = (c.m + 127) / 128 * (int64_t)c.mats.size();
-  int ks = 1;
+  int ks = 1;   // every K slice keeps >= 1024 columns, so no slice is ever empty
   while (ks < 8 && tiles * ks < 148 * 2 && c.n / (ks * 2) >= 1024) ks *= 2;
   return ks;
 }
@@ -91,7 +92,7 @@ int choose_ksplit(const ShapeClass& c) {
 // Lays the whole workspace out. With p->ws == nullptr nothing is dereferenced: it only measures.
 size_t layout(sc_plan* p, bool assign) {
   Carver cv(assign ? p->ws : nullptr);
-  const int n_mats = p->n_mats, rp = p->rp, lp = p->lp;
+  const int n_mats = p->n_mats, rp = p->rp, rk = p->rk, lp = p->lp;
   MatDev* tab = cv.take<MatDev>(n_mats);
   float* clip = cv.take<float>(1);
   unsigned* status = cv.take<unsigned>(1);
@@ -122,9 +123,9 @@ size_t layout(sc_plan* p, bool assign) {
     md.Ct = cv.take<float>(n * rp);
     md.sqpart = cv.take<float>(kSqnormBlocks);
     if (c.tensor) {
-      md.Uhi = cv.take<bf16>(m * rp); md.Ulo = cv.take<bf16>(m * rp);
+      md.Uhi = cv.take<bf16>(m * rk); md.Ulo = cv.take<bf16>(m * rk);
       md.Vthi = cv.take<bf16>(n * rp); md.Vtlo = cv.take<bf16>(n * rp);
-      md.Cthi = cv.take<bf16>(n * rp); md.Ctlo = cv.take<bf16>(n * rp);
+      md.Cthi = cv.take<bf16>(n * rk); md.Ctlo = cv.take<bf16>(n * rk);
     }
     md.stats = assign ? p->stats_dev + (size_t)i * kStatsFloats : nullptr;
     md.omega_t = c.omega_t;
@@ -158,7 +159,7 @@ size_t layout(sc_plan* p, bool assign) {
 }
 
 void fill_plan_basics(sc_plan* p, const sc_shape* shapes, int n_mats, int rank, const sc_hparams* hp, const Dims& d) {
-  p->n_mats = n_mats; p->rank = rank; p->rp = d.rp; p->l = d.l; p->lp = d.lp; p->q = d.q;
+  p->n_mats = n_mats; p->rank = rank; p->rp = d.rp; p->rk = d.rk; p->l = d.l; p->lp = d.lp; p->q = d.q;
   p->hp = *hp;
   p->shapes.assign(shapes, shapes + n_mats);
   build_classes(shapes, n_mats, p->classes, p->class_of, p->inst_of);
@@ -207,7 +208,7 @@ void cholqr2(sc_plan* p, const int* idx, int cnt, int offY, int offTmp, int rows
 
 // Rebuild d (Eq. 2) and the bf16 operand copies of one matrix list after its U, s, V changed.
 void refresh_operands(sc_plan* p, const ShapeClass& c, const int* idx, int cnt) {
-  if (c.tensor) launch_split_basis(p->dev_tab, idx, cnt, (int)c.m, (int)c.n, p->rp, p->stream);
+  if (c.tensor) launch_split_basis(p->dev_tab, idx, cnt, (int)c.m, (int)c.n, p->rp, p->rk, p->stream);
 }
 
 sc_status check_ptr_array(const void* const* arr, int n, bool allow_null_entries) {
@@ -453,7 +454,7 @@ sc_status sc_correct_and_step(sc_plan* p, const void* const* masked_grads, void*
     launch_xs(p->dev_tab, idx, cnt, rp, p->rank, 0.f, scale, hp.alpha, s);                             // D X D
     if (rp > 0) {
       launch_gemm(gemm(p, idx, OFF(V), OFF(Xs), OFF(Ct), n, rp, rp, rp, rp, rp, 0, 1), cnt, s);      // C^T = V Xs^T
-      if (c.tensor) launch_split_ct(p->dev_tab, idx, cnt, n, rp, s);
+      if (c.tensor) launch_split_ct(p->dev_tab, idx, cnt, n, rp, p->rk, s);
     }
     return SC_OK;
   };
@@ -517,6 +518,17 @@ sc_status sc_import_basis(sc_plan* p, int mat, const void* U_dev, const void* s_
   launch_filter_weights(p->dev_tab, idx, 1, rp, r, p->hp.tau_p, s);
   refresh_operands(p, c, idx, 1);
   p->has_basis[mat] = 1;
+  return cuda_ok(cudaGetLastError());
+}
+
+sc_status sc_export_projection(sc_plan* p, int mat, void* T_dev, void* X_dev) {
+  sc_status st = check_mat(p, mat);
+  if (st != SC_OK) return st;
+  const MatDev& md = p->host_tab[mat];
+  const int r = p->rank, rp = p->rp;
+  if (r == 0) return SC_OK;
+  if (T_dev) launch_unpad_copy(static_cast<float*>(T_dev), r, md.T, rp, md.m, r, p->stream);
+  if (X_dev) launch_unpad_copy(static_cast<float*>(X_dev), r, md.X, rp, r, r, p->stream);
   return cuda_ok(cudaGetLastError());
 }
 

@@ -397,12 +397,17 @@ __device__ __forceinline__ void split2(float x, bf16& hi, bf16& lo) {
   lo = __float2bfloat16_rn(x - __bfloat162float(hi));
 }
 
-__global__ void __launch_bounds__(256) split_basis_kernel(const MatDev* tab, const int* idx, int m, int n, int rp) {
+__global__ void __launch_bounds__(256) split_basis_kernel(const MatDev* tab, const int* idx, int m, int n, int rp,
+                                                          int rk) {
   const MatDev& md = tab[idx[blockIdx.z]];
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t nu = (int64_t)m * rp, nv = (int64_t)n * rp;
-  for (int64_t e = t0; e < nu; e += stride) split2(md.U[e], md.Uhi[e], md.Ulo[e]);
+  // U is m x rp (fp32); the bf16 copies have row stride rk, columns rp..rk-1 stay zero
+  for (int64_t e = t0; e < nu; e += stride) {
+    const int64_t i = e / rp, k = e % rp;
+    split2(md.U[e], md.Uhi[i * rk + k], md.Ulo[i * rk + k]);
+  }
   // V is n x rp; write the transpose rp x n (threads run along n for coalesced stores)
   for (int64_t e = t0; e < nv; e += stride) {
     const int64_t k = e / n, j = e % n;
@@ -410,25 +415,27 @@ __global__ void __launch_bounds__(256) split_basis_kernel(const MatDev* tab, con
   }
 }
 
-void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int n, int rp, cudaStream_t s) {
+void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int n, int rp, int rk, cudaStream_t s) {
   if (count <= 0 || rp <= 0) return;
   int64_t tot = (int64_t)(m > n ? m : n) * rp;
   int blocks = (int)((tot + 255) / 256 < 1184 ? (tot + 255) / 256 : 1184);
-  split_basis_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, m, n, rp);
+  split_basis_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, m, n, rp, rk);
 }
 
-__global__ void __launch_bounds__(256) split_ct_kernel(const MatDev* tab, const int* idx, int64_t numel) {
+__global__ void __launch_bounds__(256) split_ct_kernel(const MatDev* tab, const int* idx, int64_t numel, int rp, int rk) {
   const MatDev& md = tab[idx[blockIdx.z]];
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < numel; e += stride)
-    split2(md.Ct[e], md.Cthi[e], md.Ctlo[e]);
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < numel; e += stride) {
+    const int64_t j = e / rp, k = e % rp;
+    split2(md.Ct[e], md.Cthi[j * rk + k], md.Ctlo[j * rk + k]);
+  }
 }
 
-void launch_split_ct(const MatDev* tab, const int* idx, int count, int n, int rp, cudaStream_t s) {
+void launch_split_ct(const MatDev* tab, const int* idx, int count, int n, int rp, int rk, cudaStream_t s) {
   if (count <= 0 || rp <= 0) return;
   const int64_t tot = (int64_t)n * rp;
   int blocks = (int)((tot + 255) / 256 < 296 ? (tot + 255) / 256 : 296);
-  split_ct_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, tot);
+  split_ct_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, tot, rp, rk);
 }
 
 // =====================================================================================================

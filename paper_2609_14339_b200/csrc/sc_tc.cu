@@ -1,10 +1,470 @@
-// placeholder: tensor-core kernels
+// Tensor-core (tcgen05 / TMEM / TMA) kernels of the spectral-correction step for sm_100a.
+//
+//   project_kernel        T = G (Vhi + Vlo)              streaming GEMM over the masked gradient, N = rank
+//   fused_update_kernel   G_proj = clip * (alpha_s G + (Uhi + Ulo)(Chi + Clo)^T), then AdamW, one HBM pass
+//
+// Operands: G is bf16 as given; the fp32 factors are carried as a sum of two bf16 numbers (hi + lo), so
+// the products lose nothing that matters at the 2e-3 tolerance. All MMA operands sit in shared memory in
+// the K-major, 128-byte-swizzled layout that both TMA (SWIZZLE_128B) and the UMMA descriptors understand.
+// Every wait on an mbarrier is bounded; when a wait runs out the kernel latches an error bit, drains what
+// it has in flight, frees its TMEM and returns.
+#include <cuda.h>
+
 #include "sc_internal.cuh"
+
 namespace sc {
-bool tc_shape_supported(int64_t, int64_t, int) { return false; }
-size_t tc_tmaps_bytes(int) { return 0; }
-sc_status tc_init() { return SC_OK; }
-sc_status tc_encode_class(sc_plan*, ShapeClass&, bool, bool) { return SC_OK; }
-sc_status tc_launch_project(sc_plan*, ShapeClass&, const int*, int) { return SC_ERR_INVALID_ARG; }
-sc_status tc_launch_epilogue(sc_plan*, ShapeClass&, const int*, int, const StepScalars&) { return SC_ERR_INVALID_ARG; }
+
+// ---------------------------------------------------------------------------------------------- PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: polls, backs off, gives up after ~2^22 polls (far beyond any legitimate wait here).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < (1u << 22); ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (it > 64) {
+      __nanosleep(it > 4096 ? 256 : 32);
+      if (*abort_flag) return false;
+    }
+  }
+  return false;
+}
+__device__ __forceinline__ void tensormap_acquire(const void* map) {
+  asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(map) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const void* map, uint64_t* bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(ncols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major operand tile, rows of 128 bytes, 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_k128(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 128.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+constexpr int kMapsPerMat = 7;   // G, Vthi, Vtlo, Uhi, Ulo, Cthi, Ctlo
+enum { MAP_G = 0, MAP_VTHI, MAP_VTLO, MAP_UHI, MAP_ULO, MAP_CTHI, MAP_CTLO };
+constexpr int kTileBytes = 128 * 128;   // 128 rows x 64 bf16
+
+// =====================================================================================================
+// T = G V  (per 128-row tile of G and per K slice).  Warp 0: TMA producer. Warp 1: MMA issuer (owns TMEM).
+// Warps 2-5: epilogue, TMEM -> registers -> global.
+// =====================================================================================================
+__global__ void __launch_bounds__(192, 1)
+project_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const CUtensorMap* __restrict__ maps,
+               int m, int n, int rp, int cps, int stages, uint32_t tmem_cols, unsigned* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int stage_bytes = kTileBytes + 2 * rp * 128;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+  uint64_t* empty = full + stages;
+  uint64_t* accum = empty + stages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* never_flag = abort_flag + 1;   // stays 0: lets the drain below wait although abort is set
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int inst = blockIdx.z;
+  const MatDev& md = tab[idx[inst]];
+  const CUtensorMap* mp = maps + (size_t)inst * kMapsPerMat;
+  const int row0 = blockIdx.x * 128;
+  const int nchunks = (n + 63) >> 6;
+  const int c0 = blockIdx.y * cps;
+  const int my_chunks = min(cps, nchunks - c0);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(accum, 1);
+    *abort_flag = 0;
+    *never_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_d = *tmem_slot;
+
+  if (warp == 0 && lane == 0) {
+    tensormap_acquire(mp + MAP_G); tensormap_acquire(mp + MAP_VTHI); tensormap_acquire(mp + MAP_VTLO);
+    int issued = 0;
+    for (int i = 0; i < my_chunks; ++i, ++issued) {
+      const int s = i % stages;
+      if (!mbar_wait(&empty[s], ((i / stages) & 1) ^ 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
+      uint8_t* st = smem + (size_t)s * stage_bytes;
+      mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
+      const int x = (c0 + i) * 64;
+      tma_load_2d(st, mp + MAP_G, &full[s], x, row0);
+      tma_load_2d(st + kTileBytes, mp + MAP_VTHI, &full[s], x, 0);
+      tma_load_2d(st + kTileBytes + rp * 128, mp + MAP_VTLO, &full[s], x, 0);
+    }
+    if (*abort_flag) {   // let copies already in flight land before the block's shared memory goes away
+      for (int i = max(0, issued - stages); i < issued; ++i) mbar_wait(&full[i % stages], (i / stages) & 1, never_flag);
+    }
+  } else if (warp == 1 && lane == 0) {
+    const uint32_t idesc = umma_idesc_bf16(rp);
+    for (int i = 0; i < my_chunks; ++i) {
+      const int s = i % stages;
+      if (!mbar_wait(&full[s], (i / stages) & 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
+      tc_fence_after();
+      const uint32_t a = smem_u32(smem + (size_t)s * stage_bytes);
+      const uint32_t bh = a + kTileBytes, bl = bh + rp * 128;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const uint64_t ad = umma_desc_k128(a + k * 32);
+        umma_bf16(tmem_d, ad, umma_desc_k128(bh + k * 32), idesc, (i | k) != 0);
+        umma_bf16(tmem_d, ad, umma_desc_k128(bl + k * 32), idesc, 1);
+      }
+      umma_commit(&empty[s]);
+    }
+    umma_commit(accum);
+  } else if (warp >= 2) {
+    const int q = warp & 3;
+    const int row = row0 + q * 32 + lane;
+    bool ok = mbar_wait(accum, 0, abort_flag);
+    if (!ok && lane == 0) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
+    ok = __all_sync(0xffffffffu, ok) && !*abort_flag;
+    tc_fence_after();
+    if (ok) {
+      float* Trow = md.T + ((size_t)blockIdx.y * m + row) * rp;
+      for (int c = 0; c < rp; c += 16) {
+        float v[16];
+        tmem_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + c, v);
+        tmem_ld_wait();
+        if (row < m) {
+#pragma unroll
+          for (int j = 0; j < 16; j += 4)
+            *reinterpret_cast<float4*>(Trow + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_d, tmem_cols);
+}
+
+// =====================================================================================================
+// Fused correction + AdamW for one 128 x 128 tile.
+//   mainloop (one elected thread): R = (Uhi + Ulo)(Cthi + Ctlo)^T over K = rank, three bf16 MMAs per K step
+//   (hi*hi, hi*lo, lo*hi; lo*lo is below fp32 resolution), accumulated in TMEM;
+//   epilogue (all 8 warps): TMEM -> swizzled shared staging -> coalesced 128-bit pass over G, W, m, v.
+// =====================================================================================================
+__device__ __forceinline__ void adamw4(const StepScalars& s, float clip, const float g_raw[4], const float4& r,
+                                       float4& w, float4& m1, float4& m2, float4& gp) {
+  const float rr[4] = {r.x, r.y, r.z, r.w};
+  float* W = &w.x; float* M1 = &m1.x; float* M2 = &m2.x; float* GP = &gp.x;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float g = clip * fmaf(s.alpha_s, g_raw[j], rr[j]);
+    const float mo = fmaf(s.beta1, M1[j], s.one_m_beta1 * g);
+    const float vo = fmaf(s.beta2, M2[j], s.one_m_beta2 * g * g);
+    const float den = fmaf(sqrtf(vo), s.inv_sqrt_bc2, s.eps);
+    W[j] = fmaf(-s.step_size, mo / den, W[j] * s.decay);
+    M1[j] = mo; M2[j] = vo; GP[j] = g;
+  }
+}
+
+__global__ void __launch_bounds__(256, 3)
+fused_update_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const CUtensorMap* __restrict__ maps,
+                    int m, int n, int rp, StepScalars sc, const float* __restrict__ clip_ptr, unsigned* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + 4 * kTileBytes);
+  uint64_t* mma_done = full + 1;     // per K chunk: the operand tiles may be overwritten
+  uint64_t* accum_done = full + 2;   // once: the accumulator is complete (waited on by every thread, phase 0)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_done + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int inst = blockIdx.z;
+  const MatDev& md = tab[idx[inst]];
+  const CUtensorMap* mp = maps + (size_t)inst * kMapsPerMat;
+  const int col0 = blockIdx.x * 128, row0 = blockIdx.y * 128;
+  const int nch = (rp + 63) >> 6;
+
+  if (threadIdx.x == 0) {
+    mbar_init(full, 1);
+    mbar_init(mma_done, 1);
+    mbar_init(accum_done, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 0) tmem_alloc(tmem_slot, 128);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_d = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tensormap_acquire(mp + MAP_UHI); tensormap_acquire(mp + MAP_ULO);
+      tensormap_acquire(mp + MAP_CTHI); tensormap_acquire(mp + MAP_CTLO);
+      const uint32_t idesc = umma_idesc_bf16(128);
+      const uint32_t uh = smem_u32(smem), ul = uh + kTileBytes, ch = ul + kTileBytes, cl = ch + kTileBytes;
+      for (int c = 0; c < nch; ++c) {
+        if (c > 0 && !mbar_wait(mma_done, (c - 1) & 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
+        mbar_expect_tx(full, 4 * kTileBytes);
+        tma_load_2d(smem, mp + MAP_UHI, full, c * 64, row0);
+        tma_load_2d(smem + kTileBytes, mp + MAP_ULO, full, c * 64, row0);
+        tma_load_2d(smem + 2 * kTileBytes, mp + MAP_CTHI, full, c * 64, col0);
+        tma_load_2d(smem + 3 * kTileBytes, mp + MAP_CTLO, full, c * 64, col0);
+        if (!mbar_wait(full, c & 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
+        tc_fence_after();
+        const int ksteps = min(64, rp - c * 64) >> 4;
+        for (int k = 0; k < ksteps; ++k) {
+          const uint64_t ah = umma_desc_k128(uh + k * 32), al = umma_desc_k128(ul + k * 32);
+          const uint64_t bh = umma_desc_k128(ch + k * 32), bl = umma_desc_k128(cl + k * 32);
+          umma_bf16(tmem_d, ah, bh, idesc, (c | k) != 0);
+          umma_bf16(tmem_d, ah, bl, idesc, 1);
+          umma_bf16(tmem_d, al, bh, idesc, 1);
+        }
+        umma_commit(mma_done);
+      }
+      umma_commit(accum_done);
+    }
+    __syncwarp();
+  }
+  bool ok = mbar_wait(accum_done, 0, abort_flag);
+  if (!ok) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
+  tc_fence_after();
+
+  // TMEM -> shared staging: 128 rows x 32 slots of 16 bytes, slot index XOR (row & 31) keeps both the
+  // row-per-thread writes here and the row-per-warp reads below free of bank conflicts.
+  float4* stage = reinterpret_cast<float4*>(smem);
+  {
+    const int q = warp & 3, h = warp >> 2;
+    const int r = q * 32 + lane;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float v[16];
+      const int cbase = h * 64 + j * 16;
+      tmem_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + cbase, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        stage[r * 32 + (((cbase >> 2) + i) ^ (r & 31))] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_d, 128);
+  if (*abort_flag) return;
+
+  const float clip = *clip_ptr;
+  const int col = col0 + lane * 4;
+  if (col >= n) return;
+  const uint2* __restrict__ G = reinterpret_cast<const uint2*>(md.G);
+  float4* __restrict__ W = reinterpret_cast<float4*>(md.W);
+  float4* __restrict__ M1 = reinterpret_cast<float4*>(md.m1);
+  float4* __restrict__ M2 = reinterpret_cast<float4*>(md.m2);
+  uint2* __restrict__ Wb = reinterpret_cast<uint2*>(md.Wb);
+  float4* __restrict__ GP = reinterpret_cast<float4*>(md.gproj_dbg);
+  constexpr int kUnroll = 2;
+  for (int rr = warp; rr < 128; rr += 8 * kUnroll) {
+    uint2 graw[kUnroll];
+    float4 w[kUnroll], m1[kUnroll], m2[kUnroll];
+    size_t off[kUnroll];
+    bool live[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int row = row0 + rr + 8 * u;
+      live[u] = row < m;
+      off[u] = ((size_t)row * n + col) >> 2;
+      if (live[u]) {
+        graw[u] = __ldg(G + off[u]);
+        w[u] = __ldcs(W + off[u]);
+        m1[u] = __ldcs(M1 + off[u]);
+        m2[u] = __ldcs(M2 + off[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      if (!live[u]) continue;
+      const int lr = rr + 8 * u;
+      const float4 r = stage[lr * 32 + (lane ^ (lr & 31))];
+      const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&graw[u].x);
+      const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&graw[u].y);
+      const float g4[4] = {__low2float(g01), __high2float(g01), __low2float(g23), __high2float(g23)};
+      float4 gp;
+      adamw4(sc, clip, g4, r, w[u], m1[u], m2[u], gp);
+      __stcs(W + off[u], w[u]);
+      __stcs(M1 + off[u], m1[u]);
+      __stcs(M2 + off[u], m2[u]);
+      if (Wb) {
+        __nv_bfloat162 b01 = __floats2bfloat162_rn(w[u].x, w[u].y), b23 = __floats2bfloat162_rn(w[u].z, w[u].w);
+        uint2 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&b01);
+        pk.y = *reinterpret_cast<uint32_t*>(&b23);
+        __stcs(Wb + off[u], pk);
+      }
+      if (GP) GP[off[u]] = gp;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------- host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+
+bool tc_shape_supported(int64_t m, int64_t n, int rp) {
+  return rp >= 16 && rp <= 256 && (n % 8) == 0 && m >= 1 && n >= 64;
+}
+
+size_t tc_tmaps_bytes(int count) { return (size_t)count * kMapsPerMat * sizeof(CUtensorMap); }
+
+sc_status tc_init() {
+  if (g_encode) return SC_OK;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+      qres != cudaDriverEntryPointSuccess)
+    return SC_ERR_CUDA;
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  static bool attrs_done = false;
+  if (!attrs_done) {
+    if (cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(fused_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024) != cudaSuccess)
+      return SC_ERR_CUDA;
+    attrs_done = true;
+  }
+  return SC_OK;
+}
+
+// bf16 row-major matrix [outer][inner] -> 2-D map with a 64 x box_rows box and the 128-byte swizzle.
+static bool encode_bf16(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_elems,
+                        uint32_t box_rows) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {row_stride_elems * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return g_encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// (Re)encode the tensor maps of a class and copy them to the device. The source is pageable host memory,
+// so the runtime has taken its copy of the bytes when cudaMemcpyAsync returns.
+sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_call_part) {
+  const int cnt = (int)c.mats.size();
+  const int rp = p->rp, rk = p->rk;
+  std::vector<CUtensorMap> maps((size_t)cnt * kMapsPerMat);
+  CUtensorMap* dev = static_cast<CUtensorMap*>(c.tmaps);
+  for (int i = 0; i < cnt; ++i) {
+    const MatDev& md = p->host_tab[c.mats[i]];
+    CUtensorMap* mp = &maps[(size_t)i * kMapsPerMat];
+    bool ok = true;
+    if (per_call_part) {
+      ok = ok && encode_bf16(mp + MAP_G, md.G, c.n, c.m, c.n, 128);
+      if (!ok) return SC_ERR_CUDA;
+      if (cudaMemcpyAsync(dev + (size_t)i * kMapsPerMat + MAP_G, mp + MAP_G, sizeof(CUtensorMap), cudaMemcpyHostToDevice,
+                          p->stream) != cudaSuccess)
+        return SC_ERR_CUDA;
+    }
+    if (static_part) {
+      ok = ok && encode_bf16(mp + MAP_VTHI, md.Vthi, c.n, rp, c.n, rp);
+      ok = ok && encode_bf16(mp + MAP_VTLO, md.Vtlo, c.n, rp, c.n, rp);
+      ok = ok && encode_bf16(mp + MAP_UHI, md.Uhi, rk, c.m, rk, 128);
+      ok = ok && encode_bf16(mp + MAP_ULO, md.Ulo, rk, c.m, rk, 128);
+      ok = ok && encode_bf16(mp + MAP_CTHI, md.Cthi, rk, c.n, rk, 128);
+      ok = ok && encode_bf16(mp + MAP_CTLO, md.Ctlo, rk, c.n, rk, 128);
+      if (!ok) return SC_ERR_CUDA;
+      if (cudaMemcpyAsync(dev + (size_t)i * kMapsPerMat + MAP_VTHI, mp + MAP_VTHI, 6 * sizeof(CUtensorMap),
+                          cudaMemcpyHostToDevice, p->stream) != cudaSuccess)
+        return SC_ERR_CUDA;
+    }
+  }
+  return SC_OK;
+}
+
+static int project_stages(int rp) {
+  const int stage_bytes = kTileBytes + 2 * rp * 128;
+  int s = (200 * 1024) / stage_bytes;
+  return s > 6 ? 6 : (s < 2 ? 2 : s);
+}
+
+sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count) {
+  const int rp = p->rp, m = (int)c.m, n = (int)c.n;
+  const int nchunks = (n + 63) / 64;
+  const int cps = (nchunks + c.ksplit - 1) / c.ksplit;
+  const int stages = project_stages(rp);
+  const size_t smem = (size_t)stages * (kTileBytes + 2 * rp * 128) + 1024 + 256;
+  uint32_t cols = 32;
+  while ((int)cols < rp) cols <<= 1;
+  dim3 grid((m + 127) / 128, c.ksplit, count);
+  project_kernel<<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), m, n, rp,
+                                                 cps, stages, cols, p->status_dev);
+  return cuda_ok(cudaGetLastError());
+}
+
+sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc) {
+  const int m = (int)c.m, n = (int)c.n;
+  dim3 grid((n + 127) / 128, (m + 127) / 128, count);
+  const size_t smem = 4 * kTileBytes + 1024 + 64;
+  fused_update_kernel<<<grid, 256, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), m, n,
+                                                      p->rp, sc, p->clip_dev, p->status_dev);
+  return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace sc

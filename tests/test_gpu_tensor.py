@@ -1,0 +1,81 @@
+"""GPU parity of the tensor-core (tcgen05) engine for bf16 gradients against the fp64 oracle.
+
+Tolerance: 2e-3 relative Frobenius error (the bar for bf16 operands); bases compared as projectors."""
+import numpy as np
+import pytest
+
+from oracle import spectral_oracle as so
+from parity_util import Case, GpuRun, OracleRun, compare_basis, compare_step, make_inputs, rel
+from synth import generator as gen
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-3
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    return torch
+
+
+def _check(case, torch, tol=TOL):
+    inp = make_inputs(case)
+    g = GpuRun(case, inp, torch)
+    assert g.uses_tc, "expected the tcgen05 engine"
+    assert g.dev_status == 0 and g.status_after_anchor == 0
+    o = OracleRun(case, inp, "mirror")
+    # the two contractions on their own, against the oracle with the GPU's own basis
+    for i in range(len(case.shapes)):
+        U, s, V = g.basis[i]
+        T, X = g.plan.export_projection(i)
+        assert rel(T.double().cpu().numpy(), o.G[i] @ V) < 1e-4, "T = G V"
+        assert rel(X.double().cpu().numpy(), U.T @ o.G[i] @ V) < 1e-4, "X = U^T G V"
+    eb = compare_basis(g, o)
+    assert eb["M"] < 1e-6 and max(eb["PU"], eb["PV"], eb["s"]) < tol and eb["orth"] < 1e-4, eb
+    es = compare_step(g, o)
+    assert max(es["gproj"], es["m"], es["v"], es["dW"]) < tol, es
+    # rule parity on the oracle's exact basis
+    oe = OracleRun(case, inp, "exact")
+    g2 = GpuRun(case, inp, torch, import_bases=[(st.U, st.s, st.V) for st in oe.states])
+    es2 = compare_step(g2, oe)
+    assert max(es2["gproj"], es2["m"], es2["v"], es2["dW"]) < tol, es2
+    return g, o, es, es2
+
+
+def test_small_two_shapes(torch):
+    case = Case(shapes=[(256, 384), (384, 256)], rank=16, tokens=256, keep=0.25, planted=8, seed=1, tau_p=50.0)
+    _check(case, torch)
+
+
+def test_rank64_several_tiles(torch):
+    case = Case(shapes=[(512, 1024), (512, 1024), (1024, 512)], rank=64, tokens=512, keep=0.1, planted=32, seed=2,
+                tau_p=100.0)
+    _check(case, torch)
+
+
+def test_ragged_tail_shapes(torch):
+    # rows and columns that are not multiples of the 128 x 128 tile, rank not a multiple of 16
+    case = Case(shapes=[(200, 136), (72, 520), (330, 264)], rank=5, tokens=192, keep=0.5, planted=3, seed=3, tau_p=40.0,
+                n_anchor=2)
+    _check(case, torch)
+
+
+def test_rank_above_one_k_chunk(torch):
+    case = Case(shapes=[(384, 640)], rank=96, tokens=512, keep=0.25, planted=48, seed=4, tau_p=80.0)
+    _check(case, torch)
+
+
+def test_split_k_single_matrix(torch):
+    # one matrix with few row tiles and a long K: the projection splits K over several blocks
+    case = Case(shapes=[(256, 4096)], rank=32, tokens=256, keep=0.25, planted=16, seed=5, tau_p=80.0)
+    _check(case, torch)
+
+
+def test_engines_agree(torch):
+    case = Case(shapes=[(256, 384)], rank=16, tokens=256, keep=0.25, planted=8, seed=6, tau_p=50.0)
+    inp = make_inputs(case)
+    a = GpuRun(case, inp, torch)
+    case2 = Case(**{**case.__dict__, "engine": 1})
+    b = GpuRun(case2, inp, torch)
+    assert a.uses_tc and not b.uses_tc
+    assert rel(a.gproj[0], b.gproj[0]) < 1e-4 and rel(a.m[0], b.m[0]) < 1e-4 and rel(a.W[0], b.W[0]) < 1e-5
