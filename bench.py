@@ -1,0 +1,298 @@
+#!/usr/bin/env python
+"""Benchmark of the spectral-correction optimizer step on B200.
+
+A "step" is one pass of the whole hot path over one batch of synthetic gradients: every fourth step an anchor
+gradient arrives (anchor EMA + rank-r basis build), every step runs projection, filter, blend and AdamW over the
+whole parameter set.  The workload is the Llama-style 8B-shaped parameter set (32 layers, hidden 4096, FFN 14336,
+GQA k/v 1024x4096; bf16 gradients, fp32 state, keep 0.1, rank 64).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line on rank 0.  `--impl reference` times the fp64 CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "spectral-correction step: gradient GB/s (and ms per step) on the 8B-shaped parameter set"
+REFRESH_EVERY = 4
+BYTES_PER_ELEM_STEADY = 28.0      # read G (2) + read/write fp32 W, m, v (24) + write bf16 W (2)
+BYTES_PER_ELEM_UPDATE = 28.0      # what the fused update kernel itself moves per element (G is re-read here)
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama8b")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.tmp,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        rows = [l.strip().split(", ") for l in open(self.tmp.name) if l.strip()]
+        os.unlink(self.tmp.name)
+        sm, reasons, mx = [], set(), None
+        for r in rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------ reference arm
+def oracle_sample_run(cfg, steps, warmup):
+    """The fp64 oracle, as it stands, on a bounded sample of the workload: ONE matrix of the set (the smallest
+    shape), full method: every REFRESH_EVERY-th step Eq. 1 + full SVD + truncation, every step projection,
+    filter, blend, AdamW.  Returns (seconds per step, elements, cores, description)."""
+    import numpy as np
+    from oracle import spectral_oracle as so
+    from synth import generator as gen
+    m, n = min(cfg["shapes"], key=lambda s: s[0] * s[1])
+    spec = gen.GradSpec(m=m, n=n, tokens=min(cfg["tokens"], 1024), keep=cfg["keep"], planted_rank=cfg["k"], seed=0)
+    hp = so.Hyper(keep=cfg["keep"])
+    Ganc = gen.stored_to_f64(gen.round_to(gen.anchor_gradient(spec, 0), cfg["dtype"]), cfg["dtype"])
+    G = gen.stored_to_f64(gen.round_to(gen.masked_gradient(spec, 1), cfg["dtype"]), cfg["dtype"])
+    W, mm, vv = [np.asarray(x, np.float64) for x in gen.optimizer_state(spec)]
+    st = so.new_state(m, n)
+    t_total = 0.0
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        if i % REFRESH_EVERY == 0:
+            so.anchor_update(st, Ganc, hp, cfg["r"], mode="exact")
+        Ws, ms, vs, _ = so.correct_and_step([st], [G], [W], [mm], [vv], 100 + i, hp)
+        W, mm, vv = Ws[0], ms[0], vs[0]
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            t_total += dt
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    desc = ("one %dx%d matrix of the set (%d elements of %d), exact mode: Eq.1 + full fp64 SVD every %d steps, "
+            "projection/filter/blend/AdamW every step; %d timed steps" % (m, n, m * n, 0, REFRESH_EVERY, steps))
+    return t_total / max(steps, 1), m * n, cores, desc
+
+
+def run_reference(args):
+    from synth import generator as gen
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = gen.CONFIGS[args.workload]
+    sec, elems, cores, desc = oracle_sample_run(cfg, args.steps, max(args.warmup, 1))
+    gbs = elems * 2 / sec / 1e9
+    total = sum(m * n for m, n in gen.config_shapes(args.workload))
+    desc = desc.replace(" of 0)", " of %d)" % total)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload + " (bounded sample)", "rank": cfg["r"], "keep": cfg["keep"],
+                   "anchor_refresh_every": REFRESH_EVERY, "parallelism": "cpu"},
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ our arm
+def build_workload(name, device, torch):
+    """Parameter set, optimizer state and seeded synthetic gradients resident on the device."""
+    from synth import generator as gen
+    cfg = gen.CONFIGS[name]
+    shapes = gen.config_shapes(name)
+    gdt = torch.bfloat16 if cfg["dtype"] == "bf16" else torch.float32
+    G, Ga, W, M1, M2, Wb = [], [], [], [], [], []
+    per_layer = len(cfg["shapes"])
+    for i, (m, n) in enumerate(shapes):
+        spec = gen.GradSpec(m=m, n=n, tokens=cfg["tokens"], keep=cfg["keep"], planted_rank=cfg["k"], snr=1.0, seed=0,
+                            layer=i // per_layer, mat_id=i % per_layer)
+        G.append(gen.torch_gradients(spec, 1, device, gdt))
+        Ga.append(gen.torch_gradients(spec, 0, device, gdt, anchor=True))
+        g = torch.Generator(device=device); g.manual_seed(1000 + i)
+        W.append(torch.randn((m, n), generator=g, device=device, dtype=torch.float32) * 0.02)
+        M1.append(torch.randn((m, n), generator=g, device=device, dtype=torch.float32) * 10.0)
+        M2.append(torch.rand((m, n), generator=g, device=device, dtype=torch.float32) * 4000.0 + 100.0)
+        Wb.append(torch.empty((m, n), device=device, dtype=torch.bfloat16))
+    return cfg, shapes, dict(G=G, Ga=Ga, W=W, M1=M1, M2=M2, Wb=Wb)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2609_14339_b200 as sc
+    from paper_2609_14339_b200 import build as _build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    sc.load_library()
+
+    cfg, shapes, buf = build_workload(args.workload, device, torch)
+    n_elems = sum(m * n for m, n in shapes)
+    gsize = 2 if cfg["dtype"] == "bf16" else 4
+    hp = sc.Hparams.default(grad_dtype=sc.SC_DTYPE_BF16 if cfg["dtype"] == "bf16" else sc.SC_DTYPE_FP32,
+                            power_iters=1, tau_p=1e-3)
+    plan = sc.Plan(shapes, cfg["r"], cfg["keep"], hp, device=device)
+    lib = sc.load_library()
+
+    def one_step(i):
+        if i % REFRESH_EVERY == 0:
+            plan.anchor_update(buf["Ga"], i)
+        plan.correct_and_step(buf["G"], buf["W"], buf["M1"], buf["M2"], 100 + i, params_bf16=buf["Wb"])
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        one_step(i)
+    sync_all()
+    if plan.get_device_status() != 0:
+        raise SystemExit("device status error after warm-up")
+
+    # ---- timed region: exactly K steps, device-timed, inputs (155 GB) far larger than L2 -------------
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = lib.sc_kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    e0.record()
+    for i in range(args.steps):
+        one_step(args.warmup + i)
+    e1.record()
+    sync_all()
+    ms_total = e0.elapsed_time(e1)
+    launches = lib.sc_kernel_launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    if world > 1:
+        t = torch.tensor([ms_total], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * n_elems * gsize / (ms_step * 1e-3) / 1e9
+
+    # ---- per-phase device times (separate pass, profiling events on) -------------------------------
+    plan.set_profiling(True)
+    nprof = REFRESH_EVERY
+    for i in range(nprof):
+        one_step(args.warmup + args.steps + i)
+    prof = plan.get_profile()
+    plan.set_profiling(False)
+    steady_ms = (prof["projection"]["ms"] + prof["filter"]["ms"] + prof["update"]["ms"]) / nprof
+    refresh_ms = prof["anchor_ema"]["ms"] + prof["basis_passes"]["ms"] + prof["basis_small"]["ms"]
+    update_ms = prof["update"]["ms"] / nprof
+
+    peaks = measured_peaks()
+    upd_gbs = n_elems * BYTES_PER_ELEM_UPDATE / (update_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "fused_update_kernel", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "algorithmic_bytes_per_element": BYTES_PER_ELEM_UPDATE,
+                "launch_ms": update_ms / max(prof["update"]["spans"] / nprof, 1)}
+    step_roofline_ms = max(n_elems * BYTES_PER_ELEM_STEADY / (peaks["hbm_gbs"] * 1e9),
+                           n_elems * 4.0 * cfg["r"] / (peaks["bf16_tflops"] * 1e12)) * 1e3
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "matrices": len(shapes), "elements": n_elems, "rank": cfg["r"],
+                   "keep": cfg["keep"], "tokens": cfg["tokens"], "anchor_refresh_every": REFRESH_EVERY,
+                   "power_iters": 1, "parallelism": "replicas x%d" % world,
+                   "l2": "inputs (>100 GB resident) far larger than L2; no flush needed"},
+        "gpu_launches": int(launches),
+        "steady_step_ms": steady_ms, "anchor_refresh_ms": refresh_ms,
+        "steady_step_roofline_ms": step_roofline_ms, "steady_step_roofline_frac": step_roofline_ms / steady_ms,
+        "phases_ms_per_step": {k: v["ms"] / nprof for k, v in prof.items()},
+        "roofline": roofline,
+        "clocks": clocks,
+        "tensor_cores": plan.uses_tensor_cores(),
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sec, elems, cores, desc = oracle_sample_run(cfg, 4, 1)
+        desc = desc.replace(" of 0)", " of %d)" % n_elems)
+        line["cpu_baseline"] = {"value": elems * gsize / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                                "sample": desc}
+    line["e2e"] = None
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -181,6 +181,25 @@ SC_API sc_status sc_get_stats(sc_plan* plan, sc_mat_stats* stats, float* clip);
 /* Wait for the plan's stream and return the latched device status (SC_OK, SC_ERR_TIMEOUT, SC_ERR_NONFINITE), then clear it. */
 SC_API sc_status sc_get_device_status(sc_plan* plan);
 
+/* Device-time profile by phase of the method. Categories:
+ *   0 anchor EMA (Eq. 1)            1 basis build, passes over the momentum     2 basis build, small factorisations
+ *   3 projection T = G V            4 r x r filter, C^T, norms                  5 fused correction + AdamW update */
+#define SC_PROFILE_CATEGORIES 6
+typedef struct sc_profile {
+  double ms[SC_PROFILE_CATEGORIES];       /* summed device time between event pairs around each group of launches */
+  int64_t spans[SC_PROFILE_CATEGORIES];   /* number of timed groups (one per shape class and phase) */
+} sc_profile;
+
+/* Switch event-based profiling on or off (off by default; when on, each phase is bracketed by CUDA events on
+ * the plan's stream). */
+SC_API sc_status sc_set_profiling(sc_plan* plan, int on);
+
+/* Wait for the plan's stream, write the profile accumulated since the last read-out into *out, and reset it. */
+SC_API sc_status sc_get_profile(sc_plan* plan, sc_profile* out);
+
+/* Number of kernels this library has launched in this process so far. */
+SC_API int64_t sc_kernel_launch_count(void);
+
 /* Step tag of the last accepted anchor (-1 if none) and number of matrices that have a basis. */
 SC_API sc_status sc_get_anchor_info(sc_plan* plan, int64_t* last_tag, int* n_with_basis);
 

@@ -52,6 +52,13 @@ class OptState(C.Structure):
                 ("params_bf16", C.POINTER(C.c_void_p))]
 
 
+class Profile(C.Structure):
+    _fields_ = [("ms", C.c_double * 6), ("spans", C.c_int64 * 6)]
+
+
+PROFILE_CATEGORIES = ("anchor_ema", "basis_passes", "basis_small", "projection", "filter", "update")
+
+
 class MatStats(C.Structure):
     _fields_ = [("g_sqnorm", C.c_float), ("x_sqnorm", C.c_float), ("gproj_sqnorm", C.c_float), ("r_eff", C.c_float)]
 
@@ -75,6 +82,9 @@ EXPORTS = {
     "sc_set_debug_gproj_out": (C.c_int, [_VP, _VPP]),
     "sc_get_stats": (C.c_int, [_VP, C.POINTER(MatStats), C.POINTER(C.c_float)]),
     "sc_get_device_status": (C.c_int, [_VP]),
+    "sc_set_profiling": (C.c_int, [_VP, C.c_int]),
+    "sc_get_profile": (C.c_int, [_VP, C.POINTER(Profile)]),
+    "sc_kernel_launch_count": (C.c_int64, []),
     "sc_get_anchor_info": (C.c_int, [_VP, C.POINTER(C.c_int64), C.POINTER(C.c_int)]),
     "sc_plan_uses_tensor_cores": (C.c_int, [_VP]),
     "sc_status_string": (C.c_char_p, [C.c_int]),
@@ -253,6 +263,14 @@ class Plan:
         tag, k = C.c_int64(), C.c_int()
         _check(self.lib.sc_get_anchor_info(self.handle, C.byref(tag), C.byref(k)), "sc_get_anchor_info")
         return tag.value, k.value
+
+    def set_profiling(self, on: bool):
+        _check(self.lib.sc_set_profiling(self.handle, int(bool(on))), "sc_set_profiling")
+
+    def get_profile(self):
+        pr = Profile()
+        _check(self.lib.sc_get_profile(self.handle, C.byref(pr)), "sc_get_profile")
+        return {name: dict(ms=pr.ms[i], spans=pr.spans[i]) for i, name in enumerate(PROFILE_CATEGORIES)}
 
     def uses_tensor_cores(self) -> bool:
         return bool(self.lib.sc_plan_uses_tensor_cores(self.handle))

@@ -17,6 +17,7 @@ typedef __nv_bfloat16 bf16;
 constexpr int kMaxRank = 256;
 constexpr int kStatsFloats = 8;        // per-matrix statistics slot
 constexpr int kSqnormBlocks = 128;     // partial sums of ||G||^2 per matrix (fixed-order reduction)
+constexpr int kAtbMaxSplits = 16;      // row slices of the A^T B kernel (fixed-order two-stage reduction)
 constexpr int kStagingSlots = 4;       // ring of pinned upload buffers for the per-call pointer table
 
 // Device status word bits (latched, read by sc_get_device_status).
@@ -43,6 +44,7 @@ struct MatDev {
   float* Ct;     // n x rp      C^T = V Xs^T, fp32
   bf16* Cthi;    // n x rk      bf16 split of C^T
   bf16* Ctlo;
+  float* xpart;  // kAtbMaxSplits x rp x rp   row-slice partials of X
   float* sqpart; // kSqnormBlocks partial sums of ||G||^2
   float* stats;  // kStatsFloats
   // anchor-update scratch (slot)
@@ -51,6 +53,7 @@ struct MatDev {
   float* Z;      // n x lp
   float* Z2;     // n x lp
   float* gram;   // lp x lp
+  float* gpart;  // kAtbMaxSplits x lp x lp   row-slice partials of the Gram matrix
   float* rmat;   // lp x lp   Cholesky factor (upper), first pass
   float* rmat2;  // lp x lp   second pass
   float* rinv;   // lp x lp   inverse of the factor
@@ -121,11 +124,17 @@ struct sc_plan {
   std::vector<void*> dbg_out;
   bool table_dirty = true;
   bool tensor_any = false;
+  // optional per-category device timing (cudaEvent pairs around groups of launches)
+  bool prof_on = false;
+  std::vector<cudaEvent_t> prof_events;
+  std::vector<int> prof_cats;         // category of span k; its events are prof_events[2k], [2k+1]
+  size_t prof_used = 0;               // spans recorded since the last read-out
 };
 
 namespace sc {
 
 // ---- host helpers (sc_plan.cu) -------------------------------------------------------------------------
+extern long long g_kernel_launches;   // kernels this library has launched in this process (all plans)
 sc_status upload_table(sc_plan* p);
 sc_status cuda_ok(cudaError_t e);
 
@@ -141,6 +150,9 @@ struct GemmArgs {
   float alpha;
 };
 void launch_gemm(const GemmArgs& a, int count, cudaStream_t s);
+int atb_splits(int rows);
+void launch_atb(const MatDev* tab, const int* idx, int count, int offA, int offB, int offPart, int offOut, int rows,
+                int ca, int cb, int lda, int ldb, cudaStream_t s);
 void launch_epilogue_simt(const MatDev* tab, const int* idx, int count, int m, int n, int rp, int g_bf16,
                           const StepScalars& sc, const float* clip, cudaStream_t s);
 void launch_ema(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, float beta, cudaStream_t s);

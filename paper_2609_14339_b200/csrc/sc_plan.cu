@@ -121,6 +121,7 @@ size_t layout(sc_plan* p, bool assign) {
     md.Xs = cv.take<float>((size_t)rp * rp);
     md.T = cv.take<float>((size_t)c.ksplit * m * rp);
     md.Ct = cv.take<float>(n * rp);
+    md.xpart = cv.take<float>((size_t)atb_splits((int)m) * rp * rp);
     md.sqpart = cv.take<float>(kSqnormBlocks);
     if (c.tensor) {
       md.Uhi = cv.take<bf16>(m * rk); md.Ulo = cv.take<bf16>(m * rk);
@@ -142,13 +143,14 @@ size_t layout(sc_plan* p, bool assign) {
       float* Y = sv.take<float>(m * lp); float* Y2 = sv.take<float>(m * lp);
       float* Z = sv.take<float>(n * lp); float* Z2 = sv.take<float>(n * lp);
       float* gram = sv.take<float>((size_t)lp * lp); float* rmat = sv.take<float>((size_t)lp * lp);
+      float* gpart = sv.take<float>((size_t)atb_splits((int)std::max(m, n)) * lp * lp);
       float* rmat2 = sv.take<float>((size_t)lp * lp); float* rinv = sv.take<float>((size_t)lp * lp);
       float* racc = sv.take<float>((size_t)lp * lp); float* jk = sv.take<float>((size_t)lp * lp);
       float* jv = sv.take<float>((size_t)lp * lp);
       float* ub = sv.take<float>((size_t)lp * rp); float* wb = sv.take<float>((size_t)lp * rp);
       if (assign) {
         MatDev& md = p->host_tab[c.mats[k]];
-        md.Y = Y; md.Y2 = Y2; md.Z = Z; md.Z2 = Z2; md.gram = gram; md.rmat = rmat; md.rmat2 = rmat2;
+        md.Y = Y; md.Y2 = Y2; md.Z = Z; md.Z2 = Z2; md.gram = gram; md.gpart = gpart; md.rmat = rmat; md.rmat2 = rmat2;
         md.rinv = rinv; md.racc = racc; md.jk = jk; md.jv = jv; md.ub = ub; md.wb = wb;
       }
     }
@@ -192,15 +194,40 @@ GemmArgs gemm(sc_plan* p, const int* idx, int offA, int offB, int offC, int M, i
 
 #define OFF(f) ((int)offsetof(MatDev, f))
 
+enum { PROF_EMA = 0, PROF_PASS, PROF_SMALL, PROF_PROJECT, PROF_FILTER, PROF_UPDATE };
+
+// Brackets the launches queued during its lifetime with a pair of events (only when profiling is on).
+struct ProfScope {
+  sc_plan* p;
+  size_t k;
+  bool live;
+  ProfScope(sc_plan* plan, int cat) : p(plan), k(0), live(plan->prof_on) {
+    if (!live) return;
+    k = p->prof_used++;
+    while (p->prof_events.size() < 2 * (k + 1)) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) { live = false; --p->prof_used; return; }
+      p->prof_events.push_back(e);
+    }
+    if (p->prof_cats.size() <= k) p->prof_cats.resize(k + 1);
+    p->prof_cats[k] = cat;
+    cudaEventRecord(p->prof_events[2 * k], p->stream);
+  }
+  ~ProfScope() {
+    if (live) cudaEventRecord(p->prof_events[2 * k + 1], p->stream);
+  }
+};
+
 // Q <- orth(Y) by two rounds of Cholesky QR; Y (rows x lp) is overwritten, tmp is scratch of the same size.
 // keepR: leave the two factors in rmat / rmat2 (and their product in racc) for the caller.
 void cholqr2(sc_plan* p, const int* idx, int cnt, int offY, int offTmp, int rows, bool keepR) {
   const int lp = p->lp;
   cudaStream_t s = p->stream;
-  launch_gemm(gemm(p, idx, offY, offY, OFF(gram), lp, lp, rows, lp, lp, lp, 1, 0), cnt, s);
+  ProfScope ps(p, PROF_SMALL);
+  launch_atb(p->dev_tab, idx, cnt, offY, offY, OFF(gpart), OFF(gram), rows, lp, lp, lp, lp, s);
   launch_chol(p->dev_tab, idx, cnt, lp, OFF(rmat), s);
   launch_gemm(gemm(p, idx, offY, OFF(rinv), offTmp, rows, lp, lp, lp, lp, lp, 0, 0), cnt, s);
-  launch_gemm(gemm(p, idx, offTmp, offTmp, OFF(gram), lp, lp, rows, lp, lp, lp, 1, 0), cnt, s);
+  launch_atb(p->dev_tab, idx, cnt, offTmp, offTmp, OFF(gpart), OFF(gram), rows, lp, lp, lp, lp, s);
   launch_chol(p->dev_tab, idx, cnt, lp, OFF(rmat2), s);
   launch_gemm(gemm(p, idx, offTmp, OFF(rinv), offY, rows, lp, lp, lp, lp, lp, 0, 0), cnt, s);
   if (keepR) launch_gemm(gemm(p, idx, OFF(rmat2), OFF(rmat), OFF(racc), lp, lp, lp, lp, lp, lp, 0, 0), cnt, s);
@@ -223,6 +250,8 @@ sc_status check_ptr_array(const void* const* arr, int n, bool allow_null_entries
 }  // namespace
 
 namespace sc {
+
+long long g_kernel_launches = 0;
 
 sc_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? SC_OK : SC_ERR_CUDA; }
 
@@ -340,6 +369,7 @@ sc_status sc_plan_destroy(sc_plan* p) {
   cudaStreamSynchronize(p->stream);
   for (int i = 0; i < kStagingSlots; ++i)
     if (p->staging_ev[i]) cudaEventDestroy(p->staging_ev[i]);
+  for (cudaEvent_t e : p->prof_events) cudaEventDestroy(e);
   if (p->staging) cudaFreeHost(p->staging);
   delete p;
   return SC_OK;
@@ -369,24 +399,35 @@ sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t 
       idx = c.idx_dyn;
     }
     const int m = (int)c.m, n = (int)c.n;
-    launch_ema(p->dev_tab, idx, cnt, (int64_t)m * n, g_bf16, p->hp.beta_anc, s);                        // Eq. 1
+    {
+      ProfScope ps(p, PROF_EMA);
+      launch_ema(p->dev_tab, idx, cnt, (int64_t)m * n, g_bf16, p->hp.beta_anc, s);                      // Eq. 1
+    }
     if (p->rank > 0) {
       // range finder: Y = M Omega, Q = orth(Y)
-      launch_gemm(gemm(p, idx, OFF(Manc), OFF(omega_t), OFF(Y), m, lp, n, n, n, lp, 0, 1), cnt, s);
+      auto pass = [&](int offB, int offC, bool transposed, int tB) {   // one sweep over the momentum
+        ProfScope ps(p, PROF_PASS);
+        if (!transposed) launch_gemm(gemm(p, idx, OFF(Manc), offB, offC, m, lp, n, n, tB ? n : lp, lp, 0, tB), cnt, s);
+        else launch_gemm(gemm(p, idx, OFF(Manc), offB, offC, n, lp, m, n, lp, lp, 1, 0), cnt, s);
+      };
+      pass(OFF(omega_t), OFF(Y), false, 1);                                                          // Y = M Omega
       cholqr2(p, idx, cnt, OFF(Y), OFF(Y2), m, false);
       for (int it = 0; it < p->q; ++it) {
-        launch_gemm(gemm(p, idx, OFF(Manc), OFF(Y), OFF(Z), n, lp, m, n, lp, lp, 1, 0), cnt, s);   // Z = M^T Q
+        pass(OFF(Y), OFF(Z), true, 0);                                                               // Z = M^T Q
         cholqr2(p, idx, cnt, OFF(Z), OFF(Z2), n, false);
-        launch_gemm(gemm(p, idx, OFF(Manc), OFF(Z), OFF(Y), m, lp, n, n, lp, lp, 0, 0), cnt, s);   // Y = M Z
+        pass(OFF(Z), OFF(Y), false, 0);                                                              // Y = M Z
         cholqr2(p, idx, cnt, OFF(Y), OFF(Y2), m, false);
       }
       // B^T = M^T Q = Qb R ; SVD of the small factor ; U = Q Ub, V = Qb Wb
-      launch_gemm(gemm(p, idx, OFF(Manc), OFF(Y), OFF(Z), n, lp, m, n, lp, lp, 1, 0), cnt, s);
+      pass(OFF(Y), OFF(Z), true, 0);
       cholqr2(p, idx, cnt, OFF(Z), OFF(Z2), n, true);
-      launch_jacobi(p->dev_tab, idx, cnt, lp, rp, p->rank, p->hp.tau_p, s);                           // + Eq. 2
-      launch_gemm(gemm(p, idx, OFF(Y), OFF(ub), OFF(U), m, rp, lp, lp, rp, rp, 0, 0), cnt, s);
-      launch_gemm(gemm(p, idx, OFF(Z), OFF(wb), OFF(V), n, rp, lp, lp, rp, rp, 0, 0), cnt, s);
-      refresh_operands(p, c, idx, cnt);
+      {
+        ProfScope ps(p, PROF_SMALL);
+        launch_jacobi(p->dev_tab, idx, cnt, lp, rp, p->rank, p->hp.tau_p, s);                         // + Eq. 2
+        launch_gemm(gemm(p, idx, OFF(Y), OFF(ub), OFF(U), m, rp, lp, lp, rp, rp, 0, 0), cnt, s);
+        launch_gemm(gemm(p, idx, OFF(Z), OFF(wb), OFF(V), n, rp, lp, lp, rp, rp, 0, 0), cnt, s);
+        refresh_operands(p, c, idx, cnt);
+      }
     }
     for (int id : act) p->has_basis[id] = 1;
   }
@@ -441,6 +482,7 @@ sc_status sc_correct_and_step(sc_plan* p, const void* const* masked_grads, void*
     const int cnt = (int)c.mats.size(), m = (int)c.m, n = (int)c.n;
     const int* idx = c.idx_all;
     if (rp > 0) {
+      ProfScope ps(p, PROF_PROJECT);
       if (c.tensor) {
         sc_status e = tc_launch_project(p, c, idx, cnt);                                                  // T = G V
         if (e != SC_OK) return e;
@@ -448,8 +490,9 @@ sc_status sc_correct_and_step(sc_plan* p, const void* const* masked_grads, void*
       } else {
         launch_gemm(gemm(p, idx, OFF(G), OFF(V), OFF(T), m, rp, n, n, rp, rp, 0, 0, g_bf16), cnt, s);
       }
-      launch_gemm(gemm(p, idx, OFF(U), OFF(T), OFF(X), rp, rp, m, rp, rp, rp, 1, 0), cnt, s);        // X = U^T T
     }
+    ProfScope ps(p, PROF_FILTER);
+    if (rp > 0) launch_atb(p->dev_tab, idx, cnt, OFF(U), OFF(T), OFF(xpart), OFF(X), m, rp, rp, rp, rp, s);  // X = U^T T
     if (want_norm) launch_sqnorm(p->dev_tab, idx, cnt, (int64_t)m * n, g_bf16, s);
     launch_xs(p->dev_tab, idx, cnt, rp, p->rank, 0.f, scale, hp.alpha, s);                             // D X D
     if (rp > 0) {
@@ -460,6 +503,7 @@ sc_status sc_correct_and_step(sc_plan* p, const void* const* masked_grads, void*
   };
   auto update = [&](ShapeClass& c) -> sc_status {
     const int cnt = (int)c.mats.size(), m = (int)c.m, n = (int)c.n;
+    ProfScope ps(p, PROF_UPDATE);
     if (c.tensor) return tc_launch_epilogue(p, c, c.idx_all, cnt, sc);
     launch_epilogue_simt(p->dev_tab, c.idx_all, cnt, m, n, rp, g_bf16, sc, p->clip_dev, s);
     return SC_OK;
@@ -602,6 +646,30 @@ sc_status sc_get_anchor_info(sc_plan* p, int64_t* last_tag, int* n_with_basis) {
   }
   return SC_OK;
 }
+
+sc_status sc_set_profiling(sc_plan* p, int on) {
+  if (!p) return SC_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(p->stream) != cudaSuccess) return SC_ERR_CUDA;
+  p->prof_on = on != 0;
+  p->prof_used = 0;
+  return SC_OK;
+}
+
+sc_status sc_get_profile(sc_plan* p, sc_profile* out) {
+  if (!p || !out) return SC_ERR_INVALID_ARG;
+  memset(out, 0, sizeof(*out));
+  if (cudaStreamSynchronize(p->stream) != cudaSuccess) return SC_ERR_CUDA;
+  for (size_t k = 0; k < p->prof_used; ++k) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, p->prof_events[2 * k], p->prof_events[2 * k + 1]) != cudaSuccess) return SC_ERR_CUDA;
+    const int cat = p->prof_cats[k];
+    if (cat >= 0 && cat < SC_PROFILE_CATEGORIES) { out->ms[cat] += ms; out->spans[cat] += 1; }
+  }
+  p->prof_used = 0;
+  return SC_OK;
+}
+
+int64_t sc_kernel_launch_count(void) { return (int64_t)g_kernel_launches; }
 
 int sc_plan_uses_tensor_cores(const sc_plan* p) { return p && p->tensor_any ? 1 : 0; }
 

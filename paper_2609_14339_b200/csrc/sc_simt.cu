@@ -124,6 +124,7 @@ void launch_gemm(const GemmArgs& a, int count, cudaStream_t s) {
   if (count <= 0 || a.M <= 0 || a.N <= 0) return;
   dim3 grid((a.N + BN - 1) / BN, (a.M + BM - 1) / BM, count);
   gemm_kernel<false><<<grid, 256, 0, s>>>(a, EpiAdamW{});
+  ++g_kernel_launches;
 }
 
 void launch_epilogue_simt(const MatDev* tab, const int* idx, int count, int m, int n, int rp, int g_bf16,
@@ -138,6 +139,97 @@ void launch_epilogue_simt(const MatDev* tab, const int* idx, int count, int m, i
   EpiAdamW e{sc, clip, g_bf16};
   dim3 grid((n + BN - 1) / BN, (m + BM - 1) / BM, count);
   gemm_kernel<true><<<grid, 256, 0, s>>>(a, e);
+  ++g_kernel_launches;
+}
+
+// =====================================================================================================
+// Tall-skinny Gram-type product  C = A^T B  (A: rows x ca, B: rows x cb, both row-major) split over the
+// rows: block s of the grid reduces its slice of rows into part[s] (ca x cb), a second kernel adds the
+// slices in a fixed order. Used for X = U^T T and for the Gram matrices of the Cholesky QR.
+// =====================================================================================================
+template <int MT>
+__global__ void __launch_bounds__(256) atb_kernel(const MatDev* tab, const int* idx, int offA, int offB, int offPart,
+                                                  int rows, int ca, int cb, int lda, int ldb, int rows_per_split) {
+  constexpr int TS = 16 * MT;          // output tile edge
+  __shared__ float As[32][TS + 1];
+  __shared__ float Bs[32][TS + 1];
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const float* A = field<const float>(md, offA);
+  const float* B = field<const float>(md, offB);
+  float* part = field<float>(md, offPart) + (size_t)blockIdx.x * ca * cb;
+  const int tiles_b = (cb + TS - 1) / TS;
+  const int i0 = (blockIdx.y / tiles_b) * TS, j0 = (blockIdx.y % tiles_b) * TS;
+  const int r_lo = blockIdx.x * rows_per_split, r_hi = min(rows, r_lo + rows_per_split);
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  float acc[MT][MT] = {};
+  for (int r0 = r_lo; r0 < r_hi; r0 += 32) {
+    for (int e = tid; e < 32 * TS; e += 256) {
+      const int rr = e / TS, c = e % TS;
+      const int gr = r0 + rr;
+      As[rr][c] = (gr < r_hi && i0 + c < ca) ? A[(size_t)gr * lda + i0 + c] : 0.f;
+      Bs[rr][c] = (gr < r_hi && j0 + c < cb) ? B[(size_t)gr * ldb + j0 + c] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int rr = 0; rr < 32; ++rr) {
+      float av[MT], bv[MT];
+#pragma unroll
+      for (int i = 0; i < MT; ++i) av[i] = As[rr][ty + 16 * i];
+#pragma unroll
+      for (int j = 0; j < MT; ++j) bv[j] = Bs[rr][tx + 16 * j];
+#pragma unroll
+      for (int i = 0; i < MT; ++i)
+#pragma unroll
+        for (int j = 0; j < MT; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < MT; ++i)
+#pragma unroll
+    for (int j = 0; j < MT; ++j) {
+      const int gi = i0 + ty + 16 * i, gj = j0 + tx + 16 * j;
+      if (gi < ca && gj < cb) part[(size_t)gi * cb + gj] = acc[i][j];
+    }
+}
+
+__global__ void __launch_bounds__(256) sum_slices_kernel(const MatDev* tab, const int* idx, int offPart, int offOut,
+                                                         int numel, int nsplit) {
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const float* part = field<const float>(md, offPart);
+  float* out = field<float>(md, offOut);
+  for (int e = blockIdx.x * 256 + threadIdx.x; e < numel; e += gridDim.x * 256) {
+    float t = 0.f;
+    for (int s = 0; s < nsplit; ++s) t += part[(size_t)s * numel + e];
+    out[e] = t;
+  }
+}
+
+int atb_splits(int rows) {
+  int s = (rows + 1023) / 1024;
+  return s < 1 ? 1 : (s > kAtbMaxSplits ? kAtbMaxSplits : s);
+}
+
+void launch_atb(const MatDev* tab, const int* idx, int count, int offA, int offB, int offPart, int offOut, int rows,
+                int ca, int cb, int lda, int ldb, cudaStream_t s) {
+  if (count <= 0 || ca <= 0 || cb <= 0) return;
+  const int nsplit = atb_splits(rows);
+  const int rps = ((rows + nsplit - 1) / nsplit + 31) / 32 * 32;
+  const int big = ca > cb ? ca : cb;
+  const int mt = big <= 16 ? 1 : big <= 32 ? 2 : big <= 64 ? 4 : 8;
+  const int ts = 16 * mt;
+  dim3 grid(nsplit, ((ca + ts - 1) / ts) * ((cb + ts - 1) / ts), count);
+  switch (mt) {
+    case 1: atb_kernel<1><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps); break;
+    case 2: atb_kernel<2><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps); break;
+    case 4: atb_kernel<4><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps); break;
+    default: atb_kernel<8><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps); break;
+  }
+  ++g_kernel_launches;
+  const int numel = ca * cb;
+  sum_slices_kernel<<<dim3((numel + 255) / 256 < 64 ? (numel + 255) / 256 : 64, 1, count), 256, 0, s>>>(
+      tab, idx, offPart, offOut, numel, nsplit);
+  ++g_kernel_launches;
 }
 
 // =====================================================================================================
@@ -184,6 +276,7 @@ void launch_ema(const MatDev* tab, const int* idx, int count, int64_t numel, int
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (blocks < 1) blocks = 1;
   ema_kernel<<<dim3((unsigned)blocks, 1, count), 256, 0, s>>>(tab, idx, numel, g_bf16, beta);
+  ++g_kernel_launches;
 }
 
 // =====================================================================================================
@@ -208,6 +301,7 @@ __global__ void sketch_t_kernel(float* omega_t, int lp, int l, int64_t n, uint64
 void launch_sketch(float* omega_t, int lp, int l, int64_t n, uint64_t seed, cudaStream_t s) {
   if (lp <= 0) return;
   sketch_t_kernel<<<dim3((unsigned)((n + 255) / 256), lp), 256, 0, s>>>(omega_t, lp, l, n, seed);
+  ++g_kernel_launches;
 }
 
 __global__ void sketch_rm_kernel(float* omega, int64_t rows, int width, uint64_t seed) {
@@ -220,6 +314,7 @@ void launch_sketch_rowmajor(float* omega, int64_t rows, int width, uint64_t seed
   const int64_t tot = rows * width;
   if (tot <= 0) return;
   sketch_rm_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, s>>>(omega, rows, width, seed);
+  ++g_kernel_launches;
 }
 
 // =====================================================================================================
@@ -271,6 +366,7 @@ __global__ void __launch_bounds__(256) chol_kernel(const MatDev* tab, const int*
 void launch_chol(const MatDev* tab, const int* idx, int count, int lp, int offR, cudaStream_t s) {
   if (count <= 0 || lp <= 0) return;
   chol_kernel<<<count, 256, 0, s>>>(tab, idx, lp, offR);
+  ++g_kernel_launches;
 }
 
 // =====================================================================================================
@@ -372,6 +468,7 @@ void launch_jacobi(const MatDev* tab, const int* idx, int count, int lp, int rp,
                    cudaStream_t s) {
   if (count <= 0 || lp <= 0 || rp <= 0) return;
   jacobi_kernel<<<count, kJacobiThreads, 0, s>>>(tab, idx, lp, rp, rank, tau_p);
+  ++g_kernel_launches;
 }
 
 // Eq. 2 from stored singular values (used after a basis import).
@@ -387,6 +484,7 @@ void launch_filter_weights(const MatDev* tab, const int* idx, int count, int rp,
                            cudaStream_t s) {
   if (count <= 0 || rp <= 0) return;
   filter_weights_kernel<<<count, 256, 0, s>>>(tab, idx, rp, rank, tau_p);
+  ++g_kernel_launches;
 }
 
 // =====================================================================================================
@@ -420,6 +518,7 @@ void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int
   int64_t tot = (int64_t)(m > n ? m : n) * rp;
   int blocks = (int)((tot + 255) / 256 < 1184 ? (tot + 255) / 256 : 1184);
   split_basis_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, m, n, rp, rk);
+  ++g_kernel_launches;
 }
 
 __global__ void __launch_bounds__(256) split_ct_kernel(const MatDev* tab, const int* idx, int64_t numel, int rp, int rk) {
@@ -436,6 +535,7 @@ void launch_split_ct(const MatDev* tab, const int* idx, int count, int n, int rp
   const int64_t tot = (int64_t)n * rp;
   int blocks = (int)((tot + 255) / 256 < 296 ? (tot + 255) / 256 : 296);
   split_ct_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, tot, rp, rk);
+  ++g_kernel_launches;
 }
 
 // =====================================================================================================
@@ -465,6 +565,7 @@ __global__ void __launch_bounds__(256) sqnorm_kernel(const MatDev* tab, const in
 void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, cudaStream_t s) {
   if (count <= 0) return;
   sqnorm_kernel<<<dim3(kSqnormBlocks, 1, count), 256, 0, s>>>(tab, idx, numel, g_bf16);
+  ++g_kernel_launches;
 }
 
 // =====================================================================================================
@@ -506,6 +607,7 @@ void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, f
                cudaStream_t s) {
   if (count <= 0) return;
   xs_kernel<<<count, 256, 0, s>>>(tab, idx, rp, rank, coef, scale, alpha);
+  ++g_kernel_launches;
 }
 
 // Global-norm clip factor over all matrices, summed in matrix order by one thread block.
@@ -525,6 +627,7 @@ __global__ void clip_kernel(const MatDev* tab, int n_mats, float max_norm, float
 
 void launch_clip(const MatDev* tab, int n_mats, float max_norm, float* clip, cudaStream_t s) {
   clip_kernel<<<1, 256, 0, s>>>(tab, n_mats, max_norm, clip);
+  ++g_kernel_launches;
 }
 
 // Copies between a dense rows x cols matrix and its zero-padded rows x cols_dst copy (basis import/export).
@@ -540,6 +643,7 @@ void launch_pad_copy(float* dst, int ldd, const float* src, int lds, int rows, i
   const int64_t tot = (int64_t)rows * cols_dst;
   if (tot <= 0) return;
   pad_copy_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, s>>>(dst, ldd, src, lds, rows, cols, cols_dst);
+  ++g_kernel_launches;
 }
 
 void launch_unpad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, cudaStream_t s) {
@@ -561,6 +665,7 @@ void launch_reduce_partials(const MatDev* tab, const int* idx, int count, int64_
   if (count <= 0 || ksplit <= 1) return;
   int blocks = (int)((numel + 255) / 256 < 592 ? (numel + 255) / 256 : 592);
   reduce_partials_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, numel, ksplit);
+  ++g_kernel_launches;
 }
 
 }  // namespace sc

@@ -455,6 +455,7 @@ sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count
   dim3 grid((m + 127) / 128, c.ksplit, count);
   project_kernel<<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), m, n, rp,
                                                  cps, stages, cols, p->status_dev);
+  ++g_kernel_launches;
   return cuda_ok(cudaGetLastError());
 }
 
@@ -464,6 +465,7 @@ sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int coun
   const size_t smem = 4 * kTileBytes + 1024 + 64;
   fused_update_kernel<<<grid, 256, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), m, n,
                                                       p->rp, sc, p->clip_dev, p->status_dev);
+  ++g_kernel_launches;
   return cuda_ok(cudaGetLastError());
 }
 
