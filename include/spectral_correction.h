@@ -163,6 +163,34 @@ SC_API sc_status sc_import_basis(sc_plan* plan, int mat, const void* U_dev, cons
  * row-major, on the raw masked gradient) and X = U^T G V (rank x rank fp32, row-major). */
 SC_API sc_status sc_export_projection(sc_plan* plan, int mat, void* T_dev, void* X_dev);
 
+/* sc_project_static - X = U^T G V for ONE matrix, without a plan, a workspace or any allocation.
+ * (The paper has no counterpart to this call; it is a packaging of the projection step for constrained callers.)
+ *
+ * Who needs it: code that may not allocate device memory at the point where it wants the projection - for
+ * example a hook that runs after a framework's caching allocator has taken all of HBM, or a monitoring path
+ * that must not take the allocator lock or cause the device-wide synchronisation an allocation implies. Such
+ * callers cannot pass a workspace either, so the intermediates (T = G V and the row-slice partial sums of
+ * U^T T) live in one fixed 8 MiB array that is part of the library image: every GPU that loads the library
+ * holds those 8 MiB until the process exits.
+ *
+ *   G_dev       device: rows x cols, row-major, grad_dtype (sc_dtype)          U_dev  device: rows x rank fp32
+ *   V_dev       device: cols x rank fp32                                        X_dev  device: rank x rank fp32 (out)
+ *   stream      a cudaStream_t (as void*), NULL = default stream. The three kernels are queued on it.
+ *
+ * Limits and sharing:
+ *   - rows * rank + 16 * rank * rank floats must fit in the 8 MiB array (2,097,152 floats), rank <= 256;
+ *     anything larger returns SC_ERR_TOO_LARGE and nothing is launched.
+ *   - The call never calls cudaMalloc, cudaFree or any allocating routine.
+ *   - All calls (from any thread, on any stream of one device) use the SAME array, which keeps whatever the
+ *     previous call left in it. Every element this call reads it has written first, so nothing has to be cleared;
+ *     but two calls whose kernels overlap on the GPU would overwrite each other's intermediates: queue them on
+ *     one stream, or order them with events.
+ *   - The first call on each device looks up the array's device address (that device must be current, as for
+ *     every call). Make that first call during set-up, before any stream capture is begun.
+ * Errors: INVALID_ARG (NULL pointer), DTYPE, SHAPE, TOO_LARGE, CUDA. */
+SC_API sc_status sc_project_static(const void* G_dev, int grad_dtype, const void* U_dev, const void* V_dev,
+                                   int64_t rows, int64_t cols, int rank, void* X_dev, void* stream);
+
 /* Copy the anchor momentum (rows x cols fp32) to / from a caller device buffer. */
 SC_API sc_status sc_export_anchor_momentum(sc_plan* plan, int mat, void* M_dev);
 SC_API sc_status sc_import_anchor_momentum(sc_plan* plan, int mat, const void* M_dev);

@@ -76,6 +76,7 @@ EXPORTS = {
     "sc_export_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
     "sc_import_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
     "sc_export_projection": (C.c_int, [_VP, C.c_int, _VP, _VP]),
+    "sc_project_static": (C.c_int, [_VP, C.c_int, _VP, _VP, C.c_int64, C.c_int64, C.c_int, _VP, _VP]),
     "sc_export_anchor_momentum": (C.c_int, [_VP, C.c_int, _VP]),
     "sc_import_anchor_momentum": (C.c_int, [_VP, C.c_int, _VP]),
     "sc_export_sketch": (C.c_int, [_VP, C.c_int64, C.c_int, _VP]),
@@ -142,6 +143,32 @@ def _ptr_array(tensors: Optional[Sequence], n: int, allow_none: bool):
                 raise ValueError("tensor %d must be a contiguous CUDA tensor" % i)
             arr[i] = t.data_ptr()
     return arr
+
+
+def project_static(G, U, V, X_out=None, stream=None):
+    """X = U^T G V through sc_project_static: no plan, no workspace, no allocation inside the library.
+
+    For callers that cannot allocate device memory where they need the projection (all of HBM already owned by
+    a caching allocator, or a path that must not synchronise the device). G: rows x cols bf16/fp32, U: rows x r
+    fp32, V: cols x r fp32, all contiguous CUDA tensors. Pass X_out (r x r fp32) to keep this wrapper from
+    allocating too. Calls share one 8 MiB scratch array: do not let two of them overlap on the GPU.
+    """
+    import torch
+    lib = load_library()
+    rows, cols = G.shape
+    r = U.shape[1]
+    assert U.shape == (rows, r) and V.shape == (cols, r) and U.dtype == torch.float32 and V.dtype == torch.float32
+    for t in (G, U, V):
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError("tensors must be contiguous CUDA tensors")
+    if X_out is None:
+        X_out = torch.empty((r, r), dtype=torch.float32, device=G.device)
+    dt = SC_DTYPE_BF16 if G.dtype == torch.bfloat16 else SC_DTYPE_FP32
+    st = stream if stream is not None else torch.cuda.current_stream(G.device)
+    with torch.cuda.device(G.device):
+        _check(lib.sc_project_static(G.data_ptr(), dt, U.data_ptr(), V.data_ptr(), rows, cols, r, X_out.data_ptr(),
+                                     st.cuda_stream), "sc_project_static")
+    return X_out
 
 
 class Plan:
