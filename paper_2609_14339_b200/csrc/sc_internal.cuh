@@ -63,6 +63,7 @@ struct MatDev {
   float* ub;     // lp x rp   left singular vectors of the small factor (selected, sorted)
   float* wb;     // lp x rp   right singular vectors
   const float* omega_t;  // lp x n  Rademacher sketch, transposed (shared by a shape class)
+  const float* omega;    // n x lp  the same sketch, row-major (tensor-core classes only)
   // per call
   const void* G;      // masked gradient
   const void* Ganc;   // anchor gradient
@@ -72,7 +73,8 @@ struct MatDev {
   bf16* Wb;           // optional bf16 weight copy
   float* gproj_dbg;   // optional G_proj output
   int m, n;
-  int pad0, pad1;
+  int inst;           // index of this matrix inside its shape class (selects its tensor maps)
+  int pad1;
 };
 
 // All matrices of one shape; kernels are launched once per class with blockIdx.z = instance.
@@ -80,6 +82,7 @@ struct ShapeClass {
   int64_t m = 0, n = 0;
   std::vector<int> mats;   // matrix ids, in plan order
   float* omega_t = nullptr;
+  float* omega = nullptr;
   int* idx_all = nullptr;  // device: mats[]
   int* idx_dyn = nullptr;  // device: subset list written per call (anchor arrivals)
   bool tensor = false;     // served by the tcgen05 kernels
@@ -158,6 +161,7 @@ void launch_epilogue_simt(const MatDev* tab, const int* idx, int count, int m, i
 void launch_ema(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, float beta, cudaStream_t s);
 void launch_sketch(float* omega_t, int lp, int l, int64_t n, uint64_t seed, cudaStream_t s);
 void launch_sketch_rowmajor(float* omega, int64_t rows, int width, uint64_t seed, cudaStream_t s);
+void launch_sketch_padded(float* omega, int64_t rows, int lp, int l, uint64_t seed, cudaStream_t s);
 void launch_chol(const MatDev* tab, const int* idx, int count, int lp, int offR, cudaStream_t s);
 void launch_jacobi(const MatDev* tab, const int* idx, int count, int lp, int rp, int rank, float tau_p, cudaStream_t s);
 void launch_filter_weights(const MatDev* tab, const int* idx, int count, int rp, int rank, float tau_p, cudaStream_t s);
@@ -178,5 +182,6 @@ sc_status tc_init();   // resolves the driver entry point for tensor-map encodin
 sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_call_part);
 sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count);   // T = G V
 sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc);
+sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, int which);
 
 }  // namespace sc

@@ -42,7 +42,7 @@ bool derive_dims(int rank, const sc_hparams* hp, Dims* d) {
   d->rp = rank > 0 ? round_up_int(rank, 16) : 0;
   d->rk = round_up_int(d->rp, 64);
   d->l = l;
-  d->lp = rank > 0 ? round_up_int(l, 16) : 0;
+  d->lp = rank > 0 ? round_up_int(l, 32) : 0;   // whole 32-column swizzle atoms for the tf32 operands
   d->q = hp->power_iters;
   return true;
 }
@@ -102,6 +102,8 @@ size_t layout(sc_plan* p, bool assign) {
     int* a = cv.take<int>(c.mats.size());
     int* b = cv.take<int>(c.mats.size());
     float* om = cv.take<float>((size_t)lp * c.n);
+    float* omr = c.tensor ? cv.take<float>((size_t)lp * c.n) : nullptr;
+    if (assign) c.omega = omr;
     void* tm = c.tensor ? (void*)cv.take<char>(tc_tmaps_bytes((int)c.mats.size())) : nullptr;
     if (assign) { c.idx_all = a; c.idx_dyn = b; c.omega_t = om; c.tmaps = tm; }
   }
@@ -130,6 +132,8 @@ size_t layout(sc_plan* p, bool assign) {
     }
     md.stats = assign ? p->stats_dev + (size_t)i * kStatsFloats : nullptr;
     md.omega_t = c.omega_t;
+    md.omega = c.omega;
+    md.inst = p->inst_of[i];
     if (assign) p->host_tab[i] = md;
   }
   // anchor-update scratch: one region, reused by the classes in turn (slot = instance index)
@@ -335,7 +339,7 @@ sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int 
   p->dbg_out.assign(n_mats, nullptr);
   layout(p, true);
   for (auto& c : p->classes)
-    for (int id : c.mats) p->host_tab[id].omega_t = c.omega_t;
+    for (int id : c.mats) { p->host_tab[id].omega_t = c.omega_t; p->host_tab[id].omega = c.omega; }
 
   if (p->tensor_any && tc_init() != SC_OK) { delete p; return SC_ERR_CUDA; }
 
@@ -353,6 +357,7 @@ sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int 
     ok = ok && cudaMemcpyAsync(c.idx_all, c.mats.data(), c.mats.size() * sizeof(int), cudaMemcpyHostToDevice, s) ==
                    cudaSuccess;
     if (p->lp > 0) launch_sketch(c.omega_t, p->lp, p->l, c.n, p->hp.seed, s);
+    if (p->lp > 0 && c.omega) launch_sketch_padded(c.omega, c.n, p->lp, p->l, p->hp.seed, s);
     if (c.tensor && ok) ok = tc_encode_class(p, c, true, false) == SC_OK;
   }
   p->table_dirty = true;
@@ -407,6 +412,7 @@ sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t 
       // range finder: Y = M Omega, Q = orth(Y)
       auto pass = [&](int offB, int offC, bool transposed, int tB) {   // one sweep over the momentum
         ProfScope ps(p, PROF_PASS);
+        if (c.tensor) { tc_launch_pass(p, c, idx, cnt, transposed ? 1 : (tB ? 0 : 2)); return; }
         if (!transposed) launch_gemm(gemm(p, idx, OFF(Manc), offB, offC, m, lp, n, n, tB ? n : lp, lp, 0, tB), cnt, s);
         else launch_gemm(gemm(p, idx, OFF(Manc), offB, offC, n, lp, m, n, lp, lp, 1, 0), cnt, s);
       };

@@ -310,6 +310,21 @@ __global__ void sketch_rm_kernel(float* omega, int64_t rows, int width, uint64_t
   omega[e] = sketch_entry(seed, (uint64_t)(e / width), (uint64_t)(e % width));
 }
 
+// Row-major n x lp copy of the sketch, columns l..lp-1 zero.
+__global__ void sketch_padded_kernel(float* omega, int64_t rows, int lp, int l, uint64_t seed) {
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= rows * lp) return;
+  const int c = (int)(e % lp);
+  omega[e] = c < l ? sketch_entry(seed, (uint64_t)(e / lp), (uint64_t)c) : 0.f;
+}
+
+void launch_sketch_padded(float* omega, int64_t rows, int lp, int l, uint64_t seed, cudaStream_t s) {
+  const int64_t tot = rows * lp;
+  if (tot <= 0) return;
+  sketch_padded_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, s>>>(omega, rows, lp, l, seed);
+  ++g_kernel_launches;
+}
+
 void launch_sketch_rowmajor(float* omega, int64_t rows, int width, uint64_t seed, cudaStream_t s) {
   const int64_t tot = rows * width;
   if (tot <= 0) return;

@@ -99,8 +99,11 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16(int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-constexpr int kMapsPerMat = 7;   // G, Vthi, Vtlo, Uhi, Ulo, Cthi, Ctlo
-enum { MAP_G = 0, MAP_VTHI, MAP_VTLO, MAP_UHI, MAP_ULO, MAP_CTHI, MAP_CTLO };
+constexpr int kMapsPerMat = 12;
+enum { MAP_G = 0, MAP_VTHI, MAP_VTLO, MAP_UHI, MAP_ULO, MAP_CTHI, MAP_CTLO,
+       MAP_M_K,      // anchor momentum as a K-major A operand: box 32 floats x 128 rows
+       MAP_M_MN,     // anchor momentum as an MN-major A operand: box 32 floats x 32 rows (one swizzle atom column)
+       MAP_Y, MAP_Z, MAP_OMEGA };   // m x lp, n x lp, n x lp row-major fp32 as MN-major B operands: box 32 x 32
 constexpr int kTileBytes = 128 * 128;   // 128 rows x 64 bf16
 
 // =====================================================================================================
@@ -123,7 +126,7 @@ project_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, cons
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int inst = blockIdx.z;
   const MatDev& md = tab[idx[inst]];
-  const CUtensorMap* mp = maps + (size_t)inst * kMapsPerMat;
+  const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
   const int row0 = blockIdx.x * 128;
   const int nchunks = (n + 63) >> 6;
   const int c0 = blockIdx.y * cps;
@@ -203,6 +206,135 @@ project_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, cons
 }
 
 // =====================================================================================================
+// One sweep over the anchor momentum for the range finder, tf32 tensor cores, fp32 operands read as they are:
+//   TRANS = false:  OUT[m x lp] = M  * B,   B = Omega or Z (n x lp row-major)
+//   TRANS = true :  OUT[n x lp] = M^T * B,  B = Y (m x lp row-major)
+// K advances 32 per pipeline stage. B is always an MN-major operand (its rows are the K index): lp/32 swizzle
+// atoms of 32 K-rows x 128 bytes. A is K-major for M (rows of M are rows of OUT) and MN-major for M^T (columns
+// of M are rows of OUT: 4 atoms of 32 K-rows x 128 bytes). Same warp roles as project_kernel.
+// =====================================================================================================
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// MN-major operand of 32-bit elements: the only layout the tensor core takes is the 128-byte swizzle with
+// 32-byte atomicity (32-byte chunks of a 128-byte row XORed with the row index mod 4; TMA writes it with
+// SWIZZLE_128B_ATOM_32B). Atoms are 4 K-rows x 128 bytes; consecutive atoms along MN are `lbo` bytes apart,
+// consecutive 4-row K groups 512 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_mn128(uint32_t saddr, uint32_t lbo) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(512 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)1 << 61);
+}
+__device__ __forceinline__ uint32_t umma_idesc_tf32(int N, int a_mn, int b_mn) {
+  return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+constexpr int kPassK = 32;                       // K per stage
+constexpr int kAtomBytes = kPassK * 128;         // one MN-major atom column: 32 K-rows x 128 bytes
+
+template <bool TRANS>
+__global__ void __launch_bounds__(192, 1)
+pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const CUtensorMap* __restrict__ maps,
+            int b_map, int out_off, int rows_out, int kdim, int lp, int stages, uint32_t tmem_cols, unsigned* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int b_bytes = (lp / 32) * kAtomBytes;
+  const int stage_bytes = kTileBytes + b_bytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+  uint64_t* empty = full + stages;
+  uint64_t* accum = empty + stages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* never_flag = abort_flag + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
+  const int row0 = blockIdx.x * 128;
+  const int nchunks = (kdim + kPassK - 1) / kPassK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(accum, 1);
+    *abort_flag = 0;
+    *never_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_d = *tmem_slot;
+
+  if (warp == 0 && lane == 0) {
+    const CUtensorMap* amap = mp + (TRANS ? MAP_M_MN : MAP_M_K);
+    const CUtensorMap* bmap = mp + b_map;
+    tensormap_acquire(amap); tensormap_acquire(bmap);
+    int issued = 0;
+    for (int i = 0; i < nchunks; ++i, ++issued) {
+      const int s = i % stages;
+      if (!mbar_wait(&empty[s], ((i / stages) & 1) ^ 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
+      uint8_t* st = smem + (size_t)s * stage_bytes;
+      mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
+      const int k0 = i * kPassK;
+      if (!TRANS) {
+        tma_load_2d(st, amap, &full[s], k0, row0);                                    // 128 rows x 32 floats
+      } else {
+#pragma unroll
+        for (int a = 0; a < 4; ++a) tma_load_2d(st + a * kAtomBytes, amap, &full[s], row0 + 32 * a, k0);
+      }
+      for (int a = 0; a < lp / 32; ++a) tma_load_2d(st + kTileBytes + a * kAtomBytes, bmap, &full[s], 32 * a, k0);
+    }
+    if (*abort_flag)
+      for (int i = max(0, issued - stages); i < issued; ++i) mbar_wait(&full[i % stages], (i / stages) & 1, never_flag);
+  } else if (warp == 1 && lane == 0) {
+    const uint32_t idesc = umma_idesc_tf32(lp, TRANS ? 1 : 0, 1);
+    for (int i = 0; i < nchunks; ++i) {
+      const int s = i % stages;
+      if (!mbar_wait(&full[s], (i / stages) & 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
+      tc_fence_after();
+      const uint32_t a = smem_u32(smem + (size_t)s * stage_bytes);
+      const uint32_t b = a + kTileBytes;
+#pragma unroll
+      for (int k = 0; k < kPassK / 8; ++k) {
+        const uint64_t ad = TRANS ? umma_desc_mn128(a + k * 1024, kAtomBytes) : umma_desc_k128(a + k * 32);
+        umma_tf32(tmem_d, ad, umma_desc_mn128(b + k * 1024, kAtomBytes), idesc, (i | k) != 0);
+      }
+      umma_commit(&empty[s]);
+    }
+    umma_commit(accum);
+  } else if (warp >= 2) {
+    const int q = warp & 3;
+    const int row = row0 + q * 32 + lane;
+    bool ok = mbar_wait(accum, 0, abort_flag);
+    if (!ok && lane == 0) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
+    ok = __all_sync(0xffffffffu, ok) && !*abort_flag;
+    tc_fence_after();
+    if (ok) {
+      float* out = *reinterpret_cast<float* const*>(reinterpret_cast<const char*>(&md) + out_off) + (size_t)row * lp;
+      for (int c = 0; c < lp; c += 16) {
+        float v[16];
+        tmem_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + c, v);
+        tmem_ld_wait();
+        if (row < rows_out) {
+#pragma unroll
+          for (int j = 0; j < 16; j += 4)
+            *reinterpret_cast<float4*>(out + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_d, tmem_cols);
+}
+
+// =====================================================================================================
 // Fused correction + AdamW for one 128 x 128 tile.
 //   mainloop (one elected thread): R = (Uhi + Ulo)(Cthi + Ctlo)^T over K = rank, three bf16 MMAs per K step
 //   (hi*hi, hi*lo, lo*hi; lo*lo is below fp32 resolution), accumulated in TMEM;
@@ -237,7 +369,7 @@ fused_update_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int inst = blockIdx.z;
   const MatDev& md = tab[idx[inst]];
-  const CUtensorMap* mp = maps + (size_t)inst * kMapsPerMat;
+  const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
   const int col0 = blockIdx.x * 128, row0 = blockIdx.y * 128;
   const int nch = (rp + 63) >> 6;
 
@@ -385,7 +517,9 @@ sc_status tc_init() {
   static bool attrs_done = false;
   if (!attrs_done) {
     if (cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(fused_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024) != cudaSuccess)
+        cudaFuncSetAttribute(fused_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
       return SC_ERR_CUDA;
     attrs_done = true;
   }
@@ -402,6 +536,19 @@ static bool encode_bf16(CUtensorMap* out, const void* base, uint64_t inner, uint
   return g_encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// fp32 row-major matrix [outer][inner] read as tf32 -> 2-D map with a 32-float x box_rows box, 128-byte swizzle.
+static bool encode_tf32(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer, uint32_t box_rows,
+                        bool mn_major) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {inner * 4};
+  cuuint32_t box[2] = {32, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return g_encode(out, CU_TENSOR_MAP_DATA_TYPE_TFLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // (Re)encode the tensor maps of a class and copy them to the device. The source is pageable host memory,
@@ -430,7 +577,14 @@ sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_
       ok = ok && encode_bf16(mp + MAP_CTHI, md.Cthi, rk, c.n, rk, 128);
       ok = ok && encode_bf16(mp + MAP_CTLO, md.Ctlo, rk, c.n, rk, 128);
       if (!ok) return SC_ERR_CUDA;
-      if (cudaMemcpyAsync(dev + (size_t)i * kMapsPerMat + MAP_VTHI, mp + MAP_VTHI, 6 * sizeof(CUtensorMap),
+      const int lp = p->lp;
+      ok = ok && encode_tf32(mp + MAP_M_K, md.Manc, c.n, c.m, 128, false);
+      ok = ok && encode_tf32(mp + MAP_M_MN, md.Manc, c.n, c.m, kPassK, true);
+      ok = ok && encode_tf32(mp + MAP_Y, md.Y, lp, c.m, kPassK, true);
+      ok = ok && encode_tf32(mp + MAP_Z, md.Z, lp, c.n, kPassK, true);
+      ok = ok && encode_tf32(mp + MAP_OMEGA, md.omega, lp, c.n, kPassK, true);
+      if (!ok) return SC_ERR_CUDA;
+      if (cudaMemcpyAsync(dev + (size_t)i * kMapsPerMat + MAP_VTHI, mp + MAP_VTHI, 11 * sizeof(CUtensorMap),
                           cudaMemcpyHostToDevice, p->stream) != cudaSuccess)
         return SC_ERR_CUDA;
     }
@@ -455,6 +609,29 @@ sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count
   dim3 grid((m + 127) / 128, c.ksplit, count);
   project_kernel<<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), m, n, rp,
                                                  cps, stages, cols, p->status_dev);
+  ++g_kernel_launches;
+  return cuda_ok(cudaGetLastError());
+}
+
+// One sweep over the anchor momentum. which: 0 = Y <- M Omega, 1 = Z <- M^T Y, 2 = Y <- M Z.
+sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, int which) {
+  const int lp = p->lp, m = (int)c.m, n = (int)c.n;
+  const int stage_bytes = kTileBytes + (lp / 32) * kAtomBytes;
+  int stages = (200 * 1024) / stage_bytes;
+  stages = stages > 8 ? 8 : (stages < 2 ? 2 : stages);
+  const size_t smem = (size_t)stages * stage_bytes + 1024 + 256;
+  uint32_t cols = 32;
+  while ((int)cols < lp) cols <<= 1;
+  const CUtensorMap* maps = static_cast<const CUtensorMap*>(c.tmaps);
+  if (which == 1) {
+    dim3 grid((n + 127) / 128, 1, count);
+    pass_kernel<true><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, MAP_Y, (int)offsetof(MatDev, Z), n, m, lp,
+                                                       stages, cols, p->status_dev);
+  } else {
+    dim3 grid((m + 127) / 128, 1, count);
+    pass_kernel<false><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, which == 0 ? MAP_OMEGA : MAP_Z,
+                                                        (int)offsetof(MatDev, Y), m, n, lp, stages, cols, p->status_dev);
+  }
   ++g_kernel_launches;
   return cuda_ok(cudaGetLastError());
 }
