@@ -459,12 +459,14 @@ sc_status sc_correct_and_step(sc_plan* p, const void* const* masked_grads, void*
   bool g_changed = false;
   for (int i = 0; i < p->n_mats; ++i) {
     MatDev& md = p->host_tab[i];
-    g_changed = g_changed || md.G != masked_grads[i];
+    const MatDev before = md;
     md.G = masked_grads[i];
     md.W = static_cast<float*>(params[i]);
     md.m1 = static_cast<float*>(state->exp_avg[i]);
     md.m2 = static_cast<float*>(state->exp_avg_sq[i]);
     md.Wb = state->params_bf16 ? static_cast<bf16*>(state->params_bf16[i]) : nullptr;
+    g_changed = g_changed || before.G != md.G || before.W != md.W || before.m1 != md.m1 || before.m2 != md.m2 ||
+                before.Wb != md.Wb;
     md.gproj_dbg = static_cast<float*>(p->dbg_out[i]);
   }
   if ((st = upload_table(p)) != SC_OK) return st;

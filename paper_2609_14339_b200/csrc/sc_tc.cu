@@ -9,6 +9,7 @@
 // Every wait on an mbarrier is bounded; when a wait runs out the kernel latches an error bit, drains what
 // it has in flight, frees its TMEM and returns.
 #include <cuda.h>
+#include <stdlib.h>
 
 #include "sc_internal.cuh"
 
@@ -88,6 +89,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
       : "r"(taddr));
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const void* map, const void* src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(smem_u32(src)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // K-major operand tile, rows of 128 bytes, 128-byte swizzle: 8-row groups are 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc_k128(uint32_t saddr) {
@@ -99,11 +115,18 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16(int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-constexpr int kMapsPerMat = 12;
-enum { MAP_G = 0, MAP_VTHI, MAP_VTLO, MAP_UHI, MAP_ULO, MAP_CTHI, MAP_CTLO,
+constexpr int kMapsPerMat = 20;
+constexpr int kPerCallMaps = 6;   // the first six are rebuilt whenever the caller's buffers move
+enum { MAP_G = 0,    // masked gradient, bf16, box 64 x 128 (MMA A operand of the projection)
+       MAP_G32,      // masked gradient, bf16, box 32 x 128, 64-byte swizzle (streaming tile of the fused update)
+       MAP_W, MAP_M1, MAP_M2,   // fp32 weights and AdamW moments, box 32 x 128, 128-byte swizzle (load and store)
+       MAP_WB,       // bf16 weight copy, box 32 x 128, 64-byte swizzle (store only)
+       MAP_VTHI, MAP_VTLO, MAP_UHI, MAP_ULO, MAP_CTHI, MAP_CTLO,
+       MAP_CT64HI, MAP_CT64LO,   // C^T with a 64 x 64 box (N = 64 tiles of the streaming update)
        MAP_M_K,      // anchor momentum as a K-major A operand: box 32 floats x 128 rows
        MAP_M_MN,     // anchor momentum as an MN-major A operand: box 32 floats x 32 rows (one swizzle atom column)
-       MAP_Y, MAP_Z, MAP_OMEGA };   // m x lp, n x lp, n x lp row-major fp32 as MN-major B operands: box 32 x 32
+       MAP_Y, MAP_Z, MAP_OMEGA,  // m x lp, n x lp, n x lp row-major fp32 as MN-major B operands: box 32 x 32
+       MAP_SPARE };
 constexpr int kTileBytes = 128 * 128;   // 128 rows x 64 bf16
 
 // =====================================================================================================
@@ -494,6 +517,261 @@ fused_update_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx,
   }
 }
 
+// =====================================================================================================
+// Fused correction + AdamW, streaming form: no thread touches global memory for the state.
+//   Persistent blocks (one per SM) walk over work items (matrix, 128-row panel, range of 64-column tiles).
+//   warp 0   producer: TMA loads of the MMA operands (U panel, C^T tile) and of the streaming units
+//            (128 rows x 32 columns of W, m, v fp32 and G bf16) into a 3-stage ring
+//   warp 1   MMA issuer: R = (Uhi + Ulo)(Chi + Clo)^T for a 128 x 64 tile into one of two TMEM accumulators
+//   warps 2-9  consumers, one thread per (row, half unit): R from TMEM, W/m/v/G from swizzled shared memory,
+//            blend + AdamW, results written back in place; one elected thread sends the unit out with TMA stores
+//            and hands the stage back once those stores have read it.
+// =====================================================================================================
+constexpr int kUnitW = 32;                                   // columns per streaming unit
+constexpr int kTileN = 64;                                   // columns per MMA tile (2 units)
+constexpr int kUnitF32 = 128 * kUnitW * 4;                   // 16 KB: one fp32 array of a unit
+constexpr int kUnitBf16 = 128 * kUnitW * 2;                  // 8 KB
+constexpr int kStreamStageBytes = 3 * kUnitF32 + kUnitBf16;  // 56 KB
+constexpr int kStreamStages = 3;
+constexpr int kOpndU = 2 * kTileBytes;                       // U hi + lo, 128 rows x 64 bf16 each
+constexpr int kOpndC = 2 * (kTileN * 128);                   // C^T hi + lo, 64 rows x 64 bf16 each
+constexpr int kStreamSmem = kStreamStages * kStreamStageBytes + kOpndU + kOpndC;
+
+struct StreamBars {
+  uint64_t full[kStreamStages], empty[kStreamStages];
+  uint64_t opnd_full, opnd_empty;
+  uint64_t acc_full[2], acc_empty[2];
+  uint32_t tmem_slot;
+  int abort_flag;
+};
+
+struct StreamGeom {
+  int m, n, rp;
+  int row_tiles, col_tiles, csplit, tiles_per_chunk, n_items;
+};
+
+__device__ __forceinline__ void decode_item(const StreamGeom& g, int item, int& inst, int& rt, int& ct0, int& ct1) {
+  const int per_inst = g.row_tiles * g.csplit;
+  inst = item / per_inst;
+  const int rem = item - inst * per_inst;
+  rt = rem / g.csplit;
+  const int ch = rem - rt * g.csplit;
+  ct0 = ch * g.tiles_per_chunk;
+  ct1 = min(g.col_tiles, ct0 + g.tiles_per_chunk);
+}
+
+__global__ void __launch_bounds__(320, 1)
+fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx,
+                           const CUtensorMap* __restrict__ maps, StreamGeom g, StepScalars sc,
+                           const float* __restrict__ clip_ptr, unsigned* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* opnd = smem + kStreamStages * kStreamStageBytes;
+  StreamBars* bars = reinterpret_cast<StreamBars*>(smem + kStreamSmem);
+  volatile int* abort_flag = &bars->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nch = (g.rp + 63) >> 6;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStreamStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+    mbar_init(&bars->opnd_full, 1);
+    mbar_init(&bars->opnd_empty, 1);
+    for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 8); }
+    bars->abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) tmem_alloc(&bars->tmem_slot, 2 * kTileN);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------------------------------------------ producer
+      uint32_t unit_it = 0, op_it = 0;
+      int last_inst = -1, last_panel = -1;
+      bool dead = false;
+      for (int item = blockIdx.x; item < g.n_items && !dead; item += gridDim.x) {
+        int inst, rt, ct0, ct1;
+        decode_item(g, item, inst, rt, ct0, ct1);
+        const MatDev& md = tab[idx[inst]];
+        const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
+        if (inst != last_inst) {
+          tensormap_acquire(mp + MAP_UHI); tensormap_acquire(mp + MAP_ULO);
+          tensormap_acquire(mp + MAP_CT64HI); tensormap_acquire(mp + MAP_CT64LO);
+          tensormap_acquire(mp + MAP_W); tensormap_acquire(mp + MAP_M1); tensormap_acquire(mp + MAP_M2);
+          tensormap_acquire(mp + MAP_G32);
+          last_inst = inst;
+          last_panel = -1;
+        }
+        const int row0 = rt * 128;
+        for (int ct = ct0; ct < ct1 && !dead; ++ct) {
+          for (int kc = 0; kc < nch; ++kc, ++op_it) {
+            if (!mbar_wait(&bars->opnd_empty, (op_it & 1) ^ 1, abort_flag)) { dead = true; break; }
+            const bool load_u = nch > 1 || last_panel != rt;
+            mbar_expect_tx(&bars->opnd_full, kOpndC + (load_u ? kOpndU : 0));
+            if (load_u) {
+              tma_load_2d(opnd, mp + MAP_UHI, &bars->opnd_full, kc * 64, row0);
+              tma_load_2d(opnd + kTileBytes, mp + MAP_ULO, &bars->opnd_full, kc * 64, row0);
+            }
+            tma_load_2d(opnd + kOpndU, mp + MAP_CT64HI, &bars->opnd_full, kc * 64, ct * kTileN);
+            tma_load_2d(opnd + kOpndU + kTileN * 128, mp + MAP_CT64LO, &bars->opnd_full, kc * 64, ct * kTileN);
+          }
+          if (dead) break;
+          last_panel = rt;
+          const int units = (g.n - ct * kTileN > kUnitW) ? 2 : 1;
+          for (int u = 0; u < units; ++u, ++unit_it) {
+            const int s = unit_it % kStreamStages;
+            if (!mbar_wait(&bars->empty[s], ((unit_it / kStreamStages) & 1) ^ 1, abort_flag)) { dead = true; break; }
+            uint8_t* st = smem + (size_t)s * kStreamStageBytes;
+            const int x = ct * kTileN + u * kUnitW;
+            mbar_expect_tx(&bars->full[s], kStreamStageBytes);
+            tma_load_2d(st, mp + MAP_W, &bars->full[s], x, row0);
+            tma_load_2d(st + kUnitF32, mp + MAP_M1, &bars->full[s], x, row0);
+            tma_load_2d(st + 2 * kUnitF32, mp + MAP_M2, &bars->full[s], x, row0);
+            tma_load_2d(st + 3 * kUnitF32, mp + MAP_G32, &bars->full[s], x, row0);
+          }
+        }
+      }
+      if (dead) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ------------------------------------------------------------------ MMA issuer
+      const uint32_t idesc = umma_idesc_bf16(kTileN);
+      const uint32_t uh = smem_u32(opnd), ul = uh + kTileBytes, ch = uh + kOpndU, cl = ch + kTileN * 128;
+      uint32_t op_it = 0, t = 0;
+      bool dead = false;
+      for (int item = blockIdx.x; item < g.n_items && !dead; item += gridDim.x) {
+        int inst, rt, ct0, ct1;
+        decode_item(g, item, inst, rt, ct0, ct1);
+        for (int ct = ct0; ct < ct1 && !dead; ++ct, ++t) {
+          const uint32_t ab = t & 1;
+          if (!mbar_wait(&bars->acc_empty[ab], ((t >> 1) & 1) ^ 1, abort_flag)) { dead = true; break; }
+          tc_fence_after();
+          const uint32_t d = tmem_base + ab * kTileN;
+          for (int kc = 0; kc < nch; ++kc, ++op_it) {
+            if (!mbar_wait(&bars->opnd_full, op_it & 1, abort_flag)) { dead = true; break; }
+            tc_fence_after();
+            const int ksteps = min(64, g.rp - kc * 64) >> 4;
+            for (int k = 0; k < ksteps; ++k) {
+              const uint64_t ah = umma_desc_k128(uh + k * 32), al = umma_desc_k128(ul + k * 32);
+              const uint64_t bh = umma_desc_k128(ch + k * 32), bl = umma_desc_k128(cl + k * 32);
+              umma_bf16(d, ah, bh, idesc, (kc | k) != 0);
+              umma_bf16(d, ah, bl, idesc, 1);
+              umma_bf16(d, al, bh, idesc, 1);
+            }
+            umma_commit(&bars->opnd_empty);
+          }
+          if (dead) break;
+          umma_commit(&bars->acc_full[ab]);
+        }
+      }
+      if (dead) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
+    }
+    __syncwarp();
+  } else {
+    // -------------------------------------------------------------------- consumers
+    const int q = warp & 3, h = (warp - 2) >> 2;
+    const int r = q * 32 + lane;                 // row inside the 128-row panel
+    const bool leader = warp == 2 && lane == 0;
+    const float clip = *clip_ptr;
+    uint32_t unit_it = 0, t = 0;
+    int last_inst = -1;
+    bool dead = false;
+    for (int item = blockIdx.x; item < g.n_items && !dead; item += gridDim.x) {
+      int inst, rt, ct0, ct1;
+      decode_item(g, item, inst, rt, ct0, ct1);
+      const MatDev& md = tab[idx[inst]];
+      const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
+      if (leader && inst != last_inst) {
+        tensormap_acquire(mp + MAP_W); tensormap_acquire(mp + MAP_M1); tensormap_acquire(mp + MAP_M2);
+        tensormap_acquire(mp + MAP_WB);
+      }
+      last_inst = inst;
+      const int row0 = rt * 128;
+      float* gp_dbg = md.gproj_dbg;
+      const bool has_wb = md.Wb != nullptr;
+      for (int ct = ct0; ct < ct1 && !dead; ++ct, ++t) {
+        const uint32_t ab = t & 1;
+        if (!mbar_wait(&bars->acc_full[ab], (t >> 1) & 1, abort_flag)) { dead = true; break; }
+        tc_fence_after();
+        const int units = (g.n - ct * kTileN > kUnitW) ? 2 : 1;
+        for (int u = 0; u < units; ++u, ++unit_it) {
+          const int s = unit_it % kStreamStages;
+          if (!mbar_wait(&bars->full[s], (unit_it / kStreamStages) & 1, abort_flag)) { dead = true; break; }
+          uint8_t* st = smem + (size_t)s * kStreamStageBytes;
+          float rv[16];
+          tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + ab * kTileN + u * kUnitW + h * 16, rv);
+          tmem_ld_wait();
+          float4* Ws = reinterpret_cast<float4*>(st);
+          float4* M1s = reinterpret_cast<float4*>(st + kUnitF32);
+          float4* M2s = reinterpret_cast<float4*>(st + 2 * kUnitF32);
+          uint4* Gs = reinterpret_cast<uint4*>(st + 3 * kUnitF32);
+          float gout[16];
+          uint4 wb_pk[2];
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const int gidx = r * 4 + ((2 * h + j) ^ ((r >> 1) & 3));
+            const uint4 graw = Gs[gidx];
+            const uint32_t gw[4] = {graw.x, graw.y, graw.z, graw.w};
+            uint32_t wbw[4];
+#pragma unroll
+            for (int i2 = 0; i2 < 2; ++i2) {
+              const int i = 2 * j + i2;            // 16-byte chunk of the fp32 rows
+              const int fidx = r * 8 + ((4 * h + i) ^ (r & 7));
+              float4 w = Ws[fidx], m1 = M1s[fidx], m2 = M2s[fidx], gp;
+              const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gw[2 * i2]);
+              const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&gw[2 * i2 + 1]);
+              const float g4[4] = {__low2float(g01), __high2float(g01), __low2float(g23), __high2float(g23)};
+              const float4 rr = make_float4(rv[4 * i], rv[4 * i + 1], rv[4 * i + 2], rv[4 * i + 3]);
+              adamw4(sc, clip, g4, rr, w, m1, m2, gp);
+              Ws[fidx] = w; M1s[fidx] = m1; M2s[fidx] = m2;
+              gout[4 * i] = gp.x; gout[4 * i + 1] = gp.y; gout[4 * i + 2] = gp.z; gout[4 * i + 3] = gp.w;
+              __nv_bfloat162 b01 = __floats2bfloat162_rn(w.x, w.y), b23 = __floats2bfloat162_rn(w.z, w.w);
+              wbw[2 * i2] = *reinterpret_cast<uint32_t*>(&b01);
+              wbw[2 * i2 + 1] = *reinterpret_cast<uint32_t*>(&b23);
+            }
+            wb_pk[j] = make_uint4(wbw[0], wbw[1], wbw[2], wbw[3]);
+            Gs[gidx] = wb_pk[j];
+          }
+          const int x = ct * kTileN + u * kUnitW;
+          if (gp_dbg) {   // test hook: plain stores, one row per thread
+            const int row = row0 + r, col = x + h * 16;
+            if (row < g.m)
+              for (int e = 0; e < 16; ++e)
+                if (col + e < g.n) gp_dbg[(size_t)row * g.n + col + e] = gout[e];
+          }
+          fence_proxy_async();
+          consumer_barrier();
+          if (leader) {
+            tma_store_2d(mp + MAP_W, st, x, row0);
+            tma_store_2d(mp + MAP_M1, st + kUnitF32, x, row0);
+            tma_store_2d(mp + MAP_M2, st + 2 * kUnitF32, x, row0);
+            if (has_wb) tma_store_2d(mp + MAP_WB, st + 3 * kUnitF32, x, row0);
+            tma_store_commit();
+            // hand the previous unit's stage back once its stores have finished reading shared memory
+            tma_store_wait_read<1>();
+            if (unit_it > 0) mbar_arrive(&bars->empty[(unit_it - 1) % kStreamStages]);
+          }
+        }
+        if (dead) break;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->acc_empty[ab]);
+      }
+    }
+    if (dead && lane == 0) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
+    if (leader) tma_store_wait_all();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, 2 * kTileN);
+}
+
 // ---------------------------------------------------------------------------------------------- host
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -518,6 +796,8 @@ sc_status tc_init() {
   if (!attrs_done) {
     if (cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(fused_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(fused_update_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kStreamSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
         cudaFuncSetAttribute(pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
       return SC_ERR_CUDA;
@@ -526,36 +806,35 @@ sc_status tc_init() {
   return SC_OK;
 }
 
-// bf16 row-major matrix [outer][inner] -> 2-D map with a 64 x box_rows box and the 128-byte swizzle.
+// Row-major matrix [outer][inner] -> 2-D tiled map.
+static bool encode2d(CUtensorMap* out, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t inner,
+                     uint64_t outer, uint64_t row_stride_elems, uint32_t box_inner, uint32_t box_rows,
+                     CUtensorMapSwizzle swz) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {row_stride_elems * (uint64_t)elem_bytes};
+  cuuint32_t box[2] = {box_inner, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return g_encode(out, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// bf16, 64-element (128-byte) rows, 128-byte swizzle: K-major MMA operand tiles.
 static bool encode_bf16(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer, uint64_t row_stride_elems,
                         uint32_t box_rows) {
-  cuuint64_t dims[2] = {inner, outer};
-  cuuint64_t strides[1] = {row_stride_elems * 2};
-  cuuint32_t box[2] = {64, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return g_encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode2d(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, inner, outer, row_stride_elems, 64, box_rows,
+                  CU_TENSOR_MAP_SWIZZLE_128B);
 }
-
-// fp32 row-major matrix [outer][inner] read as tf32 -> 2-D map with a 32-float x box_rows box, 128-byte swizzle.
+// fp32 read as tf32, 32-element (128-byte) rows; MN-major operands need the 32-byte-atom flavour of the swizzle.
 static bool encode_tf32(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer, uint32_t box_rows,
                         bool mn_major) {
-  cuuint64_t dims[2] = {inner, outer};
-  cuuint64_t strides[1] = {inner * 4};
-  cuuint32_t box[2] = {32, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return g_encode(out, CU_TENSOR_MAP_DATA_TYPE_TFLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode2d(out, CU_TENSOR_MAP_DATA_TYPE_TFLOAT32, 4, base, inner, outer, inner, 32, box_rows,
+                  mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 // (Re)encode the tensor maps of a class and copy them to the device. The source is pageable host memory,
-// so the runtime has taken its copy of the bytes when cudaMemcpyAsync returns.
+// so the runtime has taken its copy of the bytes when cudaMemcpy2DAsync returns.
 sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_call_part) {
   const int cnt = (int)c.mats.size();
-  const int rp = p->rp, rk = p->rk;
+  const int rp = p->rp, rk = p->rk, lp = p->lp;
   std::vector<CUtensorMap> maps((size_t)cnt * kMapsPerMat);
   CUtensorMap* dev = static_cast<CUtensorMap*>(c.tmaps);
   for (int i = 0; i < cnt; ++i) {
@@ -563,11 +842,15 @@ sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_
     CUtensorMap* mp = &maps[(size_t)i * kMapsPerMat];
     bool ok = true;
     if (per_call_part) {
+      const CUtensorMapDataType f32 = CU_TENSOR_MAP_DATA_TYPE_FLOAT32, b16 = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
       ok = ok && encode_bf16(mp + MAP_G, md.G, c.n, c.m, c.n, 128);
+      ok = ok && encode2d(mp + MAP_G32, b16, 2, md.G, c.n, c.m, c.n, 32, 128, CU_TENSOR_MAP_SWIZZLE_64B);
+      ok = ok && encode2d(mp + MAP_W, f32, 4, md.W, c.n, c.m, c.n, 32, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+      ok = ok && encode2d(mp + MAP_M1, f32, 4, md.m1, c.n, c.m, c.n, 32, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+      ok = ok && encode2d(mp + MAP_M2, f32, 4, md.m2, c.n, c.m, c.n, 32, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+      ok = ok && encode2d(mp + MAP_WB, b16, 2, md.Wb ? (const void*)md.Wb : md.G, c.n, c.m, c.n, 32, 128,
+                          CU_TENSOR_MAP_SWIZZLE_64B);
       if (!ok) return SC_ERR_CUDA;
-      if (cudaMemcpyAsync(dev + (size_t)i * kMapsPerMat + MAP_G, mp + MAP_G, sizeof(CUtensorMap), cudaMemcpyHostToDevice,
-                          p->stream) != cudaSuccess)
-        return SC_ERR_CUDA;
     }
     if (static_part) {
       ok = ok && encode_bf16(mp + MAP_VTHI, md.Vthi, c.n, rp, c.n, rp);
@@ -576,19 +859,26 @@ sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_
       ok = ok && encode_bf16(mp + MAP_ULO, md.Ulo, rk, c.m, rk, 128);
       ok = ok && encode_bf16(mp + MAP_CTHI, md.Cthi, rk, c.n, rk, 128);
       ok = ok && encode_bf16(mp + MAP_CTLO, md.Ctlo, rk, c.n, rk, 128);
-      if (!ok) return SC_ERR_CUDA;
-      const int lp = p->lp;
+      ok = ok && encode_bf16(mp + MAP_CT64HI, md.Cthi, rk, c.n, rk, kTileN);
+      ok = ok && encode_bf16(mp + MAP_CT64LO, md.Ctlo, rk, c.n, rk, kTileN);
       ok = ok && encode_tf32(mp + MAP_M_K, md.Manc, c.n, c.m, 128, false);
       ok = ok && encode_tf32(mp + MAP_M_MN, md.Manc, c.n, c.m, kPassK, true);
       ok = ok && encode_tf32(mp + MAP_Y, md.Y, lp, c.m, kPassK, true);
       ok = ok && encode_tf32(mp + MAP_Z, md.Z, lp, c.n, kPassK, true);
       ok = ok && encode_tf32(mp + MAP_OMEGA, md.omega, lp, c.n, kPassK, true);
       if (!ok) return SC_ERR_CUDA;
-      if (cudaMemcpyAsync(dev + (size_t)i * kMapsPerMat + MAP_VTHI, mp + MAP_VTHI, 11 * sizeof(CUtensorMap),
-                          cudaMemcpyHostToDevice, p->stream) != cudaSuccess)
-        return SC_ERR_CUDA;
     }
   }
+  const size_t pitch = kMapsPerMat * sizeof(CUtensorMap);
+  if (per_call_part &&
+      cudaMemcpy2DAsync(dev, pitch, maps.data(), pitch, kPerCallMaps * sizeof(CUtensorMap), cnt, cudaMemcpyHostToDevice,
+                        p->stream) != cudaSuccess)
+    return SC_ERR_CUDA;
+  if (static_part &&
+      cudaMemcpy2DAsync(dev + kPerCallMaps, pitch, maps.data() + kPerCallMaps, pitch,
+                        (kMapsPerMat - kPerCallMaps) * sizeof(CUtensorMap), cnt, cudaMemcpyHostToDevice,
+                        p->stream) != cudaSuccess)
+    return SC_ERR_CUDA;
   return SC_OK;
 }
 
@@ -638,10 +928,34 @@ sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, i
 
 sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc) {
   const int m = (int)c.m, n = (int)c.n;
-  dim3 grid((n + 127) / 128, (m + 127) / 128, count);
-  const size_t smem = 4 * kTileBytes + 1024 + 64;
-  fused_update_kernel<<<grid, 256, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), m, n,
-                                                      p->rp, sc, p->clip_dev, p->status_dev);
+  static const bool use_tiled = getenv("SC_FUSED_TILED") != nullptr;   // the older one-tile-per-block kernel
+  if (use_tiled) {
+    dim3 grid((n + 127) / 128, (m + 127) / 128, count);
+    const size_t smem = 4 * kTileBytes + 1024 + 64;
+    fused_update_kernel<<<grid, 256, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), m, n,
+                                                        p->rp, sc, p->clip_dev, p->status_dev);
+    ++g_kernel_launches;
+    return cuda_ok(cudaGetLastError());
+  }
+  static int n_sm = 0;
+  if (!n_sm) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) n_sm = 148;
+  }
+  StreamGeom g;
+  g.m = m; g.n = n; g.rp = p->rp;
+  g.row_tiles = (m + 127) / 128;
+  g.col_tiles = (n + kTileN - 1) / kTileN;
+  int csplit = 1;
+  while ((long long)count * g.row_tiles * csplit < 4LL * n_sm && g.col_tiles / (csplit * 2) >= 4) csplit *= 2;
+  g.tiles_per_chunk = (g.col_tiles + csplit - 1) / csplit;
+  g.csplit = (g.col_tiles + g.tiles_per_chunk - 1) / g.tiles_per_chunk;
+  g.n_items = count * g.row_tiles * g.csplit;
+  const int grid = g.n_items < n_sm ? g.n_items : n_sm;
+  const size_t smem = kStreamSmem + sizeof(StreamBars) + 1024;
+  fused_update_stream_kernel<<<grid, 320, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps),
+                                                             g, sc, p->clip_dev, p->status_dev);
   ++g_kernel_launches;
   return cuda_ok(cudaGetLastError());
 }
