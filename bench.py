@@ -171,6 +171,46 @@ def build_workload(name, device, torch):
     return cfg, shapes, dict(G=G, Ga=Ga, W=W, M1=M1, M2=M2, Wb=Wb)
 
 
+def run_e2e(args, torch, plan, buf, shapes, n_elems, gsize, world, device):
+    """The same metric through sc_correct_and_step_host: every step's masked gradients start in pinned HOST memory
+    (as they would after the data-parallel reduction over the network), are copied to the device inside the
+    timed region, and the step's statistics are read back to the host. Anchor gradients also start on the host."""
+    gdt = buf["G"][0].dtype
+    total = sum(m * n for m, n in shapes)
+    try:
+        host_g = torch.empty(total, dtype=gdt, pin_memory=True)
+        host_a = torch.empty(total, dtype=gdt, pin_memory=True)
+    except RuntimeError as e:      # not enough lockable host memory on this box
+        return {"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0, "skipped": str(e)[:120]}
+    hg, ha, off = [], [], 0
+    for (m, n), g, a in zip(shapes, buf["G"], buf["Ga"]):
+        hg.append(host_g[off:off + m * n].view(m, n)); ha.append(host_a[off:off + m * n].view(m, n))
+        hg[-1].copy_(g); ha[-1].copy_(a)
+        off += m * n
+    torch.cuda.synchronize()
+    steps = max(REFRESH_EVERY, min(args.steps, 2 * REFRESH_EVERY))
+    base = 10_000
+
+    def one(i):
+        if i % REFRESH_EVERY == 0:
+            for d, h in zip(buf["Ga"], ha):
+                d.copy_(h, non_blocking=True)
+            plan.anchor_update(buf["Ga"], base + i)
+        plan.correct_and_step_host(hg, buf["G"], buf["W"], buf["M1"], buf["M2"], 100 + base + i, params_bf16=buf["Wb"])
+
+    one(0); one(1)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(steps):
+        one(REFRESH_EVERY + i)
+    torch.cuda.synchronize()
+    ms = (time.perf_counter() - t0) * 1e3 / steps
+    return {"value": world * n_elems * gsize / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": int(total * gsize * (1 + 1.0 / REFRESH_EVERY)),
+            "d2h_bytes_per_step": int(len(shapes) * 16 + 4),
+            "note": "gradients (and, every %d-th step, anchor gradients) start in pinned host memory" % REFRESH_EVERY}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -278,7 +318,12 @@ def run_ours(args):
         desc = desc.replace(" of 0)", " of %d)" % n_elems)
         line["cpu_baseline"] = {"value": elems * gsize / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
                                 "sample": desc}
-    line["e2e"] = None
+    line["e2e"] = None if args.no_e2e else run_e2e(args, torch, plan, buf, shapes, n_elems, gsize, world, device)
+    if world > 1 and line["e2e"] is not None:
+        t = torch.tensor([line["e2e"]["ms_per_step"]], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        line["e2e"]["ms_per_step"] = float(t.item())
+        line["e2e"]["value"] = world * n_elems * gsize / (float(t.item()) * 1e-3) / 1e9
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:

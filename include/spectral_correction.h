@@ -149,6 +149,19 @@ SC_API sc_status sc_anchor_update(sc_plan* plan, const void* const* anchor_grads
 SC_API sc_status sc_correct_and_step(sc_plan* plan, const void* const* masked_grads, void* const* params,
                                      const sc_opt_state* state, int64_t step);
 
+/* sc_correct_and_step_host - the same step for gradients that arrive in HOST memory (in the paper's setting the
+ * data-parallel all-reduce of Algorithm 1 line 6 delivers them over the network).
+ *   host_grads     host array of n_mats HOST pointers (grad_dtype, rows x cols). Page-locked memory lets the copies
+ *                  overlap the kernels; pageable memory works but serialises.
+ *   grad_staging   host array of n_mats DEVICE pointers the gradients are copied into (caller-owned, same sizes)
+ *   stats_out      host: n_mats entries filled with the step's statistics (the step's result read back), or NULL
+ *   clip_out       host: the clip factor applied, or NULL
+ * The copies of one shape class are queued ahead of the kernels of the class before it, on a stream the plan owns.
+ * Unlike sc_correct_and_step this call returns only after the step has finished on the device. */
+SC_API sc_status sc_correct_and_step_host(sc_plan* plan, const void* const* host_grads, void* const* grad_staging,
+                                          void* const* params, const sc_opt_state* state, int64_t step,
+                                          sc_mat_stats* stats_out, float* clip_out);
+
 /* ---- inspection / test hooks ------------------------------------------------------------------------- */
 
 /* Copy matrix `mat`'s cached basis into caller device buffers (any may be NULL):

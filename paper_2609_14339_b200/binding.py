@@ -73,6 +73,8 @@ EXPORTS = {
     "sc_plan_destroy": (C.c_int, [_VP]),
     "sc_anchor_update": (C.c_int, [_VP, _VPP, C.c_int64]),
     "sc_correct_and_step": (C.c_int, [_VP, _VPP, _VPP, C.POINTER(OptState), C.c_int64]),
+    "sc_correct_and_step_host": (C.c_int, [_VP, _VPP, _VPP, _VPP, C.POINTER(OptState), C.c_int64, C.POINTER(MatStats),
+                                           C.POINTER(C.c_float)]),
     "sc_export_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
     "sc_import_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
     "sc_export_projection": (C.c_int, [_VP, C.c_int, _VP, _VP]),
@@ -221,6 +223,28 @@ class Plan:
         return _check(self.lib.sc_correct_and_step(self.handle, _ptr_array(masked_grads, n, False),
                                                    _ptr_array(params, n, False), C.byref(st), int(step)),
                       "sc_correct_and_step", allow=(SC_OK, SC_WARN_NO_ANCHOR))
+
+    def correct_and_step_host(self, host_grads, grad_staging, params, exp_avg, exp_avg_sq, step: int, params_bf16=None,
+                              want_stats: bool = True):
+        """Gradients in host tensors (pin them for overlap); returns (status, stats or None, clip)."""
+        n = self.n_mats
+        harr = (C.c_void_p * n)()
+        for i, t in enumerate(host_grads):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("host gradient %d must be a contiguous CPU tensor" % i)
+            harr[i] = t.data_ptr()
+        st = OptState(_ptr_array(exp_avg, n, False), _ptr_array(exp_avg_sq, n, False),
+                      _ptr_array(params_bf16, n, True) if params_bf16 is not None else None)
+        stats = (MatStats * n)() if want_stats else None
+        clip = C.c_float(1.0)
+        rc = _check(self.lib.sc_correct_and_step_host(self.handle, harr, _ptr_array(grad_staging, n, False),
+                                                      _ptr_array(params, n, False), C.byref(st), int(step), stats,
+                                                      C.byref(clip)),
+                    "sc_correct_and_step_host", allow=(SC_OK, SC_WARN_NO_ANCHOR))
+        out = None
+        if stats is not None:
+            out = [dict(g_sqnorm=a.g_sqnorm, x_sqnorm=a.x_sqnorm, gproj_sqnorm=a.gproj_sqnorm, r_eff=a.r_eff) for a in stats]
+        return rc, out, clip.value
 
     # ---- inspection --------------------------------------------------------------------------------
     def export_basis(self, mat: int):

@@ -127,6 +127,10 @@ struct sc_plan {
   std::vector<void*> dbg_out;
   bool table_dirty = true;
   bool tensor_any = false;
+  // host-gradient path: copies run on their own stream, one event per shape class
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t copy_gate = nullptr;
+  std::vector<cudaEvent_t> copy_done;
   // optional per-category device timing (cudaEvent pairs around groups of launches)
   bool prof_on = false;
   std::vector<cudaEvent_t> prof_events;

@@ -350,6 +350,11 @@ sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int 
                            cudaHostAllocDefault) == cudaSuccess;
   for (int i = 0; ok && i < kStagingSlots; ++i)
     ok = cudaEventCreateWithFlags(&p->staging_ev[i], cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&p->copy_gate, cudaEventDisableTiming) == cudaSuccess;
+  p->copy_done.resize(p->classes.size(), nullptr);
+  for (size_t k = 0; ok && k < p->classes.size(); ++k)
+    ok = cudaEventCreateWithFlags(&p->copy_done[k], cudaEventDisableTiming) == cudaSuccess;
   if (!ok) { sc_plan_destroy(p); return SC_ERR_CUDA; }
   const float one = 1.f;
   ok = cudaMemcpyAsync(p->clip_dev, &one, sizeof(float), cudaMemcpyHostToDevice, s) == cudaSuccess;
@@ -375,6 +380,10 @@ sc_status sc_plan_destroy(sc_plan* p) {
   for (int i = 0; i < kStagingSlots; ++i)
     if (p->staging_ev[i]) cudaEventDestroy(p->staging_ev[i]);
   for (cudaEvent_t e : p->prof_events) cudaEventDestroy(e);
+  for (cudaEvent_t e : p->copy_done)
+    if (e) cudaEventDestroy(e);
+  if (p->copy_gate) cudaEventDestroy(p->copy_gate);
+  if (p->copy_stream) { cudaStreamSynchronize(p->copy_stream); cudaStreamDestroy(p->copy_stream); }
   if (p->staging) cudaFreeHost(p->staging);
   delete p;
   return SC_OK;
@@ -441,8 +450,10 @@ sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t 
   return cuda_ok(cudaGetLastError());
 }
 
-sc_status sc_correct_and_step(sc_plan* p, const void* const* masked_grads, void* const* params,
-                              const sc_opt_state* state, int64_t step) {
+// One optimizer step. With host_grads != nullptr the masked gradients are first copied from host memory into
+// masked_grads (device staging) on the plan's copy stream, one shape class ahead of the kernels that read them.
+static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* const* params,
+                           const sc_opt_state* state, int64_t step, const void* const* host_grads) {
   if (!p || !state || step < 1) return SC_ERR_INVALID_ARG;
   sc_status st;
   if ((st = check_ptr_array(masked_grads, p->n_mats, false)) != SC_OK) return st;
@@ -486,9 +497,25 @@ sc_status sc_correct_and_step(sc_plan* p, const void* const* masked_grads, void*
   const bool clip_on = hp.max_grad_norm > 0.f;
   const bool want_norm = clip_on || hp.collect_stats;
 
+  if (host_grads) {
+    // queue every host-to-device copy now, class by class; the kernels of a class wait only for its own event
+    const size_t esz = g_bf16 ? 2 : 4;
+    if (cudaEventRecord(p->copy_gate, s) != cudaSuccess || cudaStreamWaitEvent(p->copy_stream, p->copy_gate, 0) != cudaSuccess)
+      return SC_ERR_CUDA;   // earlier work on the plan's stream may still be reading the staging buffers
+    for (size_t k = 0; k < p->classes.size(); ++k) {
+      for (int id : p->classes[k].mats) {
+        const size_t bytes = (size_t)p->shapes[id].rows * p->shapes[id].cols * esz;
+        if (cudaMemcpyAsync(const_cast<void*>(masked_grads[id]), host_grads[id], bytes, cudaMemcpyHostToDevice,
+                            p->copy_stream) != cudaSuccess)
+          return SC_ERR_CUDA;
+      }
+      if (cudaEventRecord(p->copy_done[k], p->copy_stream) != cudaSuccess) return SC_ERR_CUDA;
+    }
+  }
   auto project = [&](ShapeClass& c) -> sc_status {
     const int cnt = (int)c.mats.size(), m = (int)c.m, n = (int)c.n;
     const int* idx = c.idx_all;
+    if (host_grads && cudaStreamWaitEvent(s, p->copy_done[&c - p->classes.data()], 0) != cudaSuccess) return SC_ERR_CUDA;
     if (rp > 0) {
       ProfScope ps(p, PROF_PROJECT);
       if (c.tensor) {
@@ -531,6 +558,28 @@ sc_status sc_correct_and_step(sc_plan* p, const void* const* masked_grads, void*
   bool any = false;
   for (char h : p->has_basis) any = any || h;
   return (p->rank > 0 && !any) ? SC_WARN_NO_ANCHOR : SC_OK;
+}
+
+sc_status sc_correct_and_step(sc_plan* p, const void* const* masked_grads, void* const* params,
+                              const sc_opt_state* state, int64_t step) {
+  return step_impl(p, masked_grads, params, state, step, nullptr);
+}
+
+sc_status sc_correct_and_step_host(sc_plan* p, const void* const* host_grads, void* const* grad_staging,
+                                   void* const* params, const sc_opt_state* state, int64_t step,
+                                   sc_mat_stats* stats_out, float* clip_out) {
+  if (!p || !host_grads || !grad_staging) return SC_ERR_INVALID_ARG;
+  for (int i = 0; i < p->n_mats; ++i)
+    if (!host_grads[i]) return SC_ERR_INVALID_ARG;
+  sc_status st = step_impl(p, reinterpret_cast<const void* const*>(grad_staging), params, state, step, host_grads);
+  if (st != SC_OK && st != SC_WARN_NO_ANCHOR) return st;
+  if (stats_out) {
+    const sc_status s2 = sc_get_stats(p, stats_out, clip_out);   // device-to-host read; waits for the step
+    if (s2 != SC_OK) return s2;
+  } else if (cudaStreamSynchronize(p->stream) != cudaSuccess) {
+    return SC_ERR_CUDA;
+  }
+  return st;
 }
 
 // -------------------------------------------------------------------------------------- inspection

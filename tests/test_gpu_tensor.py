@@ -79,3 +79,31 @@ def test_engines_agree(torch):
     b = GpuRun(case2, inp, torch)
     assert a.uses_tc and not b.uses_tc
     assert rel(a.gproj[0], b.gproj[0]) < 1e-4 and rel(a.m[0], b.m[0]) < 1e-4 and rel(a.W[0], b.W[0]) < 1e-5
+
+
+def test_host_gradient_entry_point_matches_device_path(torch):
+    """sc_correct_and_step_host copies pinned host gradients class by class and must give the device path's bits."""
+    from parity_util import make_plan, to_dev
+    case = Case(shapes=[(256, 384), (384, 256), (256, 384)], rank=16, tokens=256, keep=0.25, planted=8, seed=7, tau_p=50.0)
+    inp = make_inputs(case)
+    outs = []
+    for host in (False, True):
+        plan = make_plan(case, torch)
+        n = len(case.shapes)
+        plan.anchor_update([to_dev(inp["anchors"][i][0], "bf16", torch, "cuda:0") for i in range(n)], 0)
+        G = [to_dev(inp["G"][i], "bf16", torch, "cuda:0") for i in range(n)]
+        W = [torch.from_numpy(inp["W"][i].copy()).cuda() for i in range(n)]
+        m = [torch.from_numpy(inp["m"][i].copy()).cuda() for i in range(n)]
+        v = [torch.from_numpy(inp["v"][i].copy()).cuda() for i in range(n)]
+        if host:
+            Gh = [g.cpu().pin_memory() for g in G]
+            stage = [torch.zeros_like(g) for g in G]
+            rc, stats, clip = plan.correct_and_step_host(Gh, stage, W, m, v, 100)
+            assert rc == 0 and len(stats) == n and stats[0]["g_sqnorm"] > 0 and clip == 1.0
+            assert all(torch.equal(a, b) for a, b in zip(stage, G))
+        else:
+            assert plan.correct_and_step(G, W, m, v, 100) == 0
+        torch.cuda.synchronize()
+        outs.append((W, m, v))
+    for a, b in zip(outs[0], outs[1]):
+        assert all(torch.equal(x, y) for x, y in zip(a, b))
