@@ -216,6 +216,7 @@ def run_ours(args):
     import torch.distributed as dist
     import paper_2609_14339_b200 as sc
     from paper_2609_14339_b200 import build as _build
+    from paper_2609_14339_b200 import multi
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -270,12 +271,9 @@ def run_ours(args):
     ms_total = e0.elapsed_time(e1)
     launches = lib.sc_kernel_launch_count() - launches0
     clocks = sampler.stop() if sampler else None
-    if world > 1:
-        t = torch.tensor([ms_total], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = multi.max_over_ranks(ms_total, device)
     ms_step = ms_total / args.steps
-    value = world * n_elems * gsize / (ms_step * 1e-3) / 1e9
+    value = multi.whole_job_throughput(n_elems * gsize, world, ms_step) / 1e9
 
     # ---- per-phase device times (separate pass, profiling events on) -------------------------------
     plan.set_profiling(True)
@@ -319,11 +317,9 @@ def run_ours(args):
         line["cpu_baseline"] = {"value": elems * gsize / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
                                 "sample": desc}
     line["e2e"] = None if args.no_e2e else run_e2e(args, torch, plan, buf, shapes, n_elems, gsize, world, device)
-    if world > 1 and line["e2e"] is not None:
-        t = torch.tensor([line["e2e"]["ms_per_step"]], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        line["e2e"]["ms_per_step"] = float(t.item())
-        line["e2e"]["value"] = world * n_elems * gsize / (float(t.item()) * 1e-3) / 1e9
+    if world > 1 and line["e2e"] is not None and line["e2e"].get("value") is not None:
+        line["e2e"]["ms_per_step"] = multi.max_over_ranks(line["e2e"]["ms_per_step"], device)
+        line["e2e"]["value"] = multi.whole_job_throughput(n_elems * gsize, world, line["e2e"]["ms_per_step"]) / 1e9
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
