@@ -47,7 +47,7 @@ struct MatDev {
   float* xpart;  // kAtbMaxSplits x rp x rp   row-slice partials of X
   float* sqpart; // kSqnormBlocks partial sums of ||G||^2
   float* stats;  // kStatsFloats
-  // anchor-update scratch (slot)
+  // anchor-update scratch
   float* Y;      // m x lp
   float* Y2;     // m x lp
   float* Z;      // n x lp
@@ -113,6 +113,7 @@ struct sc_plan {
   std::vector<sc::MatDev> host_tab;   // host mirror of the device table
   std::vector<sc::MatDev> last_uploaded;
   sc::MatDev* dev_tab = nullptr;
+  int* idx_glob = nullptr;            // device: flat list of the matrices an anchor call touches
   char* staging = nullptr;            // pinned, kStagingSlots * staging_bytes
   size_t staging_bytes = 0;
   cudaEvent_t staging_ev[sc::kStagingSlots]{};
@@ -186,6 +187,6 @@ sc_status tc_init();   // resolves the driver entry point for tensor-map encodin
 sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_call_part);
 sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count);   // T = G V
 sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc);
-sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, int which);
+sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, bool transposed, int b_field_off);
 
 }  // namespace sc

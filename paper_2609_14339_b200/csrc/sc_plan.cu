@@ -136,31 +136,26 @@ size_t layout(sc_plan* p, bool assign) {
     md.inst = p->inst_of[i];
     if (assign) p->host_tab[i] = md;
   }
-  // anchor-update scratch: one region, reused by the classes in turn (slot = instance index)
-  cv.off = align_up(cv.off);
-  const size_t slot_base = cv.off;
-  size_t slot_max = 0;
-  for (auto& c : p->classes) {
-    Carver sv(assign ? p->ws + slot_base : nullptr);
-    for (size_t k = 0; k < c.mats.size(); ++k) {
-      const size_t m = (size_t)c.m, n = (size_t)c.n;
-      float* Y = sv.take<float>(m * lp); float* Y2 = sv.take<float>(m * lp);
-      float* Z = sv.take<float>(n * lp); float* Z2 = sv.take<float>(n * lp);
-      float* gram = sv.take<float>((size_t)lp * lp); float* rmat = sv.take<float>((size_t)lp * lp);
-      float* gpart = sv.take<float>((size_t)atb_splits((int)std::max(m, n)) * lp * lp);
-      float* rmat2 = sv.take<float>((size_t)lp * lp); float* rinv = sv.take<float>((size_t)lp * lp);
-      float* racc = sv.take<float>((size_t)lp * lp); float* jk = sv.take<float>((size_t)lp * lp);
-      float* jv = sv.take<float>((size_t)lp * lp);
-      float* ub = sv.take<float>((size_t)lp * rp); float* wb = sv.take<float>((size_t)lp * rp);
-      if (assign) {
-        MatDev& md = p->host_tab[c.mats[k]];
-        md.Y = Y; md.Y2 = Y2; md.Z = Z; md.Z2 = Z2; md.gram = gram; md.gpart = gpart; md.rmat = rmat; md.rmat2 = rmat2;
-        md.rinv = rinv; md.racc = racc; md.jk = jk; md.jv = jv; md.ub = ub; md.wb = wb;
-      }
+  // anchor-update scratch, per matrix: the basis build runs phase by phase over all shape classes, so every
+  // matrix needs its own Y / Z panels and l x l factors at the same time
+  for (int i = 0; i < n_mats; ++i) {
+    const size_t m = (size_t)p->shapes[i].rows, n = (size_t)p->shapes[i].cols;
+    float* Y = cv.take<float>(m * lp); float* Y2 = cv.take<float>(m * lp);
+    float* Z = cv.take<float>(n * lp); float* Z2 = cv.take<float>(n * lp);
+    float* gram = cv.take<float>((size_t)lp * lp); float* rmat = cv.take<float>((size_t)lp * lp);
+    float* gpart = cv.take<float>((size_t)atb_splits((int)std::max(m, n)) * lp * lp);
+    float* rmat2 = cv.take<float>((size_t)lp * lp); float* rinv = cv.take<float>((size_t)lp * lp);
+    float* racc = cv.take<float>((size_t)lp * lp); float* jk = cv.take<float>((size_t)lp * lp);
+    float* jv = cv.take<float>((size_t)lp * lp);
+    float* ub = cv.take<float>((size_t)lp * rp); float* wb = cv.take<float>((size_t)lp * rp);
+    if (assign) {
+      MatDev& md = p->host_tab[i];
+      md.Y = Y; md.Y2 = Y2; md.Z = Z; md.Z2 = Z2; md.gram = gram; md.gpart = gpart; md.rmat = rmat; md.rmat2 = rmat2;
+      md.rinv = rinv; md.racc = racc; md.jk = jk; md.jv = jv; md.ub = ub; md.wb = wb;
     }
-    slot_max = std::max(slot_max, align_up(sv.off));
   }
-  cv.off = slot_base + slot_max;
+  int* glob = cv.take<int>(n_mats);
+  if (assign) p->idx_glob = glob;
   return align_up(cv.off);
 }
 
@@ -222,19 +217,35 @@ struct ProfScope {
   }
 };
 
-// Q <- orth(Y) by two rounds of Cholesky QR; Y (rows x lp) is overwritten, tmp is scratch of the same size.
-// keepR: leave the two factors in rmat / rmat2 (and their product in racc) for the caller.
-void cholqr2(sc_plan* p, const int* idx, int cnt, int offY, int offTmp, int rows, bool keepR) {
+// One class's share of an anchor arrival: the matrices that received a gradient.
+struct ActiveClass {
+  ShapeClass* c;
+  const int* idx;
+  int cnt;
+};
+
+// Q <- orth(Y) by Cholesky QR over all active classes; Y (rows x lp) is overwritten, tmp is scratch of the same
+// size. rounds = 2 (Cholesky QR twice) gives a basis orthonormal to working precision; rounds = 1 is enough for
+// an intermediate basis of the subspace iteration, whose only job is to keep the next sweep well conditioned
+// (the spanned subspace is the same either way); with one round the result is left in tmp.
+// The tall products run per class; the l x l factorisations of every class go out in one launch.
+// keepR: leave the two factors in rmat / rmat2 and their product in racc.
+void cholqr(sc_plan* p, const std::vector<ActiveClass>& act, const int* idx_all, int n_all, int offY, int offTmp,
+            bool left, bool keepR, int rounds) {
   const int lp = p->lp;
   cudaStream_t s = p->stream;
   ProfScope ps(p, PROF_SMALL);
-  launch_atb(p->dev_tab, idx, cnt, offY, offY, OFF(gpart), OFF(gram), rows, lp, lp, lp, lp, s);
-  launch_chol(p->dev_tab, idx, cnt, lp, OFF(rmat), s);
-  launch_gemm(gemm(p, idx, offY, OFF(rinv), offTmp, rows, lp, lp, lp, lp, lp, 0, 0), cnt, s);
-  launch_atb(p->dev_tab, idx, cnt, offTmp, offTmp, OFF(gpart), OFF(gram), rows, lp, lp, lp, lp, s);
-  launch_chol(p->dev_tab, idx, cnt, lp, OFF(rmat2), s);
-  launch_gemm(gemm(p, idx, offTmp, OFF(rinv), offY, rows, lp, lp, lp, lp, lp, 0, 0), cnt, s);
-  if (keepR) launch_gemm(gemm(p, idx, OFF(rmat2), OFF(rmat), OFF(racc), lp, lp, lp, lp, lp, lp, 0, 0), cnt, s);
+  for (int round = 0; round < rounds; ++round) {
+    const int src = round == 0 ? offY : offTmp, dst = round == 0 ? offTmp : offY;
+    for (const auto& a : act)
+      launch_atb(p->dev_tab, a.idx, a.cnt, src, src, OFF(gpart), OFF(gram), (int)(left ? a.c->m : a.c->n), lp, lp, lp,
+                 lp, s);
+    launch_chol(p->dev_tab, idx_all, n_all, lp, round == 0 ? OFF(rmat) : OFF(rmat2), s);
+    for (const auto& a : act)
+      launch_gemm(gemm(p, a.idx, src, OFF(rinv), dst, (int)(left ? a.c->m : a.c->n), lp, lp, lp, lp, lp, 0, 0), a.cnt, s);
+  }
+  if (keepR && rounds == 2)
+    launch_gemm(gemm(p, idx_all, OFF(rmat2), OFF(rmat), OFF(racc), lp, lp, lp, lp, lp, lp, 0, 0), n_all, s);
 }
 
 // Rebuild d (Eq. 2) and the bf16 operand copies of one matrix list after its U, s, V changed.
@@ -399,53 +410,74 @@ sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t 
   const int g_bf16 = p->hp.grad_dtype == SC_DTYPE_BF16;
   for (int i = 0; i < p->n_mats; ++i) p->host_tab[i].Ganc = anchor_grads[i];
   if ((st = upload_table(p)) != SC_OK) return st;
+  // the matrices that received a gradient, class by class, plus one flat list for the class-independent kernels
+  std::vector<ActiveClass> act;
+  std::vector<int> flat;
   for (auto& c : p->classes) {
-    std::vector<int> act;
+    std::vector<int> ids;
     for (int id : c.mats)
-      if (anchor_grads[id]) act.push_back(id);
-    const int cnt = (int)act.size();
-    if (!cnt) continue;
+      if (anchor_grads[id]) ids.push_back(id);
+    if (ids.empty()) continue;
     const int* idx = c.idx_all;
-    if (cnt != (int)c.mats.size()) {
-      // pageable source: the runtime has taken its copy of `act` when this returns
-      if (cudaMemcpyAsync(c.idx_dyn, act.data(), cnt * sizeof(int), cudaMemcpyHostToDevice, s) != cudaSuccess)
+    if (ids.size() != c.mats.size()) {
+      // pageable source: the runtime has taken its copy of `ids` when this returns
+      if (cudaMemcpyAsync(c.idx_dyn, ids.data(), ids.size() * sizeof(int), cudaMemcpyHostToDevice, s) != cudaSuccess)
         return SC_ERR_CUDA;
       idx = c.idx_dyn;
     }
-    const int m = (int)c.m, n = (int)c.n;
-    {
-      ProfScope ps(p, PROF_EMA);
-      launch_ema(p->dev_tab, idx, cnt, (int64_t)m * n, g_bf16, p->hp.beta_anc, s);                      // Eq. 1
-    }
-    if (p->rank > 0) {
-      // range finder: Y = M Omega, Q = orth(Y)
-      auto pass = [&](int offB, int offC, bool transposed, int tB) {   // one sweep over the momentum
-        ProfScope ps(p, PROF_PASS);
-        if (c.tensor) { tc_launch_pass(p, c, idx, cnt, transposed ? 1 : (tB ? 0 : 2)); return; }
-        if (!transposed) launch_gemm(gemm(p, idx, OFF(Manc), offB, offC, m, lp, n, n, tB ? n : lp, lp, 0, tB), cnt, s);
-        else launch_gemm(gemm(p, idx, OFF(Manc), offB, offC, n, lp, m, n, lp, lp, 1, 0), cnt, s);
-      };
-      pass(OFF(omega_t), OFF(Y), false, 1);                                                          // Y = M Omega
-      cholqr2(p, idx, cnt, OFF(Y), OFF(Y2), m, false);
-      for (int it = 0; it < p->q; ++it) {
-        pass(OFF(Y), OFF(Z), true, 0);                                                               // Z = M^T Q
-        cholqr2(p, idx, cnt, OFF(Z), OFF(Z2), n, false);
-        pass(OFF(Z), OFF(Y), false, 0);                                                              // Y = M Z
-        cholqr2(p, idx, cnt, OFF(Y), OFF(Y2), m, false);
-      }
-      // B^T = M^T Q = Qb R ; SVD of the small factor ; U = Q Ub, V = Qb Wb
-      pass(OFF(Y), OFF(Z), true, 0);
-      cholqr2(p, idx, cnt, OFF(Z), OFF(Z2), n, true);
-      {
-        ProfScope ps(p, PROF_SMALL);
-        launch_jacobi(p->dev_tab, idx, cnt, lp, rp, p->rank, p->hp.tau_p, s);                         // + Eq. 2
-        launch_gemm(gemm(p, idx, OFF(Y), OFF(ub), OFF(U), m, rp, lp, lp, rp, rp, 0, 0), cnt, s);
-        launch_gemm(gemm(p, idx, OFF(Z), OFF(wb), OFF(V), n, rp, lp, lp, rp, rp, 0, 0), cnt, s);
-        refresh_operands(p, c, idx, cnt);
-      }
-    }
-    for (int id : act) p->has_basis[id] = 1;
+    act.push_back(ActiveClass{&c, idx, (int)ids.size()});
+    flat.insert(flat.end(), ids.begin(), ids.end());
   }
+  if (flat.empty()) { p->last_tag = step_tag; return SC_OK; }
+  const int n_all = (int)flat.size();
+  if (cudaMemcpyAsync(p->idx_glob, flat.data(), flat.size() * sizeof(int), cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return SC_ERR_CUDA;
+  {
+    ProfScope ps(p, PROF_EMA);
+    for (const auto& a : act)
+      launch_ema(p->dev_tab, a.idx, a.cnt, a.c->m * a.c->n, g_bf16, p->hp.beta_anc, s);               // Eq. 1
+  }
+  if (p->rank > 0) {
+    // one sweep over the momentum: transposed ? Z <- M^T B : Y <- M B
+    auto pass = [&](int offB, bool transposed) {
+      ProfScope ps(p, PROF_PASS);
+      for (const auto& a : act) {
+        const int m = (int)a.c->m, n = (int)a.c->n;
+        if (a.c->tensor) { tc_launch_pass(p, *a.c, a.idx, a.cnt, transposed, offB); continue; }
+        const int tB = offB == OFF(omega_t);
+        if (!transposed)
+          launch_gemm(gemm(p, a.idx, OFF(Manc), offB, OFF(Y), m, lp, n, n, tB ? n : lp, lp, 0, tB), a.cnt, s);
+        else
+          launch_gemm(gemm(p, a.idx, OFF(Manc), offB, OFF(Z), n, lp, m, n, lp, lp, 1, 0), a.cnt, s);
+      }
+    };
+    // range finder: Y = M Omega, Q = orth(Y), q subspace iterations
+    pass(OFF(omega_t), false);
+    int curY = OFF(Y);
+    if (p->q == 0) cholqr(p, act, p->idx_glob, n_all, OFF(Y), OFF(Y2), true, false, 2);
+    else { cholqr(p, act, p->idx_glob, n_all, OFF(Y), OFF(Y2), true, false, 1); curY = OFF(Y2); }
+    for (int it = 0; it < p->q; ++it) {
+      pass(curY, true);                                                            // Z = M^T Q
+      cholqr(p, act, p->idx_glob, n_all, OFF(Z), OFF(Z2), false, false, 1);
+      pass(OFF(Z2), false);                                                        // Y = M Z
+      if (it == p->q - 1) { cholqr(p, act, p->idx_glob, n_all, OFF(Y), OFF(Y2), true, false, 2); curY = OFF(Y); }
+      else { cholqr(p, act, p->idx_glob, n_all, OFF(Y), OFF(Y2), true, false, 1); curY = OFF(Y2); }
+    }
+    // B^T = M^T Q = Qb R ; SVD of the small factor ; U = Q Ub, V = Qb Wb
+    pass(OFF(Y), true);
+    cholqr(p, act, p->idx_glob, n_all, OFF(Z), OFF(Z2), false, true, 2);
+    {
+      ProfScope ps(p, PROF_SMALL);
+      launch_jacobi(p->dev_tab, p->idx_glob, n_all, lp, rp, p->rank, p->hp.tau_p, s);                 // + Eq. 2
+      for (const auto& a : act) {
+        const int m = (int)a.c->m, n = (int)a.c->n;
+        launch_gemm(gemm(p, a.idx, OFF(Y), OFF(ub), OFF(U), m, rp, lp, lp, rp, rp, 0, 0), a.cnt, s);
+        launch_gemm(gemm(p, a.idx, OFF(Z), OFF(wb), OFF(V), n, rp, lp, lp, rp, rp, 0, 0), a.cnt, s);
+        refresh_operands(p, *a.c, a.idx, a.cnt);
+      }
+    }
+  }
+  for (int id : flat) p->has_basis[id] = 1;
   p->last_tag = step_tag;
   return cuda_ok(cudaGetLastError());
 }

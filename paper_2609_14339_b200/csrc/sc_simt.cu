@@ -22,7 +22,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // =====================================================================================================
 // Batched tiled GEMM  C = alpha * op(A) * op(B), fp32 accumulate, with an optional fused AdamW epilogue.
 // =====================================================================================================
-constexpr int BM = 64, BN = 64, BK = 16;
+constexpr int BM = 128, BN = 64, BK = 16;   // block tile; each of the 256 threads owns 8 rows x 4 columns
 
 struct EpiStore {};
 struct EpiAdamW {
@@ -33,15 +33,15 @@ struct EpiAdamW {
 
 template <bool kAdamW>
 __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs a, EpiAdamW epi) {
-  __shared__ float As[BK][BM + 1];
-  __shared__ float Bs[BK][BN + 1];
+  __shared__ __align__(16) float As[BK][BM + 4];
+  __shared__ __align__(16) float Bs[BK][BN + 4];
   const MatDev& md = a.tab[a.idx[blockIdx.z]];
   const float* A = field<const float>(md, a.offA);
   const bf16* Ab = reinterpret_cast<const bf16*>(A);
   const float* B = field<const float>(md, a.offB);
   const int row0 = blockIdx.y * BM, col0 = blockIdx.x * BN;
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
-  float acc[4][4] = {};
+  float acc[8][4] = {};
   for (int k0 = 0; k0 < a.K; k0 += BK) {
     for (int e = tid; e < BM * BK; e += 256) {
       int r, k;
@@ -65,13 +65,13 @@ __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs a, EpiAdamW epi) {
     __syncthreads();
 #pragma unroll
     for (int k = 0; k < BK; ++k) {
-      float av[4], bv[4];
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[k][ty * 8]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&As[k][ty * 8 + 4]);
+      const float4 b0 = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
+      const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+      const float bv[4] = {b0.x, b0.y, b0.z, b0.w};
 #pragma unroll
-      for (int i = 0; i < 4; ++i) av[i] = As[k][ty * 4 + i];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) bv[j] = Bs[k][tx * 4 + j];
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < 8; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
     }
@@ -80,8 +80,8 @@ __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs a, EpiAdamW epi) {
   if (!kAdamW) {
     float* C = field<float>(md, a.offC);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int gr = row0 + ty * 4 + i;
+    for (int i = 0; i < 8; ++i) {
+      const int gr = row0 + ty * 8 + i;
       if (gr >= a.M) continue;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -96,8 +96,8 @@ __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs a, EpiAdamW epi) {
     const float* Gf = reinterpret_cast<const float*>(md.G);
     const bf16* Gb = reinterpret_cast<const bf16*>(md.G);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int gr = row0 + ty * 4 + i;
+    for (int i = 0; i < 8; ++i) {
+      const int gr = row0 + ty * 8 + i;
       if (gr >= a.M) continue;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
@@ -151,8 +151,8 @@ template <int MT>
 __global__ void __launch_bounds__(256) atb_kernel(const MatDev* tab, const int* idx, int offA, int offB, int offPart,
                                                   int rows, int ca, int cb, int lda, int ldb, int rows_per_split) {
   constexpr int TS = 16 * MT;          // output tile edge
-  __shared__ float As[32][TS + 1];
-  __shared__ float Bs[32][TS + 1];
+  __shared__ __align__(16) float As[32][TS + 4];
+  __shared__ __align__(16) float Bs[32][TS + 4];
   const MatDev& md = tab[idx[blockIdx.z]];
   const float* A = field<const float>(md, offA);
   const float* B = field<const float>(md, offB);
@@ -174,9 +174,9 @@ __global__ void __launch_bounds__(256) atb_kernel(const MatDev* tab, const int* 
     for (int rr = 0; rr < 32; ++rr) {
       float av[MT], bv[MT];
 #pragma unroll
-      for (int i = 0; i < MT; ++i) av[i] = As[rr][ty + 16 * i];
+      for (int i = 0; i < MT; ++i) av[i] = As[rr][ty * MT + i];     // contiguous: compiles to 128-bit loads
 #pragma unroll
-      for (int j = 0; j < MT; ++j) bv[j] = Bs[rr][tx + 16 * j];
+      for (int j = 0; j < MT; ++j) bv[j] = Bs[rr][tx * MT + j];
 #pragma unroll
       for (int i = 0; i < MT; ++i)
 #pragma unroll
@@ -188,7 +188,7 @@ __global__ void __launch_bounds__(256) atb_kernel(const MatDev* tab, const int* 
   for (int i = 0; i < MT; ++i)
 #pragma unroll
     for (int j = 0; j < MT; ++j) {
-      const int gi = i0 + ty + 16 * i, gj = j0 + tx + 16 * j;
+      const int gi = i0 + ty * MT + i, gj = j0 + tx * MT + j;
       if (gi < ca && gj < cb) part[(size_t)gi * cb + gj] = acc[i][j];
     }
 }
@@ -347,21 +347,31 @@ __global__ void __launch_bounds__(256) chol_kernel(const MatDev* tab, const int*
   const int t = threadIdx.x;
   for (int j = 0; j < lp; ++j) {
     const int i = t;
-    double s = 0.0;
+    float s = 0.f;
     if (i >= j && i < lp) {
-      s = (double)G[(size_t)j * lp + i];
-      for (int k = 0; k < j; ++k) s -= (double)R[(size_t)k * lp + j] * (double)R[(size_t)k * lp + i];
+      // four independent partial sums: the dot product is a latency chain otherwise. fp32 is enough: the Gram
+      // matrix itself was accumulated in fp32, and the second Cholesky QR round repairs what is lost here.
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+      int k = 0;
+      for (; k + 3 < j; k += 4) {
+        s0 = fmaf(R[(size_t)k * lp + j], R[(size_t)k * lp + i], s0);
+        s1 = fmaf(R[(size_t)(k + 1) * lp + j], R[(size_t)(k + 1) * lp + i], s1);
+        s2 = fmaf(R[(size_t)(k + 2) * lp + j], R[(size_t)(k + 2) * lp + i], s2);
+        s3 = fmaf(R[(size_t)(k + 3) * lp + j], R[(size_t)(k + 3) * lp + i], s3);
+      }
+      for (; k < j; ++k) s0 = fmaf(R[(size_t)k * lp + j], R[(size_t)k * lp + i], s0);
+      s = G[(size_t)j * lp + i] - ((s0 + s1) + (s2 + s3));
     }
     if (i == j) {
-      const double gjj = (double)G[(size_t)j * lp + j];
-      const bool ok = (s > 1e-6 * gjj) && (gjj > 0.0);
-      const float rjj = ok ? (float)sqrt(s) : 0.f;
+      const float gjj = G[(size_t)j * lp + j];
+      const bool ok = (s > 1e-6f * gjj) && (gjj > 0.f);
+      const float rjj = ok ? sqrtf(s) : 0.f;
       piv_inv = ok ? 1.f / rjj : 0.f;
       invd[j] = piv_inv;
       R[(size_t)j * lp + j] = rjj;
     }
     __syncthreads();
-    if (i > j && i < lp) R[(size_t)j * lp + i] = (float)s * piv_inv;
+    if (i > j && i < lp) R[(size_t)j * lp + i] = s * piv_inv;
     if (i < j) R[(size_t)j * lp + i] = 0.f;
     __syncthreads();
   }
@@ -371,9 +381,16 @@ __global__ void __launch_bounds__(256) chol_kernel(const MatDev* tab, const int*
     for (int i = lp - 1; i > c; --i) Ri[(size_t)i * lp + c] = 0.f;
     Ri[(size_t)c * lp + c] = invd[c];
     for (int i = c - 1; i >= 0; --i) {
-      double s = 0.0;
-      for (int k = i + 1; k <= c; ++k) s += (double)R[(size_t)i * lp + k] * (double)Ri[(size_t)k * lp + c];
-      Ri[(size_t)i * lp + c] = (float)(-s) * invd[i];
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+      int k = i + 1;
+      for (; k + 3 <= c; k += 4) {
+        s0 = fmaf(R[(size_t)i * lp + k], Ri[(size_t)k * lp + c], s0);
+        s1 = fmaf(R[(size_t)i * lp + k + 1], Ri[(size_t)(k + 1) * lp + c], s1);
+        s2 = fmaf(R[(size_t)i * lp + k + 2], Ri[(size_t)(k + 2) * lp + c], s2);
+        s3 = fmaf(R[(size_t)i * lp + k + 3], Ri[(size_t)(k + 3) * lp + c], s3);
+      }
+      for (; k <= c; ++k) s0 = fmaf(R[(size_t)i * lp + k], Ri[(size_t)k * lp + c], s0);
+      Ri[(size_t)i * lp + c] = -((s0 + s1) + (s2 + s3)) * invd[i];
     }
   }
 }
@@ -409,7 +426,7 @@ __global__ void __launch_bounds__(kJacobiThreads) jacobi_kernel(const MatDev* ta
   }
   __syncthreads();
   const int half = lp / 2;
-  for (int sweep = 0; sweep < 24; ++sweep) {
+  for (int sweep = 0; sweep < 16; ++sweep) {
     if (tid == 0) rotated = 0;
     __syncthreads();
     for (int rd = 0; rd < lp - 1; ++rd) {
@@ -426,7 +443,7 @@ __global__ void __launch_bounds__(kJacobiThreads) jacobi_kernel(const MatDev* ta
         a = warp_sum(a); b = warp_sum(b); c = warp_sum(c);
         const float lim = sqrtf(a) * sqrtf(b);
         if (!(fabsf(c) > 1e-7f * lim) || lim == 0.f) continue;
-        if (fabsf(c) > 2e-6f * lim && lane == 0) rotated = 1;
+        if (fabsf(c) > 4e-6f * lim && lane == 0) rotated = 1;   // below this the fp32 dot product is noise
         const float zeta = (b - a) / (2.f * c);
         const float tt = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
         const float cs = rsqrtf(1.f + tt * tt), sn = cs * tt;

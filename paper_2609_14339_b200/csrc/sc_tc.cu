@@ -115,7 +115,7 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16(int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-constexpr int kMapsPerMat = 20;
+constexpr int kMapsPerMat = 22;
 constexpr int kPerCallMaps = 6;   // the first six are rebuilt whenever the caller's buffers move
 enum { MAP_G = 0,    // masked gradient, bf16, box 64 x 128 (MMA A operand of the projection)
        MAP_G32,      // masked gradient, bf16, box 32 x 128, 64-byte swizzle (streaming tile of the fused update)
@@ -126,6 +126,7 @@ enum { MAP_G = 0,    // masked gradient, bf16, box 64 x 128 (MMA A operand of th
        MAP_M_K,      // anchor momentum as a K-major A operand: box 32 floats x 128 rows
        MAP_M_MN,     // anchor momentum as an MN-major A operand: box 32 floats x 32 rows (one swizzle atom column)
        MAP_Y, MAP_Z, MAP_OMEGA,  // m x lp, n x lp, n x lp row-major fp32 as MN-major B operands: box 32 x 32
+       MAP_Y2, MAP_Z2,           // the scratch twins of Y and Z (a single-round Cholesky QR leaves its result there)
        MAP_SPARE };
 constexpr int kTileBytes = 128 * 128;   // 128 rows x 64 bf16
 
@@ -866,6 +867,8 @@ sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_
       ok = ok && encode_tf32(mp + MAP_Y, md.Y, lp, c.m, kPassK, true);
       ok = ok && encode_tf32(mp + MAP_Z, md.Z, lp, c.n, kPassK, true);
       ok = ok && encode_tf32(mp + MAP_OMEGA, md.omega, lp, c.n, kPassK, true);
+      ok = ok && encode_tf32(mp + MAP_Y2, md.Y2, lp, c.m, kPassK, true);
+      ok = ok && encode_tf32(mp + MAP_Z2, md.Z2, lp, c.n, kPassK, true);
       if (!ok) return SC_ERR_CUDA;
     }
   }
@@ -903,8 +906,8 @@ sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count
   return cuda_ok(cudaGetLastError());
 }
 
-// One sweep over the anchor momentum. which: 0 = Y <- M Omega, 1 = Z <- M^T Y, 2 = Y <- M Z.
-sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, int which) {
+// One sweep over the anchor momentum: transposed ? Z <- M^T B : Y <- M B, with B one of the n x lp / m x lp buffers.
+sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, bool transposed, int b_field_off) {
   const int lp = p->lp, m = (int)c.m, n = (int)c.n;
   const int stage_bytes = kTileBytes + (lp / 32) * kAtomBytes;
   int stages = (200 * 1024) / stage_bytes;
@@ -912,15 +915,22 @@ sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, i
   const size_t smem = (size_t)stages * stage_bytes + 1024 + 256;
   uint32_t cols = 32;
   while ((int)cols < lp) cols <<= 1;
+  int b_map;
+  if (b_field_off == (int)offsetof(MatDev, omega_t) || b_field_off == (int)offsetof(MatDev, omega)) b_map = MAP_OMEGA;
+  else if (b_field_off == (int)offsetof(MatDev, Y)) b_map = MAP_Y;
+  else if (b_field_off == (int)offsetof(MatDev, Y2)) b_map = MAP_Y2;
+  else if (b_field_off == (int)offsetof(MatDev, Z)) b_map = MAP_Z;
+  else if (b_field_off == (int)offsetof(MatDev, Z2)) b_map = MAP_Z2;
+  else return SC_ERR_INVALID_ARG;
   const CUtensorMap* maps = static_cast<const CUtensorMap*>(c.tmaps);
-  if (which == 1) {
+  if (transposed) {
     dim3 grid((n + 127) / 128, 1, count);
-    pass_kernel<true><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, MAP_Y, (int)offsetof(MatDev, Z), n, m, lp,
+    pass_kernel<true><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, b_map, (int)offsetof(MatDev, Z), n, m, lp,
                                                        stages, cols, p->status_dev);
   } else {
     dim3 grid((m + 127) / 128, 1, count);
-    pass_kernel<false><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, which == 0 ? MAP_OMEGA : MAP_Z,
-                                                        (int)offsetof(MatDev, Y), m, n, lp, stages, cols, p->status_dev);
+    pass_kernel<false><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, b_map, (int)offsetof(MatDev, Y), m, n, lp,
+                                                        stages, cols, p->status_dev);
   }
   ++g_kernel_launches;
   return cuda_ok(cudaGetLastError());
