@@ -29,6 +29,8 @@ METRIC = "spectral-correction step: gradient GB/s (and ms per step) on the 8B-sh
 REFRESH_EVERY = 4
 BYTES_PER_ELEM_STEADY = 28.0      # read G (2) + read/write fp32 W, m, v (24) + write bf16 W (2)
 BYTES_PER_ELEM_UPDATE = 28.0      # what the fused update kernel itself moves per element (G is re-read here)
+TRAFFIC_PER_ELEM_UPDATE = 27.24   # dram read+write bytes per element of that kernel from one ncu capture
+                                  # (profiles/fused_update_stream_kernel_ffn14336x4096.md); scales with elements
 
 
 def parse_args():
@@ -288,10 +290,13 @@ def run_ours(args):
 
     peaks = measured_peaks()
     upd_gbs = n_elems * BYTES_PER_ELEM_UPDATE / (update_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "fused_update_kernel", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+    upd_launches = max(prof["update"]["spans"] / nprof, 1)          # one launch per shape class and step
+    roofline = {"bound": "hbm", "kernel": "fused_update_stream_kernel", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"],
+                "traffic": TRAFFIC_PER_ELEM_UPDATE * n_elems / upd_launches, "peak_source": peaks["source"],
                 "algorithmic_bytes_per_element": BYTES_PER_ELEM_UPDATE,
-                "launch_ms": update_ms / max(prof["update"]["spans"] / nprof, 1)}
+                "algorithmic_bytes_per_launch": BYTES_PER_ELEM_UPDATE * n_elems / upd_launches,
+                "launches_per_step": upd_launches, "launch_ms": update_ms / upd_launches}
     step_roofline_ms = max(n_elems * BYTES_PER_ELEM_STEADY / (peaks["hbm_gbs"] * 1e9),
                            n_elems * 4.0 * cfg["r"] / (peaks["bf16_tflops"] * 1e12)) * 1e3
 

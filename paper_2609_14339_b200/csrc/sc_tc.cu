@@ -1,7 +1,8 @@
 // Tensor-core (tcgen05 / TMEM / TMA) kernels of the spectral-correction step for sm_100a.
 //
 //   project_kernel        T = G (Vhi + Vlo)              streaming GEMM over the masked gradient, N = rank
-//   fused_update_kernel   G_proj = clip * (alpha_s G + (Uhi + Ulo)(Chi + Clo)^T), then AdamW, one HBM pass
+//   pass_kernel           Y = M B / Z = M^T B         sweeps over the anchor momentum (tf32), range finder
+//   fused_update_stream_kernel   G_proj = clip * (alpha_s G + (Uhi + Ulo)(Chi + Clo)^T), then AdamW, one HBM pass
 //
 // Operands: G is bf16 as given; the fp32 factors are carried as a sum of two bf16 numbers (hi + lo), so
 // the products lose nothing that matters at the 2e-3 tolerance. All MMA operands sit in shared memory in
@@ -9,7 +10,6 @@
 // Every wait on an mbarrier is bounded; when a wait runs out the kernel latches an error bit, drains what
 // it has in flight, frees its TMEM and returns.
 #include <cuda.h>
-#include <stdlib.h>
 
 #include "sc_internal.cuh"
 
@@ -359,10 +359,7 @@ pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const C
 }
 
 // =====================================================================================================
-// Fused correction + AdamW for one 128 x 128 tile.
-//   mainloop (one elected thread): R = (Uhi + Ulo)(Cthi + Ctlo)^T over K = rank, three bf16 MMAs per K step
-//   (hi*hi, hi*lo, lo*hi; lo*lo is below fp32 resolution), accumulated in TMEM;
-//   epilogue (all 8 warps): TMEM -> swizzled shared staging -> coalesced 128-bit pass over G, W, m, v.
+// AdamW on four elements of G_proj = clip * (alpha_s * G + R), R = the low-rank part from the tensor cores.
 // =====================================================================================================
 __device__ __forceinline__ void adamw4(const StepScalars& s, float clip, const float g_raw[4], const float4& r,
                                        float4& w, float4& m1, float4& m2, float4& gp) {
@@ -376,145 +373,6 @@ __device__ __forceinline__ void adamw4(const StepScalars& s, float clip, const f
     const float den = fmaf(sqrtf(vo), s.inv_sqrt_bc2, s.eps);
     W[j] = fmaf(-s.step_size, mo / den, W[j] * s.decay);
     M1[j] = mo; M2[j] = vo; GP[j] = g;
-  }
-}
-
-__global__ void __launch_bounds__(256, 3)
-fused_update_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const CUtensorMap* __restrict__ maps,
-                    int m, int n, int rp, StepScalars sc, const float* __restrict__ clip_ptr, unsigned* status) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + 4 * kTileBytes);
-  uint64_t* mma_done = full + 1;     // per K chunk: the operand tiles may be overwritten
-  uint64_t* accum_done = full + 2;   // once: the accumulator is complete (waited on by every thread, phase 0)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_done + 1);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int inst = blockIdx.z;
-  const MatDev& md = tab[idx[inst]];
-  const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
-  const int col0 = blockIdx.x * 128, row0 = blockIdx.y * 128;
-  const int nch = (rp + 63) >> 6;
-
-  if (threadIdx.x == 0) {
-    mbar_init(full, 1);
-    mbar_init(mma_done, 1);
-    mbar_init(accum_done, 1);
-    *abort_flag = 0;
-    fence_barrier_init();
-    fence_proxy_async();
-  }
-  if (warp == 0) tmem_alloc(tmem_slot, 128);
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_d = *tmem_slot;
-
-  if (warp == 0) {
-    if (lane == 0) {
-      tensormap_acquire(mp + MAP_UHI); tensormap_acquire(mp + MAP_ULO);
-      tensormap_acquire(mp + MAP_CTHI); tensormap_acquire(mp + MAP_CTLO);
-      const uint32_t idesc = umma_idesc_bf16(128);
-      const uint32_t uh = smem_u32(smem), ul = uh + kTileBytes, ch = ul + kTileBytes, cl = ch + kTileBytes;
-      for (int c = 0; c < nch; ++c) {
-        if (c > 0 && !mbar_wait(mma_done, (c - 1) & 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
-        mbar_expect_tx(full, 4 * kTileBytes);
-        tma_load_2d(smem, mp + MAP_UHI, full, c * 64, row0);
-        tma_load_2d(smem + kTileBytes, mp + MAP_ULO, full, c * 64, row0);
-        tma_load_2d(smem + 2 * kTileBytes, mp + MAP_CTHI, full, c * 64, col0);
-        tma_load_2d(smem + 3 * kTileBytes, mp + MAP_CTLO, full, c * 64, col0);
-        if (!mbar_wait(full, c & 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
-        tc_fence_after();
-        const int ksteps = min(64, rp - c * 64) >> 4;
-        for (int k = 0; k < ksteps; ++k) {
-          const uint64_t ah = umma_desc_k128(uh + k * 32), al = umma_desc_k128(ul + k * 32);
-          const uint64_t bh = umma_desc_k128(ch + k * 32), bl = umma_desc_k128(cl + k * 32);
-          umma_bf16(tmem_d, ah, bh, idesc, (c | k) != 0);
-          umma_bf16(tmem_d, ah, bl, idesc, 1);
-          umma_bf16(tmem_d, al, bh, idesc, 1);
-        }
-        umma_commit(mma_done);
-      }
-      umma_commit(accum_done);
-    }
-    __syncwarp();
-  }
-  bool ok = mbar_wait(accum_done, 0, abort_flag);
-  if (!ok) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
-  tc_fence_after();
-
-  // TMEM -> shared staging: 128 rows x 32 slots of 16 bytes, slot index XOR (row & 31) keeps both the
-  // row-per-thread writes here and the row-per-warp reads below free of bank conflicts.
-  float4* stage = reinterpret_cast<float4*>(smem);
-  {
-    const int q = warp & 3, h = warp >> 2;
-    const int r = q * 32 + lane;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      float v[16];
-      const int cbase = h * 64 + j * 16;
-      tmem_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + cbase, v);
-      tmem_ld_wait();
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        stage[r * 32 + (((cbase >> 2) + i) ^ (r & 31))] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-    }
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 0) tmem_dealloc(tmem_d, 128);
-  if (*abort_flag) return;
-
-  const float clip = *clip_ptr;
-  const int col = col0 + lane * 4;
-  if (col >= n) return;
-  const uint2* __restrict__ G = reinterpret_cast<const uint2*>(md.G);
-  float4* __restrict__ W = reinterpret_cast<float4*>(md.W);
-  float4* __restrict__ M1 = reinterpret_cast<float4*>(md.m1);
-  float4* __restrict__ M2 = reinterpret_cast<float4*>(md.m2);
-  uint2* __restrict__ Wb = reinterpret_cast<uint2*>(md.Wb);
-  float4* __restrict__ GP = reinterpret_cast<float4*>(md.gproj_dbg);
-  constexpr int kUnroll = 2;
-  for (int rr = warp; rr < 128; rr += 8 * kUnroll) {
-    uint2 graw[kUnroll];
-    float4 w[kUnroll], m1[kUnroll], m2[kUnroll];
-    size_t off[kUnroll];
-    bool live[kUnroll];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const int row = row0 + rr + 8 * u;
-      live[u] = row < m;
-      off[u] = ((size_t)row * n + col) >> 2;
-      if (live[u]) {
-        graw[u] = __ldg(G + off[u]);
-        w[u] = __ldcs(W + off[u]);
-        m1[u] = __ldcs(M1 + off[u]);
-        m2[u] = __ldcs(M2 + off[u]);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      if (!live[u]) continue;
-      const int lr = rr + 8 * u;
-      const float4 r = stage[lr * 32 + (lane ^ (lr & 31))];
-      const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&graw[u].x);
-      const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&graw[u].y);
-      const float g4[4] = {__low2float(g01), __high2float(g01), __low2float(g23), __high2float(g23)};
-      float4 gp;
-      adamw4(sc, clip, g4, r, w[u], m1[u], m2[u], gp);
-      __stcs(W + off[u], w[u]);
-      __stcs(M1 + off[u], m1[u]);
-      __stcs(M2 + off[u], m2[u]);
-      if (Wb) {
-        __nv_bfloat162 b01 = __floats2bfloat162_rn(w[u].x, w[u].y), b23 = __floats2bfloat162_rn(w[u].z, w[u].w);
-        uint2 pk;
-        pk.x = *reinterpret_cast<uint32_t*>(&b01);
-        pk.y = *reinterpret_cast<uint32_t*>(&b23);
-        __stcs(Wb + off[u], pk);
-      }
-      if (GP) GP[off[u]] = gp;
-    }
   }
 }
 
@@ -796,7 +654,6 @@ sc_status tc_init() {
   static bool attrs_done = false;
   if (!attrs_done) {
     if (cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(fused_update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 72 * 1024) != cudaSuccess ||
         cudaFuncSetAttribute(fused_update_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              kStreamSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
         cudaFuncSetAttribute(pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
@@ -938,15 +795,6 @@ sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, b
 
 sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc) {
   const int m = (int)c.m, n = (int)c.n;
-  static const bool use_tiled = getenv("SC_FUSED_TILED") != nullptr;   // the older one-tile-per-block kernel
-  if (use_tiled) {
-    dim3 grid((n + 127) / 128, (m + 127) / 128, count);
-    const size_t smem = 4 * kTileBytes + 1024 + 64;
-    fused_update_kernel<<<grid, 256, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), m, n,
-                                                        p->rp, sc, p->clip_dev, p->status_dev);
-    ++g_kernel_launches;
-    return cuda_ok(cudaGetLastError());
-  }
   static int n_sm = 0;
   if (!n_sm) {
     int dev = 0;
