@@ -239,7 +239,7 @@ def run_ours(args):
     n_elems = sum(m * n for m, n in shapes)
     gsize = 2 if cfg["dtype"] == "bf16" else 4
     hp = sc.Hparams.default(grad_dtype=sc.SC_DTYPE_BF16 if cfg["dtype"] == "bf16" else sc.SC_DTYPE_FP32,
-                            power_iters=1, tau_p=1e-3)
+                            power_iters=1, warm_start=1, warm_power_iters=0, tau_p=1e-3)
     plan = sc.Plan(shapes, cfg["r"], cfg["keep"], hp, device=device)
     lib = sc.load_library()
 
@@ -306,7 +306,8 @@ def run_ours(args):
         "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": args.workload, "matrices": len(shapes), "elements": n_elems, "rank": cfg["r"],
                    "keep": cfg["keep"], "tokens": cfg["tokens"], "anchor_refresh_every": REFRESH_EVERY,
-                   "power_iters": 1, "parallelism": "replicas x%d" % world,
+                   "power_iters": 1, "range_finder": "cold start q=1 on the first arrival, warm start (previous V) q=0 afterwards",
+                   "parallelism": "replicas x%d" % world,
                    "l2": "inputs (>100 GB resident) far larger than L2; no flush needed"},
         "gpu_launches": int(launches),
         "steady_step_ms": steady_ms, "anchor_refresh_ms": refresh_ms,

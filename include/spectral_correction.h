@@ -91,6 +91,12 @@ typedef struct sc_hparams {
   int32_t power_iters;     /* q: subspace (power) iterations of the range finder, 0..16 */
   int32_t engine;          /* sc_engine */
   int32_t collect_stats;   /* 1: also accumulate ||g||^2 every step so that sc_get_stats can report eta_r and ||G_proj|| */
+  int32_t warm_start;      /* 1: a matrix that already has a basis starts the range finder from its previous right basis V
+                              (columns rank..l-1 from the sketch) and runs warm_power_iters instead of power_iters.
+                              The anchor momentum drifts slowly, so successive arrivals act as accumulated subspace
+                              iterations at two sweeps per arrival. 0: always start from the sketch. */
+  int32_t warm_power_iters; /* q used on a warm start, 0..16 */
+  int32_t reserved;
   uint64_t seed;           /* key of the counter-based Rademacher sketch */
 } sc_hparams;
 
@@ -110,7 +116,7 @@ typedef struct sc_mat_stats {
 } sc_mat_stats;
 
 /* Fill *hp with defaults: alpha 0.3, tau_p 1e-3, beta_anc 0.9, lr 2e-5, betas (0.9, 0.999), eps 1e-8,
- * weight_decay 0, no clipping, grads prescaled, bf16 gradients, l = rank, q = 1, engine AUTO, no stats, seed 0.
+ * weight_decay 0, no clipping, grads prescaled, bf16 gradients, l = rank, q = 1, cold starts only, engine AUTO, no stats, seed 0.
  * (alpha, tau_p, lr, betas: the paper's defaults; the others are not given there.) */
 SC_API sc_status sc_hparams_default(sc_hparams* hp);
 

@@ -311,13 +311,21 @@ def new_state(m: int, n: int) -> MatrixState:
 
 
 def anchor_update(state: MatrixState, G_anc, hp: Hyper, r: int, mode: str = "exact",
-                  Omega=None, q: int = 1) -> MatrixState:
-    """Anchor arrival: Eq. 1 then the rank-r basis of the new momentum (cached until the next arrival)."""
+                  Omega=None, q: int = 1, warm: bool = False, q_warm: int = 0) -> MatrixState:
+    """Anchor arrival: Eq. 1 then the rank-r basis of the new momentum (cached until the next arrival).
+
+    mirror mode with warm=True: a matrix that already has a basis starts the range finder from
+    [previous V | sketch columns r..l-1] instead of the sketch and runs q_warm power iterations.
+    """
     state.M_anc = anchor_ema(state.M_anc, G_anc, hp.beta_anc)
     if mode == "exact":
         state.U, state.s, state.V = truncate(*svd_exact(state.M_anc), r)
     elif mode == "mirror":
-        state.U, state.s, state.V = mirror_basis(state.M_anc, Omega, q, r)
+        if warm and state.have_anchor and r > 0:
+            start = np.concatenate([state.V[:, :r], Omega[:, r:]], axis=1)
+            state.U, state.s, state.V = mirror_basis(state.M_anc, start, q_warm, r)
+        else:
+            state.U, state.s, state.V = mirror_basis(state.M_anc, Omega, q, r)
     else:
         raise ValueError(mode)
     state.have_anchor = True

@@ -34,7 +34,8 @@ class Hparams(C.Structure):
                 ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float), ("weight_decay", C.c_float),
                 ("max_grad_norm", C.c_float), ("grads_prescaled", C.c_int32), ("grad_dtype", C.c_int32),
                 ("sketch_width", C.c_int32), ("power_iters", C.c_int32), ("engine", C.c_int32),
-                ("collect_stats", C.c_int32), ("seed", C.c_uint64)]
+                ("collect_stats", C.c_int32), ("warm_start", C.c_int32), ("warm_power_iters", C.c_int32),
+                ("reserved", C.c_int32), ("seed", C.c_uint64)]
 
     @classmethod
     def default(cls, **kw) -> "Hparams":

@@ -84,7 +84,8 @@ struct ShapeClass {
   float* omega_t = nullptr;
   float* omega = nullptr;
   int* idx_all = nullptr;  // device: mats[]
-  int* idx_dyn = nullptr;  // device: subset list written per call (anchor arrivals)
+  int* idx_dyn = nullptr;  // device: subset list written per call (anchor arrivals, cold starts)
+  int* idx_dyn2 = nullptr; // device: subset list written per call (anchor arrivals, warm starts)
   bool tensor = false;     // served by the tcgen05 kernels
   int ksplit = 1;
   void* tmaps = nullptr;   // device: per-instance tensor maps (tensor engine only)
@@ -113,7 +114,8 @@ struct sc_plan {
   std::vector<sc::MatDev> host_tab;   // host mirror of the device table
   std::vector<sc::MatDev> last_uploaded;
   sc::MatDev* dev_tab = nullptr;
-  int* idx_glob = nullptr;            // device: flat list of the matrices an anchor call touches
+  int* idx_glob = nullptr;            // device: flat list of the matrices an anchor call touches (cold starts)
+  int* idx_glob2 = nullptr;           // the same for warm starts
   char* staging = nullptr;            // pinned, kStagingSlots * staging_bytes
   size_t staging_bytes = 0;
   cudaEvent_t staging_ev[sc::kStagingSlots]{};
@@ -166,6 +168,8 @@ void launch_epilogue_simt(const MatDev* tab, const int* idx, int count, int m, i
 void launch_ema(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, float beta, cudaStream_t s);
 void launch_sketch(float* omega_t, int lp, int l, int64_t n, uint64_t seed, cudaStream_t s);
 void launch_sketch_rowmajor(float* omega, int64_t rows, int width, uint64_t seed, cudaStream_t s);
+void launch_warm_start(const MatDev* tab, const int* idx, int count, int n, int lp, int l, int rp, int rank,
+                       uint64_t seed, cudaStream_t s);
 void launch_sketch_padded(float* omega, int64_t rows, int lp, int l, uint64_t seed, cudaStream_t s);
 void launch_chol(const MatDev* tab, const int* idx, int count, int lp, int offR, cudaStream_t s);
 void launch_jacobi(const MatDev* tab, const int* idx, int count, int lp, int rp, int rank, float tau_p, cudaStream_t s);

@@ -39,6 +39,7 @@ bool derive_dims(int rank, const sc_hparams* hp, Dims* d) {
   int l = hp->sketch_width > 0 ? hp->sketch_width : rank;
   if (l < rank || l > kMaxRank) return false;
   if (hp->power_iters < 0 || hp->power_iters > 16) return false;
+  if (hp->warm_power_iters < 0 || hp->warm_power_iters > 16) return false;
   d->rp = rank > 0 ? round_up_int(rank, 16) : 0;
   d->rk = round_up_int(d->rp, 64);
   d->l = l;
@@ -101,6 +102,8 @@ size_t layout(sc_plan* p, bool assign) {
   for (auto& c : p->classes) {
     int* a = cv.take<int>(c.mats.size());
     int* b = cv.take<int>(c.mats.size());
+    int* b2 = cv.take<int>(c.mats.size());
+    if (assign) c.idx_dyn2 = b2;
     float* om = cv.take<float>((size_t)lp * c.n);
     float* omr = c.tensor ? cv.take<float>((size_t)lp * c.n) : nullptr;
     if (assign) c.omega = omr;
@@ -155,7 +158,8 @@ size_t layout(sc_plan* p, bool assign) {
     }
   }
   int* glob = cv.take<int>(n_mats);
-  if (assign) p->idx_glob = glob;
+  int* glob2 = cv.take<int>(n_mats);
+  if (assign) { p->idx_glob = glob; p->idx_glob2 = glob2; }
   return align_up(cv.off);
 }
 
@@ -303,6 +307,7 @@ sc_status sc_hparams_default(sc_hparams* hp) {
   hp->lr = 2e-5f; hp->beta1 = 0.9f; hp->beta2 = 0.999f; hp->eps = 1e-8f; hp->weight_decay = 0.f;
   hp->max_grad_norm = 0.f; hp->grads_prescaled = 1; hp->grad_dtype = SC_DTYPE_BF16;
   hp->sketch_width = 0; hp->power_iters = 1; hp->engine = SC_ENGINE_AUTO; hp->collect_stats = 0; hp->seed = 0;
+  hp->warm_start = 0; hp->warm_power_iters = 0;
   return SC_OK;
 }
 
@@ -410,38 +415,50 @@ sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t 
   const int g_bf16 = p->hp.grad_dtype == SC_DTYPE_BF16;
   for (int i = 0; i < p->n_mats; ++i) p->host_tab[i].Ganc = anchor_grads[i];
   if ((st = upload_table(p)) != SC_OK) return st;
-  // the matrices that received a gradient, class by class, plus one flat list for the class-independent kernels
-  std::vector<ActiveClass> act;
-  std::vector<int> flat;
+  // The matrices that received a gradient, class by class, in two groups: cold starts (range finder from the
+  // sketch) and warm starts (from the previous right basis), each with one flat list for the class-independent kernels.
+  std::vector<ActiveClass> act[2];
+  std::vector<int> flat[2];
   for (auto& c : p->classes) {
-    std::vector<int> ids;
+    std::vector<int> ids[2];
     for (int id : c.mats)
-      if (anchor_grads[id]) ids.push_back(id);
-    if (ids.empty()) continue;
-    const int* idx = c.idx_all;
-    if (ids.size() != c.mats.size()) {
-      // pageable source: the runtime has taken its copy of `ids` when this returns
-      if (cudaMemcpyAsync(c.idx_dyn, ids.data(), ids.size() * sizeof(int), cudaMemcpyHostToDevice, s) != cudaSuccess)
-        return SC_ERR_CUDA;
-      idx = c.idx_dyn;
+      if (anchor_grads[id]) ids[(p->hp.warm_start && p->has_basis[id] && p->rank > 0) ? 1 : 0].push_back(id);
+    for (int w = 0; w < 2; ++w) {
+      if (ids[w].empty()) continue;
+      const int* idx = c.idx_all;
+      if (ids[w].size() != c.mats.size()) {
+        int* dyn = w ? c.idx_dyn2 : c.idx_dyn;
+        // pageable source: the runtime has taken its copy of the list when this returns
+        if (cudaMemcpyAsync(dyn, ids[w].data(), ids[w].size() * sizeof(int), cudaMemcpyHostToDevice, s) != cudaSuccess)
+          return SC_ERR_CUDA;
+        idx = dyn;
+      }
+      act[w].push_back(ActiveClass{&c, idx, (int)ids[w].size()});
+      flat[w].insert(flat[w].end(), ids[w].begin(), ids[w].end());
     }
-    act.push_back(ActiveClass{&c, idx, (int)ids.size()});
-    flat.insert(flat.end(), ids.begin(), ids.end());
   }
-  if (flat.empty()) { p->last_tag = step_tag; return SC_OK; }
-  const int n_all = (int)flat.size();
-  if (cudaMemcpyAsync(p->idx_glob, flat.data(), flat.size() * sizeof(int), cudaMemcpyHostToDevice, s) != cudaSuccess)
-    return SC_ERR_CUDA;
+  if (flat[0].empty() && flat[1].empty()) { p->last_tag = step_tag; return SC_OK; }
+  for (int w = 0; w < 2; ++w)
+    if (!flat[w].empty() &&
+        cudaMemcpyAsync(w ? p->idx_glob2 : p->idx_glob, flat[w].data(), flat[w].size() * sizeof(int),
+                        cudaMemcpyHostToDevice, s) != cudaSuccess)
+      return SC_ERR_CUDA;
   {
     ProfScope ps(p, PROF_EMA);
-    for (const auto& a : act)
-      launch_ema(p->dev_tab, a.idx, a.cnt, a.c->m * a.c->n, g_bf16, p->hp.beta_anc, s);               // Eq. 1
+    for (int w = 0; w < 2; ++w)
+      for (const auto& a : act[w])
+        launch_ema(p->dev_tab, a.idx, a.cnt, a.c->m * a.c->n, g_bf16, p->hp.beta_anc, s);             // Eq. 1
   }
-  if (p->rank > 0) {
+  for (int w = 0; w < 2 && p->rank > 0; ++w) {
+    if (flat[w].empty()) continue;
+    const std::vector<ActiveClass>& ac = act[w];
+    const int* glob = w ? p->idx_glob2 : p->idx_glob;
+    const int n_all = (int)flat[w].size();
+    const int q = w ? p->hp.warm_power_iters : p->q;
     // one sweep over the momentum: transposed ? Z <- M^T B : Y <- M B
     auto pass = [&](int offB, bool transposed) {
       ProfScope ps(p, PROF_PASS);
-      for (const auto& a : act) {
+      for (const auto& a : ac) {
         const int m = (int)a.c->m, n = (int)a.c->n;
         if (a.c->tensor) { tc_launch_pass(p, *a.c, a.idx, a.cnt, transposed, offB); continue; }
         const int tB = offB == OFF(omega_t);
@@ -451,25 +468,34 @@ sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t 
           launch_gemm(gemm(p, a.idx, OFF(Manc), offB, OFF(Z), n, lp, m, n, lp, lp, 1, 0), a.cnt, s);
       }
     };
-    // range finder: Y = M Omega, Q = orth(Y), q subspace iterations
-    pass(OFF(omega_t), false);
+    // range finder: Y = M S with S the sketch (cold) or [previous V | sketch columns] (warm); Q = orth(Y)
+    if (w) {
+      {
+        ProfScope ps(p, PROF_SMALL);
+        for (const auto& a : ac)
+          launch_warm_start(p->dev_tab, a.idx, a.cnt, (int)a.c->n, lp, p->l, rp, p->rank, p->hp.seed, s);
+      }
+      pass(OFF(Z2), false);
+    } else {
+      pass(OFF(omega_t), false);
+    }
     int curY = OFF(Y);
-    if (p->q == 0) cholqr(p, act, p->idx_glob, n_all, OFF(Y), OFF(Y2), true, false, 2);
-    else { cholqr(p, act, p->idx_glob, n_all, OFF(Y), OFF(Y2), true, false, 1); curY = OFF(Y2); }
-    for (int it = 0; it < p->q; ++it) {
+    if (q == 0) cholqr(p, ac, glob, n_all, OFF(Y), OFF(Y2), true, false, 2);
+    else { cholqr(p, ac, glob, n_all, OFF(Y), OFF(Y2), true, false, 1); curY = OFF(Y2); }   // intermediate basis
+    for (int it = 0; it < q; ++it) {
       pass(curY, true);                                                            // Z = M^T Q
-      cholqr(p, act, p->idx_glob, n_all, OFF(Z), OFF(Z2), false, false, 1);
+      cholqr(p, ac, glob, n_all, OFF(Z), OFF(Z2), false, false, 1);
       pass(OFF(Z2), false);                                                        // Y = M Z
-      if (it == p->q - 1) { cholqr(p, act, p->idx_glob, n_all, OFF(Y), OFF(Y2), true, false, 2); curY = OFF(Y); }
-      else { cholqr(p, act, p->idx_glob, n_all, OFF(Y), OFF(Y2), true, false, 1); curY = OFF(Y2); }
+      if (it == q - 1) { cholqr(p, ac, glob, n_all, OFF(Y), OFF(Y2), true, false, 2); curY = OFF(Y); }
+      else { cholqr(p, ac, glob, n_all, OFF(Y), OFF(Y2), true, false, 1); curY = OFF(Y2); }
     }
     // B^T = M^T Q = Qb R ; SVD of the small factor ; U = Q Ub, V = Qb Wb
     pass(OFF(Y), true);
-    cholqr(p, act, p->idx_glob, n_all, OFF(Z), OFF(Z2), false, true, 2);
+    cholqr(p, ac, glob, n_all, OFF(Z), OFF(Z2), false, true, 2);
     {
       ProfScope ps(p, PROF_SMALL);
-      launch_jacobi(p->dev_tab, p->idx_glob, n_all, lp, rp, p->rank, p->hp.tau_p, s);                 // + Eq. 2
-      for (const auto& a : act) {
+      launch_jacobi(p->dev_tab, glob, n_all, lp, rp, p->rank, p->hp.tau_p, s);                        // + Eq. 2
+      for (const auto& a : ac) {
         const int m = (int)a.c->m, n = (int)a.c->n;
         launch_gemm(gemm(p, a.idx, OFF(Y), OFF(ub), OFF(U), m, rp, lp, lp, rp, rp, 0, 0), a.cnt, s);
         launch_gemm(gemm(p, a.idx, OFF(Z), OFF(wb), OFF(V), n, rp, lp, lp, rp, rp, 0, 0), a.cnt, s);
@@ -477,7 +503,8 @@ sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t 
       }
     }
   }
-  for (int id : flat) p->has_basis[id] = 1;
+  for (int w = 0; w < 2; ++w)
+    for (int id : flat[w]) p->has_basis[id] = 1;
   p->last_tag = step_tag;
   return cuda_ok(cudaGetLastError());
 }

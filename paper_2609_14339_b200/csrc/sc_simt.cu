@@ -325,6 +325,30 @@ void launch_sketch_padded(float* omega, int64_t rows, int lp, int l, uint64_t se
   ++g_kernel_launches;
 }
 
+// Start block of a warm range finder: Z2[:, :rank] = previous V, Z2[:, rank:l] = sketch columns, rest zero.
+__global__ void warm_start_kernel(const MatDev* tab, const int* idx, int n, int lp, int l, int rp, int rank,
+                                  uint64_t seed) {
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x, tot = (int64_t)n * lp;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < tot; e += stride) {
+    const int64_t j = e / lp;
+    const int c = (int)(e % lp);
+    float v = 0.f;
+    if (c < rank) v = md.V[(size_t)j * rp + c];
+    else if (c < l) v = sketch_entry(seed, (uint64_t)j, (uint64_t)c);
+    md.Z2[e] = v;
+  }
+}
+
+void launch_warm_start(const MatDev* tab, const int* idx, int count, int n, int lp, int l, int rp, int rank,
+                       uint64_t seed, cudaStream_t s) {
+  if (count <= 0 || lp <= 0) return;
+  const int64_t tot = (int64_t)n * lp;
+  const int blocks = (int)((tot + 255) / 256 < 592 ? (tot + 255) / 256 : 592);
+  warm_start_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, n, lp, l, rp, rank, seed);
+  ++g_kernel_launches;
+}
+
 void launch_sketch_rowmajor(float* omega, int64_t rows, int width, uint64_t seed, cudaStream_t s) {
   const int64_t tot = rows * width;
   if (tot <= 0) return;

@@ -39,6 +39,8 @@ class Case:
     t0: int = 100                  # optimizer step count used with a warmed state
     engine: int = 0
     n_anchor: int = 1              # anchor arrivals before the step
+    warm: bool = False             # warm-started range finder from the second arrival on
+    q_warm: int = 0
     extra: dict = field(default_factory=dict)
 
 
@@ -81,6 +83,7 @@ def make_plan(case: Case, torch, device="cuda:0"):
                             grads_prescaled=int(case.prescaled),
                             grad_dtype=sc.SC_DTYPE_BF16 if case.dtype == "bf16" else sc.SC_DTYPE_FP32,
                             sketch_width=case.l, power_iters=case.q, engine=case.engine, collect_stats=1,
+                            warm_start=int(case.warm), warm_power_iters=case.q_warm,
                             seed=case.seed)
     return sc.Plan(case.shapes, case.rank, case.keep, hp, device=device)
 
@@ -138,7 +141,8 @@ class OracleRun:
                 Ga = gen.stored_to_f64(inputs["anchors"][i][a], case.dtype)
                 if isinstance(basis_mode, str) and basis_mode == "mirror":
                     Om = so.rademacher_sketch(case.seed, 0, nn, l) if case.rank > 0 else None
-                    so.anchor_update(st, Ga, hp, case.rank, mode="mirror", Omega=Om, q=case.q)
+                    so.anchor_update(st, Ga, hp, case.rank, mode="mirror", Omega=Om, q=case.q, warm=case.warm,
+                                     q_warm=case.q_warm)
                 elif isinstance(basis_mode, str):
                     so.anchor_update(st, Ga, hp, case.rank, mode="exact")
                 else:

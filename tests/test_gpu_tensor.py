@@ -107,3 +107,26 @@ def test_host_gradient_entry_point_matches_device_path(torch):
         outs.append((W, m, v))
     for a, b in zip(outs[0], outs[1]):
         assert all(torch.equal(x, y) for x, y in zip(a, b))
+
+
+@pytest.mark.parametrize("engine", [0, 1])
+def test_warm_started_range_finder(torch, engine):
+    """From the second anchor arrival on the range finder starts from the previous right basis (two sweeps per
+    arrival); the oracle's MIRROR mode does the same."""
+    case = Case(shapes=[(384, 512), (256, 384), (384, 512)], rank=16, l=24, tokens=256, keep=0.25, planted=8, seed=8,
+                tau_p=60.0, n_anchor=3, warm=True, q_warm=0, engine=engine)
+    inp = make_inputs(case)
+    g = GpuRun(case, inp, torch)
+    assert g.dev_status == 0
+    o = OracleRun(case, inp, "mirror")
+    eb = compare_basis(g, o)
+    assert eb["M"] < 1e-6 and max(eb["PU"], eb["PV"], eb["s"]) < TOL, eb
+    es = compare_step(g, o)
+    assert max(es["gproj"], es["m"], es["v"], es["dW"]) < TOL, es
+    # and it is a better basis than a cold start with the same two sweeps: closer to the exact truncated SVD
+    cold = Case(**{**case.__dict__, "warm": False, "q": 0})
+    oc = OracleRun(cold, inp, "mirror")
+    oe = OracleRun(case, inp, "exact")
+    d_warm = so.projector_distance(o.states[0].V, oe.states[0].V)
+    d_cold = so.projector_distance(oc.states[0].V, oe.states[0].V)
+    assert d_warm < d_cold

@@ -349,3 +349,22 @@ def test_projector_distance_matches_explicit_projectors():
     if True:
         Pa, Pb = A @ A.T, B @ B.T
         assert abs(so.projector_distance(A, B) - np.linalg.norm(Pa - Pb) / np.sqrt(12)) < 1e-12
+
+
+def test_mirror_warm_start_reduces_to_cold_on_first_arrival_and_improves_later():
+    m, n, r = 70, 50, 4
+    A, _ = np.linalg.qr(RNG.standard_normal((m, n)))
+    B, _ = np.linalg.qr(RNG.standard_normal((n, n)))
+    s = np.concatenate([np.linspace(10, 7, r), np.linspace(2.0, 0.1, n - r)])
+    G1 = (A * s) @ B.T
+    hp = so.Hyper(beta_anc=0.5)
+    Om = so.rademacher_sketch(3, 0, n, r)
+    cold = so.anchor_update(so.new_state(m, n), G1, hp, r, mode="mirror", Omega=Om, q=0)
+    warm = so.anchor_update(so.new_state(m, n), G1, hp, r, mode="mirror", Omega=Om, q=0, warm=True)
+    assert np.array_equal(cold.V, warm.V)                              # no basis yet: same as a cold start
+    Ve = so.truncate(*so.svd_exact(G1), r)[2]
+    errs = []
+    for _ in range(6):                                                 # same gradient again and again: M -> G1
+        so.anchor_update(warm, G1, hp, r, mode="mirror", Omega=Om, q=0, warm=True)
+        errs.append(so.projector_distance(warm.V, Ve))
+    assert errs[-1] < 1e-2 * errs[0] and all(b <= a * 1.0001 for a, b in zip(errs, errs[1:]))
