@@ -228,6 +228,19 @@ SC_API sc_status sc_get_stats(sc_plan* plan, sc_mat_stats* stats, float* clip);
 /* Wait for the plan's stream and return the latched device status (SC_OK, SC_ERR_TIMEOUT, SC_ERR_NONFINITE), then clear it. */
 SC_API sc_status sc_get_device_status(sc_plan* plan);
 
+/* Checkpoint / resume. The blob holds, for every matrix, the anchor momentum, the cached basis (U, s, V, d), whether a
+ * basis exists, and the last accepted step tag; AdamW state and weights stay with the caller. host_buf is HOST memory
+ * of at least sc_state_bytes(plan) bytes. Both calls wait for the plan's stream. Import needs a plan created with the
+ * same shapes and rank (SC_ERR_SHAPE otherwise); a step after import continues bit-identically. */
+SC_API size_t sc_state_bytes(const sc_plan* plan);
+SC_API sc_status sc_state_export(sc_plan* plan, void* host_buf, size_t bytes);
+SC_API sc_status sc_state_import(sc_plan* plan, const void* host_buf, size_t bytes);
+
+/* Test hook for the failure path of the device-side bounded waits: queues one tiny kernel that waits on a barrier
+ * nothing will ever signal, gives up after max_polls polls (1..2^20, i.e. at most a few milliseconds), latches the
+ * time-out bit and returns normally. sc_get_device_status then reports SC_ERR_TIMEOUT once. Nothing hangs or traps. */
+SC_API sc_status sc_debug_wait_probe(sc_plan* plan, int max_polls);
+
 /* Device-time profile by phase of the method. Categories:
  *   0 anchor EMA (Eq. 1)            1 basis build, passes over the momentum     2 basis build, small factorisations
  *   3 projection T = G V            4 r x r filter, C^T, norms                  5 fused correction + AdamW update */

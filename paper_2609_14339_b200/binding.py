@@ -86,6 +86,10 @@ EXPORTS = {
     "sc_set_debug_gproj_out": (C.c_int, [_VP, _VPP]),
     "sc_get_stats": (C.c_int, [_VP, C.POINTER(MatStats), C.POINTER(C.c_float)]),
     "sc_get_device_status": (C.c_int, [_VP]),
+    "sc_state_bytes": (C.c_size_t, [_VP]),
+    "sc_state_export": (C.c_int, [_VP, _VP, C.c_size_t]),
+    "sc_state_import": (C.c_int, [_VP, _VP, C.c_size_t]),
+    "sc_debug_wait_probe": (C.c_int, [_VP, C.c_int]),
     "sc_set_profiling": (C.c_int, [_VP, C.c_int]),
     "sc_get_profile": (C.c_int, [_VP, C.POINTER(Profile)]),
     "sc_kernel_launch_count": (C.c_int64, []),
@@ -315,6 +319,19 @@ class Plan:
         tag, k = C.c_int64(), C.c_int()
         _check(self.lib.sc_get_anchor_info(self.handle, C.byref(tag), C.byref(k)), "sc_get_anchor_info")
         return tag.value, k.value
+
+    def state_export(self):
+        """Anchor momentum + cached basis of every matrix as one bytes-like host buffer (a ctypes array)."""
+        n = self.lib.sc_state_bytes(self.handle)
+        buf = (C.c_char * n)()
+        _check(self.lib.sc_state_export(self.handle, buf, n), "sc_state_export")
+        return buf
+
+    def state_import(self, buf):
+        _check(self.lib.sc_state_import(self.handle, buf, len(buf)), "sc_state_import")
+
+    def debug_wait_probe(self, max_polls: int = 4096):
+        _check(self.lib.sc_debug_wait_probe(self.handle, int(max_polls)), "sc_debug_wait_probe")
 
     def set_profiling(self, on: bool):
         _check(self.lib.sc_set_profiling(self.handle, int(bool(on))), "sc_set_profiling")

@@ -177,7 +177,7 @@ void launch_filter_weights(const MatDev* tab, const int* idx, int count, int rp,
 void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int n, int rp, int rk, cudaStream_t s);
 void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, cudaStream_t s);
 void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, float coef, float scale, float alpha,
-               cudaStream_t s);
+               unsigned* status, cudaStream_t s);
 void launch_split_ct(const MatDev* tab, const int* idx, int count, int n, int rp, int rk, cudaStream_t s);
 void launch_clip(const MatDev* tab, int n_mats, float max_norm, float* clip, cudaStream_t s);
 void launch_pad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, int cols_dst, cudaStream_t s);
@@ -191,6 +191,7 @@ sc_status tc_init();   // resolves the driver entry point for tensor-map encodin
 sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_call_part);
 sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count);   // T = G V
 sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc);
+sc_status tc_launch_wait_probe(sc_plan* p, int max_polls);
 sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, bool transposed, int b_field_off);
 
 }  // namespace sc

@@ -588,7 +588,7 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
     ProfScope ps(p, PROF_FILTER);
     if (rp > 0) launch_atb(p->dev_tab, idx, cnt, OFF(U), OFF(T), OFF(xpart), OFF(X), m, rp, rp, rp, rp, s);  // X = U^T T
     if (want_norm) launch_sqnorm(p->dev_tab, idx, cnt, (int64_t)m * n, g_bf16, s);
-    launch_xs(p->dev_tab, idx, cnt, rp, p->rank, 0.f, scale, hp.alpha, s);                             // D X D
+    launch_xs(p->dev_tab, idx, cnt, rp, p->rank, 0.f, scale, hp.alpha, p->status_dev, s);                             // D X D
     if (rp > 0) {
       launch_gemm(gemm(p, idx, OFF(V), OFF(Xs), OFF(Ct), n, rp, rp, rp, rp, rp, 0, 1), cnt, s);      // C^T = V Xs^T
       if (c.tensor) launch_split_ct(p->dev_tab, idx, cnt, n, rp, p->rk, s);
@@ -761,6 +761,89 @@ sc_status sc_get_anchor_info(sc_plan* p, int64_t* last_tag, int* n_with_basis) {
     *n_with_basis = k;
   }
   return SC_OK;
+}
+
+// ---- checkpoint / resume: anchor momentum and cached basis of every matrix as one host blob --------------
+namespace {
+struct StateHeader {
+  uint32_t magic, version;
+  int32_t n_mats, rank, rp, pad;
+  int64_t last_tag;
+};
+constexpr uint32_t kStateMagic = 0x53435354u;   // "SCST"
+
+size_t state_bytes(const sc_plan* p) {
+  size_t b = sizeof(StateHeader) + align_up((size_t)p->n_mats, 16);
+  for (int i = 0; i < p->n_mats; ++i) {
+    const size_t m = (size_t)p->shapes[i].rows, n = (size_t)p->shapes[i].cols;
+    b += (m * n + (m + n + 2) * (size_t)p->rp) * sizeof(float);
+  }
+  return b;
+}
+}  // namespace
+
+size_t sc_state_bytes(const sc_plan* p) { return p ? state_bytes(p) : 0; }
+
+sc_status sc_state_export(sc_plan* p, void* host_buf, size_t bytes) {
+  if (!p || !host_buf) return SC_ERR_INVALID_ARG;
+  if (bytes < state_bytes(p)) return SC_ERR_WORKSPACE;
+  char* out = static_cast<char*>(host_buf);
+  StateHeader h{kStateMagic, 1u, p->n_mats, p->rank, p->rp, 0, p->last_tag};
+  memcpy(out, &h, sizeof(h));
+  char* flags = out + sizeof(h);
+  memset(flags, 0, align_up((size_t)p->n_mats, 16));
+  for (int i = 0; i < p->n_mats; ++i) flags[i] = p->has_basis[i];
+  char* cur = flags + align_up((size_t)p->n_mats, 16);
+  auto pull = [&](const float* src, size_t count) {
+    const bool ok = count == 0 ||
+                    cudaMemcpyAsync(cur, src, count * sizeof(float), cudaMemcpyDeviceToHost, p->stream) == cudaSuccess;
+    cur += count * sizeof(float);
+    return ok;
+  };
+  for (int i = 0; i < p->n_mats; ++i) {
+    const MatDev& md = p->host_tab[i];
+    const size_t m = (size_t)md.m, n = (size_t)md.n, rp = (size_t)p->rp;
+    if (!pull(md.Manc, m * n) || !pull(md.U, m * rp) || !pull(md.V, n * rp) || !pull(md.sv, rp) || !pull(md.d, rp))
+      return SC_ERR_CUDA;
+  }
+  return cuda_ok(cudaStreamSynchronize(p->stream));
+}
+
+sc_status sc_state_import(sc_plan* p, const void* host_buf, size_t bytes) {
+  if (!p || !host_buf) return SC_ERR_INVALID_ARG;
+  if (bytes < state_bytes(p)) return SC_ERR_WORKSPACE;
+  const char* in = static_cast<const char*>(host_buf);
+  StateHeader h;
+  memcpy(&h, in, sizeof(h));
+  if (h.magic != kStateMagic || h.version != 1u) return SC_ERR_INVALID_ARG;
+  if (h.n_mats != p->n_mats || h.rank != p->rank || h.rp != p->rp) return SC_ERR_SHAPE;
+  sc_status st = upload_table(p);
+  if (st != SC_OK) return st;
+  const char* flags = in + sizeof(h);
+  const char* cur = flags + align_up((size_t)p->n_mats, 16);
+  auto push = [&](float* dst, size_t count) {
+    const bool ok = count == 0 ||
+                    cudaMemcpyAsync(dst, cur, count * sizeof(float), cudaMemcpyHostToDevice, p->stream) == cudaSuccess;
+    cur += count * sizeof(float);
+    return ok;
+  };
+  for (int i = 0; i < p->n_mats; ++i) {
+    const MatDev& md = p->host_tab[i];
+    const size_t m = (size_t)md.m, n = (size_t)md.n, rp = (size_t)p->rp;
+    if (!push(md.Manc, m * n) || !push(md.U, m * rp) || !push(md.V, n * rp) || !push(md.sv, rp) || !push(md.d, rp))
+      return SC_ERR_CUDA;
+  }
+  for (auto& c : p->classes) refresh_operands(p, c, c.idx_all, (int)c.mats.size());
+  // the copies above read caller memory: finish them before returning
+  if (cudaStreamSynchronize(p->stream) != cudaSuccess) return SC_ERR_CUDA;
+  for (int i = 0; i < p->n_mats; ++i) p->has_basis[i] = flags[i];
+  p->last_tag = h.last_tag;
+  return cuda_ok(cudaGetLastError());
+}
+
+sc_status sc_debug_wait_probe(sc_plan* p, int max_polls) {
+  if (!p || max_polls < 1 || max_polls > (1 << 20)) return SC_ERR_INVALID_ARG;
+  return tc_launch_wait_probe(p, max_polls);
 }
 
 sc_status sc_set_profiling(sc_plan* p, int on) {

@@ -629,7 +629,7 @@ void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, 
 //   stats[0] = ||g||^2, stats[1] = ||X||^2 (scaled), stats[2] = ||G_proj||^2 (closed form), stats[3] = sum d^2
 // =====================================================================================================
 __global__ void __launch_bounds__(256) xs_kernel(const MatDev* tab, const int* idx, int rp, int rank, float coef,
-                                                 float scale, float alpha) {
+                                                 float scale, float alpha, unsigned* status) {
   __shared__ float red[3][8];
   const MatDev& md = tab[idx[blockIdx.x]];
   float sx = 0.f, s1 = 0.f, s2 = 0.f;
@@ -656,13 +656,15 @@ __global__ void __launch_bounds__(256) xs_kernel(const MatDev* tab, const int* i
     md.stats[1] = tx;
     md.stats[2] = alpha * alpha * gg + 2.f * alpha * (1.f - alpha) * t1 + (1.f - alpha) * (1.f - alpha) * t2;
     md.stats[3] = re;
+    // a NaN or Inf anywhere in the gradient reaches X = U^T G V (or ||g||^2): latch it for the host
+    if (!isfinite(tx) || !isfinite(gg)) atomicOr(status, kDevNonfinite);
   }
 }
 
 void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, float coef, float scale, float alpha,
-               cudaStream_t s) {
+               unsigned* status, cudaStream_t s) {
   if (count <= 0) return;
-  xs_kernel<<<count, 256, 0, s>>>(tab, idx, rp, rank, coef, scale, alpha);
+  xs_kernel<<<count, 256, 0, s>>>(tab, idx, rp, rank, coef, scale, alpha, status);
   ++g_kernel_launches;
 }
 

@@ -631,6 +631,19 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
   if (warp == 1) tmem_dealloc(tmem_base, 2 * kTileN);
 }
 
+// A wait that nothing will ever satisfy, with a caller-chosen small poll limit: exercises the path by which a
+// bounded wait reports through the status word (the block gives up, latches the bit and returns normally).
+__global__ void wait_probe_kernel(int max_polls, unsigned* status) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    fence_barrier_init();
+    bool done = false;
+    for (int it = 0; it < max_polls && !done; ++it) done = mbar_try_wait(&bar, 0);
+    if (!done) atomicOr(status, kDevTimeout);
+  }
+}
+
 // ---------------------------------------------------------------------------------------------- host
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -759,6 +772,12 @@ sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count
   dim3 grid((m + 127) / 128, c.ksplit, count);
   project_kernel<<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), m, n, rp,
                                                  cps, stages, cols, p->status_dev);
+  ++g_kernel_launches;
+  return cuda_ok(cudaGetLastError());
+}
+
+sc_status tc_launch_wait_probe(sc_plan* p, int max_polls) {
+  wait_probe_kernel<<<1, 32, 0, p->stream>>>(max_polls, p->status_dev);
   ++g_kernel_launches;
   return cuda_ok(cudaGetLastError());
 }
