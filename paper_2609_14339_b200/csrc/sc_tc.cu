@@ -134,7 +134,7 @@ constexpr int kTileBytes = 128 * 128;   // 128 rows x 64 bf16
 // T = G V  (per 128-row tile of G and per K slice).  Warp 0: TMA producer. Warp 1: MMA issuer (owns TMEM).
 // Warps 2-5: epilogue, TMEM -> registers -> global.
 // =====================================================================================================
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(192, 2)
 project_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const CUtensorMap* __restrict__ maps,
                int m, int n, int rp, int cps, int stages, uint32_t tmem_cols, unsigned* status) {
   extern __shared__ uint8_t smem_raw[];
@@ -261,7 +261,7 @@ constexpr int kPassK = 32;                       // K per stage
 constexpr int kAtomBytes = kPassK * 128;         // one MN-major atom column: 32 K-rows x 128 bytes
 
 template <bool TRANS>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(192, 2)
 pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const CUtensorMap* __restrict__ maps,
             int b_map, int out_off, int rows_out, int kdim, int lp, int stages, uint32_t tmem_cols, unsigned* status) {
   extern __shared__ uint8_t smem_raw[];
@@ -755,11 +755,17 @@ sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_
   return SC_OK;
 }
 
-static int project_stages(int rp) {
-  const int stage_bytes = kTileBytes + 2 * rp * 128;
-  int s = (200 * 1024) / stage_bytes;
-  return s > 6 ? 6 : (s < 2 ? 2 : s);
+// Two blocks per SM when three stages of each fit (their prologues and epilogues then overlap the other block's
+// streaming); otherwise one block with as many stages as fit.
+static int stages_for(int stage_bytes, int max_one_block) {
+  if (3 * stage_bytes + 2048 <= 110 * 1024) {
+    const int s = (110 * 1024 - 2048) / stage_bytes;
+    return s > 4 ? 4 : s;
+  }
+  const int s = (200 * 1024) / stage_bytes;
+  return s > max_one_block ? max_one_block : (s < 2 ? 2 : s);
 }
+static int project_stages(int rp) { return stages_for(kTileBytes + 2 * rp * 128, 6); }
 
 sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count) {
   const int rp = p->rp, m = (int)c.m, n = (int)c.n;
@@ -786,8 +792,7 @@ sc_status tc_launch_wait_probe(sc_plan* p, int max_polls) {
 sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, bool transposed, int b_field_off) {
   const int lp = p->lp, m = (int)c.m, n = (int)c.n;
   const int stage_bytes = kTileBytes + (lp / 32) * kAtomBytes;
-  int stages = (200 * 1024) / stage_bytes;
-  stages = stages > 8 ? 8 : (stages < 2 ? 2 : stages);
+  const int stages = stages_for(stage_bytes, 8);
   const size_t smem = (size_t)stages * stage_bytes + 1024 + 256;
   uint32_t cols = 32;
   while ((int)cols < lp) cols <<= 1;
