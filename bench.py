@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--workload", default="llama8b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="config 4: one 14336x4096 matrix, rank x keep grid; prints one JSON line with a 'cells' list")
     return ap.parse_args()
 
 
@@ -333,8 +335,73 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Config 4: one 14336 x 4096 bf16 matrix, 4096 tokens, rank in {8..256} x keep in {0.05..0.5}, planted rank r/2
+    at SNR 1. Per cell: steady step time, refresh time and fraction of the HBM/BF16 roofline."""
+    import torch
+    import paper_2609_14339_b200 as sc
+    from paper_2609_14339_b200 import build as _build
+    from synth import generator as gen
+    _build.build()
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    peaks = measured_peaks()
+    m, n, T = 14336, 4096, 4096
+    cells = []
+    g = torch.Generator(device=device); g.manual_seed(5)
+    W = torch.randn((m, n), generator=g, device=device) * 0.02
+    M1 = torch.randn((m, n), generator=g, device=device) * 10.0
+    M2 = torch.rand((m, n), generator=g, device=device) * 4000.0 + 100.0
+    Wb = torch.empty((m, n), device=device, dtype=torch.bfloat16)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)      # larger than L2
+    for keep in (0.05, 0.1, 0.25, 0.5):
+        for r in (8, 16, 32, 64, 128, 256):
+            spec = gen.GradSpec(m=m, n=n, tokens=T, keep=keep, planted_rank=max(r // 2, 1), snr=1.0, seed=0)
+            G = gen.torch_gradients(spec, 1, device, torch.bfloat16)
+            Ga = gen.torch_gradients(spec, 0, device, torch.bfloat16, anchor=True)
+            plan = sc.Plan([(m, n)], r, keep, sc.Hparams.default(power_iters=1, warm_start=1), device=device)
+            plan.anchor_update([Ga], 0)
+            for i in range(args.warmup):
+                plan.correct_and_step([G], [W], [M1], [M2], 100 + i, params_bf16=[Wb])
+            steady, refresh = [], []
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            for i in range(args.steps):
+                flush.zero_()                                              # evict the state from L2 between iterations
+                ev[0].record()
+                plan.anchor_update([Ga], 1 + i)
+                ev[1].record()
+                flush.zero_()
+                torch.cuda.synchronize()
+                ev[1].record()
+                plan.correct_and_step([G], [W], [M1], [M2], 200 + i, params_bf16=[Wb])
+                ev[2].record()
+                torch.cuda.synchronize()
+                steady.append(ev[1].elapsed_time(ev[2]))
+            for i in range(args.steps):
+                flush.zero_()
+                torch.cuda.synchronize()
+                ev[0].record()
+                plan.anchor_update([Ga], 100 + i)
+                ev[1].record()
+                torch.cuda.synchronize()
+                refresh.append(ev[0].elapsed_time(ev[1]))
+            ms = statistics.median(steady)
+            roof = max(m * n * BYTES_PER_ELEM_STEADY / (peaks["hbm_gbs"] * 1e9), m * n * 4.0 * r / (peaks["bf16_tflops"] * 1e12)) * 1e3
+            cells.append({"rank": r, "keep": keep, "steady_step_ms": ms, "roofline_ms": roof, "roofline_frac": roof / ms,
+                          "refresh_ms": statistics.median(refresh), "gradient_gbs": m * n * 2 / (ms * 1e-3) / 1e9})
+            plan.close()
+            del plan, G, Ga
+    print(json.dumps({"metric": "config 4 sweep: steady step ms and roofline fraction per (rank, keep) cell",
+                      "workload": "one 14336x4096 bf16 matrix, 4096 tokens", "steps": args.steps, "warmup": args.warmup,
+                      "l2": "256 MB buffer rewritten between timed iterations", "peak_source": peaks["source"],
+                      "cells": cells}), flush=True)
+
+
 def main():
     args = parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:
