@@ -17,7 +17,7 @@ typedef __nv_bfloat16 bf16;
 constexpr int kMaxRank = 256;
 constexpr int kStatsFloats = 8;        // per-matrix statistics slot
 constexpr int kSqnormBlocks = 128;     // partial sums of ||G||^2 per matrix (fixed-order reduction)
-constexpr int kAtbMaxSplits = 16;      // row slices of the A^T B kernel (fixed-order two-stage reduction)
+constexpr int kAtbMaxSplits = 64;      // row slices of the A^T B kernel (fixed-order two-stage reduction)
 constexpr int kStagingSlots = 4;       // ring of pinned upload buffers for the per-call pointer table
 
 // Device status word bits (latched, read by sc_get_device_status).
@@ -88,6 +88,7 @@ struct ShapeClass {
   int* idx_dyn2 = nullptr; // device: subset list written per call (anchor arrivals, warm starts)
   bool tensor = false;     // served by the tcgen05 kernels
   int ksplit = 1;
+  int split_m = 1, split_n = 1;   // row slices of A^T B products over m / n rows (fixed at plan creation)
   void* tmaps = nullptr;   // device: per-instance tensor maps (tensor engine only)
 };
 
@@ -158,11 +159,12 @@ struct GemmArgs {
   int transA, transB;
   int a_bf16;              // A holds bf16 (gradients) instead of fp32
   float alpha;
+  int offHi, offLo, ld_split;   // when offHi != 0: also write the result as a bf16 hi/lo pair with this row stride
 };
 void launch_gemm(const GemmArgs& a, int count, cudaStream_t s);
-int atb_splits(int rows);
+int atb_splits(int rows, int count);
 void launch_atb(const MatDev* tab, const int* idx, int count, int offA, int offB, int offPart, int offOut, int rows,
-                int ca, int cb, int lda, int ldb, cudaStream_t s);
+                int ca, int cb, int lda, int ldb, int nsplit, cudaStream_t s, int b_slices = 1, bool sum_here = true);
 void launch_epilogue_simt(const MatDev* tab, const int* idx, int count, int m, int n, int rp, int g_bf16,
                           const StepScalars& sc, const float* clip, cudaStream_t s);
 void launch_ema(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, float beta, cudaStream_t s);
@@ -176,7 +178,7 @@ void launch_jacobi(const MatDev* tab, const int* idx, int count, int lp, int rp,
 void launch_filter_weights(const MatDev* tab, const int* idx, int count, int rp, int rank, float tau_p, cudaStream_t s);
 void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int n, int rp, int rk, cudaStream_t s);
 void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, cudaStream_t s);
-void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, float coef, float scale, float alpha,
+void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, int x_slices, float scale, float alpha,
                unsigned* status, cudaStream_t s);
 void launch_split_ct(const MatDev* tab, const int* idx, int count, int n, int rp, int rk, cudaStream_t s);
 void launch_clip(const MatDev* tab, int n_mats, float max_norm, float* clip, cudaStream_t s);

@@ -126,7 +126,7 @@ size_t layout(sc_plan* p, bool assign) {
     md.Xs = cv.take<float>((size_t)rp * rp);
     md.T = cv.take<float>((size_t)c.ksplit * m * rp);
     md.Ct = cv.take<float>(n * rp);
-    md.xpart = cv.take<float>((size_t)atb_splits((int)m) * rp * rp);
+    md.xpart = cv.take<float>((size_t)c.split_m * rp * rp);
     md.sqpart = cv.take<float>(kSqnormBlocks);
     if (c.tensor) {
       md.Uhi = cv.take<bf16>(m * rk); md.Ulo = cv.take<bf16>(m * rk);
@@ -146,7 +146,8 @@ size_t layout(sc_plan* p, bool assign) {
     float* Y = cv.take<float>(m * lp); float* Y2 = cv.take<float>(m * lp);
     float* Z = cv.take<float>(n * lp); float* Z2 = cv.take<float>(n * lp);
     float* gram = cv.take<float>((size_t)lp * lp); float* rmat = cv.take<float>((size_t)lp * lp);
-    float* gpart = cv.take<float>((size_t)atb_splits((int)std::max(m, n)) * lp * lp);
+    const ShapeClass& cls = p->classes[p->class_of[i]];
+    float* gpart = cv.take<float>((size_t)std::max(cls.split_m, cls.split_n) * lp * lp);
     float* rmat2 = cv.take<float>((size_t)lp * lp); float* rinv = cv.take<float>((size_t)lp * lp);
     float* racc = cv.take<float>((size_t)lp * lp); float* jk = cv.take<float>((size_t)lp * lp);
     float* jv = cv.take<float>((size_t)lp * lp);
@@ -172,6 +173,8 @@ void fill_plan_basics(sc_plan* p, const sc_shape* shapes, int n_mats, int rank, 
     c.tensor = hp->engine == SC_ENGINE_AUTO && hp->grad_dtype == SC_DTYPE_BF16 && rank > 0 &&
                tc_shape_supported(c.m, c.n, d.rp);
     c.ksplit = c.tensor ? choose_ksplit(c) : 1;
+    c.split_m = atb_splits((int)c.m, (int)c.mats.size());
+    c.split_n = atb_splits((int)c.n, (int)c.mats.size());
     p->tensor_any = p->tensor_any || c.tensor;
   }
 }
@@ -243,7 +246,7 @@ void cholqr(sc_plan* p, const std::vector<ActiveClass>& act, const int* idx_all,
     const int src = round == 0 ? offY : offTmp, dst = round == 0 ? offTmp : offY;
     for (const auto& a : act)
       launch_atb(p->dev_tab, a.idx, a.cnt, src, src, OFF(gpart), OFF(gram), (int)(left ? a.c->m : a.c->n), lp, lp, lp,
-                 lp, s);
+                 lp, left ? a.c->split_m : a.c->split_n, s);
     launch_chol(p->dev_tab, idx_all, n_all, lp, round == 0 ? OFF(rmat) : OFF(rmat2), s);
     for (const auto& a : act)
       launch_gemm(gemm(p, a.idx, src, OFF(rinv), dst, (int)(left ? a.c->m : a.c->n), lp, lp, lp, lp, lp, 0, 0), a.cnt, s);
@@ -578,20 +581,22 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
     if (rp > 0) {
       ProfScope ps(p, PROF_PROJECT);
       if (c.tensor) {
-        sc_status e = tc_launch_project(p, c, idx, cnt);                                                  // T = G V
+        sc_status e = tc_launch_project(p, c, idx, cnt);                     // T = G V, as c.ksplit partials over K
         if (e != SC_OK) return e;
-        launch_reduce_partials(p->dev_tab, idx, cnt, (int64_t)m * rp, c.ksplit, s);
       } else {
         launch_gemm(gemm(p, idx, OFF(G), OFF(V), OFF(T), m, rp, n, n, rp, rp, 0, 0, g_bf16), cnt, s);
       }
     }
     ProfScope ps(p, PROF_FILTER);
-    if (rp > 0) launch_atb(p->dev_tab, idx, cnt, OFF(U), OFF(T), OFF(xpart), OFF(X), m, rp, rp, rp, rp, s);  // X = U^T T
+    // X = U^T T as row-slice partials (the K-slice partials of T are added on the way in); xs_kernel adds them up
+    if (rp > 0)
+      launch_atb(p->dev_tab, idx, cnt, OFF(U), OFF(T), OFF(xpart), OFF(X), m, rp, rp, rp, rp, c.split_m, s, c.ksplit, false);
     if (want_norm) launch_sqnorm(p->dev_tab, idx, cnt, (int64_t)m * n, g_bf16, s);
-    launch_xs(p->dev_tab, idx, cnt, rp, p->rank, 0.f, scale, hp.alpha, p->status_dev, s);                             // D X D
+    launch_xs(p->dev_tab, idx, cnt, rp, p->rank, rp > 0 ? c.split_m : 0, scale, hp.alpha, p->status_dev, s);   // D X D
     if (rp > 0) {
-      launch_gemm(gemm(p, idx, OFF(V), OFF(Xs), OFF(Ct), n, rp, rp, rp, rp, rp, 0, 1), cnt, s);      // C^T = V Xs^T
-      if (c.tensor) launch_split_ct(p->dev_tab, idx, cnt, n, rp, p->rk, s);
+      GemmArgs ga = gemm(p, idx, OFF(V), OFF(Xs), OFF(Ct), n, rp, rp, rp, rp, rp, 0, 1);             // C^T = V Xs^T
+      if (c.tensor) { ga.offHi = OFF(Cthi); ga.offLo = OFF(Ctlo); ga.ld_split = p->rk; }
+      launch_gemm(ga, cnt, s);
     }
     return SC_OK;
   };
@@ -687,7 +692,12 @@ sc_status sc_export_projection(sc_plan* p, int mat, void* T_dev, void* X_dev) {
   const MatDev& md = p->host_tab[mat];
   const int r = p->rank, rp = p->rp;
   if (r == 0) return SC_OK;
-  if (T_dev) launch_unpad_copy(static_cast<float*>(T_dev), r, md.T, rp, md.m, r, p->stream);
+  if (T_dev) {
+    // the tensor-core projection leaves K-slice partials: add them up first (the next step rewrites them anyway)
+    ShapeClass& c = p->classes[p->class_of[mat]];
+    launch_reduce_partials(p->dev_tab, c.idx_all + p->inst_of[mat], 1, (int64_t)md.m * rp, c.ksplit, p->stream);
+    launch_unpad_copy(static_cast<float*>(T_dev), r, md.T, rp, md.m, r, p->stream);
+  }
   if (X_dev) launch_unpad_copy(static_cast<float*>(X_dev), r, md.X, rp, r, r, p->stream);
   return cuda_ok(cudaGetLastError());
 }

@@ -13,6 +13,11 @@ __device__ __forceinline__ T* field(const MatDev& md, int off) {
   return *reinterpret_cast<T* const*>(reinterpret_cast<const char*>(&md) + off);
 }
 
+__device__ __forceinline__ void split2(float x, bf16& hi, bf16& lo) {
+  hi = __float2bfloat16_rn(x);
+  lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -86,7 +91,16 @@ __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs a, EpiAdamW epi) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int gc = col0 + tx * 4 + j;
-        if (gc < a.N) C[(size_t)gr * a.ldc + gc] = a.alpha * acc[i][j];
+        if (gc < a.N) {
+          const float val = a.alpha * acc[i][j];
+          C[(size_t)gr * a.ldc + gc] = val;
+          if (a.offHi) {   // also the bf16 hi/lo pair the tensor-core kernels read
+            bf16 hi, lo;
+            split2(val, hi, lo);
+            field<bf16>(md, a.offHi)[(size_t)gr * a.ld_split + gc] = hi;
+            field<bf16>(md, a.offLo)[(size_t)gr * a.ld_split + gc] = lo;
+          }
+        }
       }
     }
   } else {
@@ -149,7 +163,8 @@ void launch_epilogue_simt(const MatDev* tab, const int* idx, int count, int m, i
 // =====================================================================================================
 template <int MT>
 __global__ void __launch_bounds__(256) atb_kernel(const MatDev* tab, const int* idx, int offA, int offB, int offPart,
-                                                  int rows, int ca, int cb, int lda, int ldb, int rows_per_split) {
+                                                  int rows, int ca, int cb, int lda, int ldb, int rows_per_split,
+                                                  int b_slices) {
   constexpr int TS = 16 * MT;          // output tile edge
   __shared__ __align__(16) float As[32][TS + 4];
   __shared__ __align__(16) float Bs[32][TS + 4];
@@ -167,7 +182,14 @@ __global__ void __launch_bounds__(256) atb_kernel(const MatDev* tab, const int* 
       const int rr = e / TS, c = e % TS;
       const int gr = r0 + rr;
       As[rr][c] = (gr < r_hi && i0 + c < ca) ? A[(size_t)gr * lda + i0 + c] : 0.f;
-      Bs[rr][c] = (gr < r_hi && j0 + c < cb) ? B[(size_t)gr * ldb + j0 + c] : 0.f;
+      float bval = 0.f;
+      if (gr < r_hi && j0 + c < cb) {
+        // B may arrive as several K-slice partials of the projection (fixed-order sum)
+        const size_t o = (size_t)gr * ldb + j0 + c;
+        bval = B[o];
+        for (int sl = 1; sl < b_slices; ++sl) bval += B[(size_t)sl * rows * ldb + o];
+      }
+      Bs[rr][c] = bval;
     }
     __syncthreads();
 #pragma unroll 8
@@ -205,27 +227,34 @@ __global__ void __launch_bounds__(256) sum_slices_kernel(const MatDev* tab, cons
   }
 }
 
-int atb_splits(int rows) {
+// Row slices of an A^T B product over `rows` rows when `count` matrices share the launch: about 1024 rows per
+// slice for batched launches, finer (down to 128 rows) when few matrices would otherwise leave most SMs idle.
+int atb_splits(int rows, int count) {
   int s = (rows + 1023) / 1024;
-  return s < 1 ? 1 : (s > kAtbMaxSplits ? kAtbMaxSplits : s);
+  const int want = (2 * 148 + count - 1) / (count > 0 ? count : 1);
+  if (s < want) s = want;
+  const int finest = (rows + 127) / 128;
+  if (s > finest) s = finest;
+  if (s > kAtbMaxSplits) s = kAtbMaxSplits;
+  return s < 1 ? 1 : s;
 }
 
 void launch_atb(const MatDev* tab, const int* idx, int count, int offA, int offB, int offPart, int offOut, int rows,
-                int ca, int cb, int lda, int ldb, cudaStream_t s) {
+                int ca, int cb, int lda, int ldb, int nsplit, cudaStream_t s, int b_slices, bool sum_here) {
   if (count <= 0 || ca <= 0 || cb <= 0) return;
-  const int nsplit = atb_splits(rows);
   const int rps = ((rows + nsplit - 1) / nsplit + 31) / 32 * 32;
   const int big = ca > cb ? ca : cb;
   const int mt = big <= 16 ? 1 : big <= 32 ? 2 : big <= 64 ? 4 : 8;
   const int ts = 16 * mt;
   dim3 grid(nsplit, ((ca + ts - 1) / ts) * ((cb + ts - 1) / ts), count);
   switch (mt) {
-    case 1: atb_kernel<1><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps); break;
-    case 2: atb_kernel<2><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps); break;
-    case 4: atb_kernel<4><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps); break;
-    default: atb_kernel<8><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps); break;
+    case 1: atb_kernel<1><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps, b_slices); break;
+    case 2: atb_kernel<2><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps, b_slices); break;
+    case 4: atb_kernel<4><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps, b_slices); break;
+    default: atb_kernel<8><<<grid, 256, 0, s>>>(tab, idx, offA, offB, offPart, rows, ca, cb, lda, ldb, rps, b_slices); break;
   }
   ++g_kernel_launches;
+  if (!sum_here) return;     // the consumer adds the row slices itself
   const int numel = ca * cb;
   sum_slices_kernel<<<dim3((numel + 255) / 256 < 64 ? (numel + 255) / 256 : 64, 1, count), 256, 0, s>>>(
       tab, idx, offPart, offOut, numel, nsplit);
@@ -546,11 +575,6 @@ void launch_filter_weights(const MatDev* tab, const int* idx, int count, int rp,
 // =====================================================================================================
 // bf16 hi/lo splits of the basis: U ~= Uhi + Ulo (m x rp), V^T ~= Vthi + Vtlo (rp x n, transposed).
 // =====================================================================================================
-__device__ __forceinline__ void split2(float x, bf16& hi, bf16& lo) {
-  hi = __float2bfloat16_rn(x);
-  lo = __float2bfloat16_rn(x - __bfloat162float(hi));
-}
-
 __global__ void __launch_bounds__(256) split_basis_kernel(const MatDev* tab, const int* idx, int m, int n, int rp,
                                                           int rk) {
   const MatDev& md = tab[idx[blockIdx.z]];
@@ -628,21 +652,23 @@ void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, 
 // The r x r filter: Xs = coef * D X D (coef = (1-alpha)*scale), and the per-matrix statistics.
 //   stats[0] = ||g||^2, stats[1] = ||X||^2 (scaled), stats[2] = ||G_proj||^2 (closed form), stats[3] = sum d^2
 // =====================================================================================================
-__global__ void __launch_bounds__(256) xs_kernel(const MatDev* tab, const int* idx, int rp, int rank, float coef,
+__global__ void __launch_bounds__(256) xs_kernel(const MatDev* tab, const int* idx, int rp, int rank, int x_slices,
                                                  float scale, float alpha, unsigned* status) {
   __shared__ float red[3][8];
   const MatDev& md = tab[idx[blockIdx.x]];
   float sx = 0.f, s1 = 0.f, s2 = 0.f;
   for (int e = threadIdx.x; e < rp * rp; e += 256) {
     const int i = e / rp, j = e % rp;
-    const float x = md.X[e] * scale;
+    float xr = 0.f;                       // X = sum of the row-slice partials of U^T T, in slice order
+    for (int sl = 0; sl < x_slices; ++sl) xr += md.xpart[(size_t)sl * rp * rp + e];
+    md.X[e] = xr;
+    const float x = xr * scale;
     const float dd = (i < rank && j < rank) ? md.d[i] * md.d[j] : 0.f;
     md.Xs[e] = (1.f - alpha) * dd * x;
     sx = fmaf(x, x, sx);
     s1 = fmaf(dd * x, x, s1);
     s2 = fmaf(dd * dd * x, x, s2);
   }
-  (void)coef;
   sx = warp_sum(sx); s1 = warp_sum(s1); s2 = warp_sum(s2);
   if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = sx; red[1][threadIdx.x >> 5] = s1; red[2][threadIdx.x >> 5] = s2; }
   __syncthreads();
@@ -661,10 +687,10 @@ __global__ void __launch_bounds__(256) xs_kernel(const MatDev* tab, const int* i
   }
 }
 
-void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, float coef, float scale, float alpha,
+void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, int x_slices, float scale, float alpha,
                unsigned* status, cudaStream_t s) {
   if (count <= 0) return;
-  xs_kernel<<<count, 256, 0, s>>>(tab, idx, rp, rank, coef, scale, alpha, status);
+  xs_kernel<<<count, 256, 0, s>>>(tab, idx, rp, rank, x_slices, scale, alpha, status);
   ++g_kernel_launches;
 }
 

@@ -830,7 +830,8 @@ sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int coun
   g.row_tiles = (m + 127) / 128;
   g.col_tiles = (n + kTileN - 1) / kTileN;
   int csplit = 1;
-  while ((long long)count * g.row_tiles * csplit < 4LL * n_sm && g.col_tiles / (csplit * 2) >= 4) csplit *= 2;
+  // enough work items that the last, partly filled round of the persistent blocks costs a few percent at most
+  while ((long long)count * g.row_tiles * csplit < 16LL * n_sm && g.col_tiles / (csplit * 2) >= 2) csplit *= 2;
   g.tiles_per_chunk = (g.col_tiles + csplit - 1) / csplit;
   g.csplit = (g.col_tiles + g.tiles_per_chunk - 1) / g.tiles_per_chunk;
   g.n_items = count * g.row_tiles * g.csplit;
