@@ -589,10 +589,13 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
     }
     ProfScope ps(p, PROF_FILTER);
     // X = U^T T as row-slice partials (the K-slice partials of T are added on the way in); xs_kernel adds them up
+    // (one block per matrix adds the slices inside xs_kernel unless that is too much for one block)
+    const bool sum_in_xs = (size_t)c.split_m * rp * rp <= (size_t)(1 << 16);
     if (rp > 0)
-      launch_atb(p->dev_tab, idx, cnt, OFF(U), OFF(T), OFF(xpart), OFF(X), m, rp, rp, rp, rp, c.split_m, s, c.ksplit, false);
+      launch_atb(p->dev_tab, idx, cnt, OFF(U), OFF(T), OFF(xpart), OFF(X), m, rp, rp, rp, rp, c.split_m, s, c.ksplit,
+                 !sum_in_xs);
     if (want_norm) launch_sqnorm(p->dev_tab, idx, cnt, (int64_t)m * n, g_bf16, s);
-    launch_xs(p->dev_tab, idx, cnt, rp, p->rank, rp > 0 ? c.split_m : 0, scale, hp.alpha, p->status_dev, s);   // D X D
+    launch_xs(p->dev_tab, idx, cnt, rp, p->rank, (rp > 0 && sum_in_xs) ? c.split_m : 0, scale, hp.alpha, p->status_dev, s);   // D X D
     if (rp > 0) {
       GemmArgs ga = gemm(p, idx, OFF(V), OFF(Xs), OFF(Ct), n, rp, rp, rp, rp, rp, 0, 1);             // C^T = V Xs^T
       if (c.tensor) { ga.offHi = OFF(Cthi); ga.offLo = OFF(Ctlo); ga.ld_split = p->rk; }

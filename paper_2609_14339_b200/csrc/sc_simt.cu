@@ -659,9 +659,14 @@ __global__ void __launch_bounds__(256) xs_kernel(const MatDev* tab, const int* i
   float sx = 0.f, s1 = 0.f, s2 = 0.f;
   for (int e = threadIdx.x; e < rp * rp; e += 256) {
     const int i = e / rp, j = e % rp;
-    float xr = 0.f;                       // X = sum of the row-slice partials of U^T T, in slice order
-    for (int sl = 0; sl < x_slices; ++sl) xr += md.xpart[(size_t)sl * rp * rp + e];
-    md.X[e] = xr;
+    float xr;
+    if (x_slices > 0) {                   // X = sum of the row-slice partials of U^T T, in slice order
+      xr = 0.f;
+      for (int sl = 0; sl < x_slices; ++sl) xr += md.xpart[(size_t)sl * rp * rp + e];
+      md.X[e] = xr;
+    } else {
+      xr = md.X[e];                       // already summed by a separate launch
+    }
     const float x = xr * scale;
     const float dd = (i < rank && j < rank) ? md.d[i] * md.d[j] : 0.f;
     md.Xs[e] = (1.f - alpha) * dd * x;
