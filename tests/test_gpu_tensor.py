@@ -130,3 +130,18 @@ def test_warm_started_range_finder(torch, engine):
     d_warm = so.projector_distance(o.states[0].V, oe.states[0].V)
     d_cold = so.projector_distance(oc.states[0].V, oe.states[0].V)
     assert d_warm < d_cold
+
+
+@pytest.mark.parametrize("shape,k", [((1024, 1024), 16), ((512, 2048), 32)])
+def test_exact_parity_where_the_rank_cut_is_well_posed(torch, shape, k):
+    """Gate G3: with r equal to the planted rank there is a wide spectral gap at the cut, the truncated SVD is
+    well conditioned, and the GPU path (l = 2r, q = 4) must match the oracle's EXACT mode."""
+    case = Case(shapes=[shape], rank=k, tokens=1024, keep=0.1, planted=k, snr=4.0, seed=12, tau_p=1e-3, q=4, l=2 * k)
+    inp = make_inputs(case)
+    g = GpuRun(case, inp, torch)
+    oe = OracleRun(case, inp, "exact")
+    s_all = np.linalg.svd(oe.states[0].M_anc, compute_uv=False)
+    assert (s_all[k - 1] - s_all[k]) / s_all[k - 1] > 0.3            # the gap is really there
+    eb, es = compare_basis(g, oe), compare_step(g, oe)
+    assert max(eb["PU"], eb["PV"], eb["s"]) < TOL, eb
+    assert max(es["gproj"], es["m"], es["v"], es["dW"]) < TOL, es
