@@ -146,6 +146,15 @@ SC_API sc_status sc_plan_destroy(sc_plan* plan);
  * (sketch width l, q power iterations), then Eq. 2. The basis is cached until the next arrival. */
 SC_API sc_status sc_anchor_update(sc_plan* plan, const void* const* anchor_grads, int64_t step_tag);
 
+/* sc_anchor_update_factored - the same arrival when the anchor gradient comes as rank-rho factors, G_anc = P Q^T
+ * (the staleness appendix has the anchor circuit push its gradient compressed to about one data-parallel
+ * all-reduce payload, i.e. low-rank factors). Eq. 1 is applied tile by tile without ever forming G_anc.
+ *   P_factors   host array of n_mats device pointers, rows x rho fp32 row-major (NULL entry = not arrived)
+ *   Q_factors   host array of n_mats device pointers, cols x rho fp32 row-major (NULL exactly where P is NULL)
+ *   rho         1..1024 */
+SC_API sc_status sc_anchor_update_factored(sc_plan* plan, const void* const* P_factors, const void* const* Q_factors,
+                                           int rho, int64_t step_tag);
+
 /* sc_correct_and_step - one fast-circuit optimizer step over all matrices (Algorithm 1 lines 10-13).
  *   masked_grads   host array of n_mats device pointers (grad_dtype, rows x cols), read only
  *   params         host array of n_mats device pointers, fp32 master weights, updated in place

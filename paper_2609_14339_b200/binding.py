@@ -73,6 +73,7 @@ EXPORTS = {
                                  _VP, C.c_size_t, _VP]),
     "sc_plan_destroy": (C.c_int, [_VP]),
     "sc_anchor_update": (C.c_int, [_VP, _VPP, C.c_int64]),
+    "sc_anchor_update_factored": (C.c_int, [_VP, _VPP, _VPP, C.c_int, C.c_int64]),
     "sc_correct_and_step": (C.c_int, [_VP, _VPP, _VPP, C.POINTER(OptState), C.c_int64]),
     "sc_correct_and_step_host": (C.c_int, [_VP, _VPP, _VPP, _VPP, C.POINTER(OptState), C.c_int64, C.POINTER(MatStats),
                                            C.POINTER(C.c_float)]),
@@ -220,6 +221,12 @@ class Plan:
     def anchor_update(self, anchor_grads: Sequence, step_tag: int) -> int:
         arr = _ptr_array(anchor_grads, self.n_mats, True)
         return _check(self.lib.sc_anchor_update(self.handle, arr, int(step_tag)), "sc_anchor_update")
+
+    def anchor_update_factored(self, P_factors: Sequence, Q_factors: Sequence, step_tag: int) -> int:
+        rho = next(t.shape[1] for t in P_factors if t is not None)
+        return _check(self.lib.sc_anchor_update_factored(self.handle, _ptr_array(P_factors, self.n_mats, True),
+                                                         _ptr_array(Q_factors, self.n_mats, True), int(rho),
+                                                         int(step_tag)), "sc_anchor_update_factored")
 
     def correct_and_step(self, masked_grads, params, exp_avg, exp_avg_sq, step: int, params_bf16=None) -> int:
         n = self.n_mats

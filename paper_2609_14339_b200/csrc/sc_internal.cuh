@@ -66,7 +66,8 @@ struct MatDev {
   const float* omega;    // n x lp  the same sketch, row-major (tensor-core classes only)
   // per call
   const void* G;      // masked gradient
-  const void* Ganc;   // anchor gradient
+  const void* Ganc;   // anchor gradient (dense), or its left factor P (rows x rho fp32)
+  const void* Qanc;   // right factor Q (cols x rho fp32) of a factored anchor gradient, else null
   float* W;           // fp32 master weights
   float* m1;          // AdamW first moment
   float* m2;          // AdamW second moment
@@ -159,6 +160,7 @@ struct GemmArgs {
   int transA, transB;
   int a_bf16;              // A holds bf16 (gradients) instead of fp32
   float alpha;
+  float beta_c;            // C = alpha * acc + beta_c * C_old (0: plain store)
   int offHi, offLo, ld_split;   // when offHi != 0: also write the result as a bf16 hi/lo pair with this row stride
 };
 void launch_gemm(const GemmArgs& a, int count, cudaStream_t s);

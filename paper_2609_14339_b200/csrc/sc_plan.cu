@@ -408,15 +408,27 @@ sc_status sc_plan_destroy(sc_plan* p) {
   return SC_OK;
 }
 
-sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t step_tag) {
+// Anchor arrival. Dense form: anchor_grads[i] is G_anc (grad_dtype). Factored form (q_factors != nullptr):
+// anchor_grads[i] is P (rows x rho fp32), q_factors[i] is Q (cols x rho fp32) and G_anc = P Q^T is never formed.
+static sc_status anchor_impl(sc_plan* p, const void* const* anchor_grads, const void* const* q_factors, int rho,
+                             int64_t step_tag) {
   if (!p) return SC_ERR_INVALID_ARG;
   sc_status st = check_ptr_array(anchor_grads, p->n_mats, true);
   if (st != SC_OK) return st;
+  if (q_factors) {
+    if (rho < 1 || rho > 1024) return SC_ERR_INVALID_ARG;
+    if ((st = check_ptr_array(q_factors, p->n_mats, true)) != SC_OK) return st;
+    for (int i = 0; i < p->n_mats; ++i)
+      if ((anchor_grads[i] == nullptr) != (q_factors[i] == nullptr)) return SC_ERR_INVALID_ARG;
+  }
   if (step_tag < p->last_tag) return SC_ERR_STALE_TAG;
   cudaStream_t s = p->stream;
   const int lp = p->lp, rp = p->rp;
   const int g_bf16 = p->hp.grad_dtype == SC_DTYPE_BF16;
-  for (int i = 0; i < p->n_mats; ++i) p->host_tab[i].Ganc = anchor_grads[i];
+  for (int i = 0; i < p->n_mats; ++i) {
+    p->host_tab[i].Ganc = anchor_grads[i];
+    p->host_tab[i].Qanc = q_factors ? q_factors[i] : nullptr;
+  }
   if ((st = upload_table(p)) != SC_OK) return st;
   // The matrices that received a gradient, class by class, in two groups: cold starts (range finder from the
   // sketch) and warm starts (from the previous right basis), each with one flat list for the class-independent kernels.
@@ -449,8 +461,18 @@ sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t 
   {
     ProfScope ps(p, PROF_EMA);
     for (int w = 0; w < 2; ++w)
-      for (const auto& a : act[w])
-        launch_ema(p->dev_tab, a.idx, a.cnt, a.c->m * a.c->n, g_bf16, p->hp.beta_anc, s);             // Eq. 1
+      for (const auto& a : act[w]) {
+        if (!q_factors) {
+          launch_ema(p->dev_tab, a.idx, a.cnt, a.c->m * a.c->n, g_bf16, p->hp.beta_anc, s);           // Eq. 1
+        } else {
+          // Eq. 1 with G_anc = P Q^T: M <- beta M + (1 - beta) P Q^T, tile by tile
+          const int m = (int)a.c->m, n = (int)a.c->n;
+          GemmArgs ga = gemm(p, a.idx, OFF(Ganc), OFF(Qanc), OFF(Manc), m, n, rho, rho, rho, n, 0, 1);
+          ga.alpha = 1.f - p->hp.beta_anc;
+          ga.beta_c = p->hp.beta_anc;
+          launch_gemm(ga, a.cnt, s);
+        }
+      }
   }
   for (int w = 0; w < 2 && p->rank > 0; ++w) {
     if (flat[w].empty()) continue;
@@ -510,6 +532,16 @@ sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t 
     for (int id : flat[w]) p->has_basis[id] = 1;
   p->last_tag = step_tag;
   return cuda_ok(cudaGetLastError());
+}
+
+sc_status sc_anchor_update(sc_plan* p, const void* const* anchor_grads, int64_t step_tag) {
+  return anchor_impl(p, anchor_grads, nullptr, 0, step_tag);
+}
+
+sc_status sc_anchor_update_factored(sc_plan* p, const void* const* P_factors, const void* const* Q_factors, int rho,
+                                    int64_t step_tag) {
+  if (!Q_factors) return SC_ERR_INVALID_ARG;
+  return anchor_impl(p, P_factors, Q_factors, rho, step_tag);
 }
 
 // One optimizer step. With host_grads != nullptr the masked gradients are first copied from host memory into

@@ -92,7 +92,8 @@ __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs a, EpiAdamW epi) {
       for (int j = 0; j < 4; ++j) {
         const int gc = col0 + tx * 4 + j;
         if (gc < a.N) {
-          const float val = a.alpha * acc[i][j];
+          float val = a.alpha * acc[i][j];
+          if (a.beta_c != 0.f) val = fmaf(a.beta_c, C[(size_t)gr * a.ldc + gc], val);
           C[(size_t)gr * a.ldc + gc] = val;
           if (a.offHi) {   // also the bf16 hi/lo pair the tensor-core kernels read
             bf16 hi, lo;

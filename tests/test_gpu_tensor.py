@@ -145,3 +145,30 @@ def test_exact_parity_where_the_rank_cut_is_well_posed(torch, shape, k):
     eb, es = compare_basis(g, oe), compare_step(g, oe)
     assert max(eb["PU"], eb["PV"], eb["s"]) < TOL, eb
     assert max(es["gproj"], es["m"], es["v"], es["dW"]) < TOL, es
+
+
+@pytest.mark.parametrize("engine", [0, 1])
+def test_factored_anchor_gradient(torch, engine):
+    """Anchor gradients arriving as rank-rho factors P Q^T: Eq. 1 without densifying, then the usual basis."""
+    from parity_util import make_plan
+    rng = np.random.default_rng(21)
+    case = Case(shapes=[(384, 256), (200, 136)], rank=8, tokens=128, tau_p=5.0, engine=engine)
+    plan = make_plan(case, torch)
+    hp = so.Hyper(beta_anc=float(np.float32(0.9)))
+    states = [so.new_state(m, n) for m, n in case.shapes]
+    for arrival, rho in enumerate((12, 5)):
+        Ps = [rng.standard_normal((m, rho)).astype(np.float32) for m, n in case.shapes]
+        Qs = [rng.standard_normal((n, rho)).astype(np.float32) for m, n in case.shapes]
+        plan.anchor_update_factored([torch.from_numpy(x).cuda() for x in Ps], [torch.from_numpy(x).cuda() for x in Qs], arrival)
+        for st, P, Q, (m, n) in zip(states, Ps, Qs, case.shapes):
+            so.anchor_update(st, P.astype(np.float64) @ Q.astype(np.float64).T, hp, 8, mode="mirror",
+                             Omega=so.rademacher_sketch(0, 0, n, 8), q=1)
+    torch.cuda.synchronize()
+    for i, st in enumerate(states):
+        assert rel(plan.export_anchor_momentum(i).double().cpu().numpy(), st.M_anc) < 1e-6
+        U, s, V = [x.double().cpu().numpy() for x in plan.export_basis(i)]
+        tol = TOL if engine == 0 else 1e-4
+        assert so.projector_distance(U, st.U) < tol and so.projector_distance(V, st.V) < tol and rel(s, st.s) < tol
+    import paper_2609_14339_b200 as sc
+    with pytest.raises(sc.SCError):
+        plan.anchor_update_factored([None, torch.zeros((200, 4), device="cuda")], [torch.zeros((256, 4), device="cuda"), None], 9)
