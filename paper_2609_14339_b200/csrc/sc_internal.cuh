@@ -132,6 +132,7 @@ struct sc_plan {
   std::vector<void*> dbg_out;
   bool table_dirty = true;
   bool tensor_any = false;
+  int n_sm = 0;                       // SM count of the plan's device
   // host-gradient path: copies run on their own stream, one event per shape class
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t copy_gate = nullptr;

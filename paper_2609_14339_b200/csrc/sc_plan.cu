@@ -342,11 +342,13 @@ sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int 
   cudaDeviceProp prop;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return SC_ERR_CUDA;
   if (prop.major != 10) return SC_ERR_UNSUPPORTED_ARCH;
+  const int n_sm = prop.multiProcessorCount;
 
   sc_plan* p = new (std::nothrow) sc_plan();
   if (!p) return SC_ERR_INVALID_ARG;
   fill_plan_basics(p, shapes, n_mats, rank, hp, d);
   p->keep = keep_ratio;
+  p->n_sm = n_sm;
   p->stream = reinterpret_cast<cudaStream_t>(stream);
   p->ws = nullptr;
   const size_t need = layout(p, false);

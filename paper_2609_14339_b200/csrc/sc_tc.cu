@@ -657,23 +657,21 @@ bool tc_shape_supported(int64_t m, int64_t n, int rp) {
 size_t tc_tmaps_bytes(int count) { return (size_t)count * kMapsPerMat * sizeof(CUtensorMap); }
 
 sc_status tc_init() {
-  if (g_encode) return SC_OK;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
-      qres != cudaDriverEntryPointSuccess)
-    return SC_ERR_CUDA;
-  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
-  static bool attrs_done = false;
-  if (!attrs_done) {
-    if (cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(fused_update_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kStreamSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess)
       return SC_ERR_CUDA;
-    attrs_done = true;
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
+  // per device: the opt-in shared-memory sizes (cheap, so simply repeated for every plan)
+  if (cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(fused_update_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kStreamSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
+    return SC_ERR_CUDA;
   return SC_OK;
 }
 
@@ -819,12 +817,7 @@ sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, b
 
 sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc) {
   const int m = (int)c.m, n = (int)c.n;
-  static int n_sm = 0;
-  if (!n_sm) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm <= 0) n_sm = 148;
-  }
+  const int n_sm = p->n_sm > 0 ? p->n_sm : 148;
   StreamGeom g;
   g.m = m; g.n = n; g.rp = p->rp;
   g.row_tiles = (m + 127) / 128;
