@@ -197,6 +197,8 @@ sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_
 sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count);   // T = G V
 sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc);
 sc_status tc_launch_wait_probe(sc_plan* p, int max_polls);
+sc_status tc_encode_anchor(sc_plan* p, ShapeClass& c, const std::vector<int>& ids);
+sc_status tc_launch_ema_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, int b_field_off);
 sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, bool transposed, int b_field_off);
 
 }  // namespace sc

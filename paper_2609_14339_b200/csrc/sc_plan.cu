@@ -434,6 +434,8 @@ static sc_status anchor_impl(sc_plan* p, const void* const* anchor_grads, const 
   if ((st = upload_table(p)) != SC_OK) return st;
   // The matrices that received a gradient, class by class, in two groups: cold starts (range finder from the
   // sketch) and warm starts (from the previous right basis), each with one flat list for the class-independent kernels.
+  // dense bf16 anchors on tensor-core classes: Eq. 1 rides on the first sweep of the range finder
+  const bool fuse_ema = !q_factors && g_bf16 && p->rank > 0;
   std::vector<ActiveClass> act[2];
   std::vector<int> flat[2];
   for (auto& c : p->classes) {
@@ -452,6 +454,7 @@ static sc_status anchor_impl(sc_plan* p, const void* const* anchor_grads, const 
       }
       act[w].push_back(ActiveClass{&c, idx, (int)ids[w].size()});
       flat[w].insert(flat[w].end(), ids[w].begin(), ids[w].end());
+      if (fuse_ema && c.tensor && (st = tc_encode_anchor(p, c, ids[w])) != SC_OK) return st;
     }
   }
   if (flat[0].empty() && flat[1].empty()) { p->last_tag = step_tag; return SC_OK; }
@@ -464,6 +467,7 @@ static sc_status anchor_impl(sc_plan* p, const void* const* anchor_grads, const 
     ProfScope ps(p, PROF_EMA);
     for (int w = 0; w < 2; ++w)
       for (const auto& a : act[w]) {
+        if (fuse_ema && a.c->tensor) continue;      // done inside the first sweep below
         if (!q_factors) {
           launch_ema(p->dev_tab, a.idx, a.cnt, a.c->m * a.c->n, g_bf16, p->hp.beta_anc, s);           // Eq. 1
         } else {
@@ -483,10 +487,12 @@ static sc_status anchor_impl(sc_plan* p, const void* const* anchor_grads, const 
     const int n_all = (int)flat[w].size();
     const int q = w ? p->hp.warm_power_iters : p->q;
     // one sweep over the momentum: transposed ? Z <- M^T B : Y <- M B
+    bool first_sweep = true;
     auto pass = [&](int offB, bool transposed) {
       ProfScope ps(p, PROF_PASS);
       for (const auto& a : ac) {
         const int m = (int)a.c->m, n = (int)a.c->n;
+        if (a.c->tensor && first_sweep && fuse_ema) { tc_launch_ema_pass(p, *a.c, a.idx, a.cnt, offB); continue; }
         if (a.c->tensor) { tc_launch_pass(p, *a.c, a.idx, a.cnt, transposed, offB); continue; }
         const int tB = offB == OFF(omega_t);
         if (!transposed)
@@ -494,6 +500,7 @@ static sc_status anchor_impl(sc_plan* p, const void* const* anchor_grads, const 
         else
           launch_gemm(gemm(p, a.idx, OFF(Manc), offB, OFF(Z), n, lp, m, n, lp, lp, 1, 0), a.cnt, s);
       }
+      first_sweep = false;
     };
     // range finder: Y = M S with S the sketch (cold) or [previous V | sketch columns] (warm); Q = orth(Y)
     if (w) {

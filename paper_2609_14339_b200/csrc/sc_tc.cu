@@ -115,7 +115,7 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16(int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-constexpr int kMapsPerMat = 22;
+constexpr int kMapsPerMat = 24;
 constexpr int kPerCallMaps = 6;   // the first six are rebuilt whenever the caller's buffers move
 enum { MAP_G = 0,    // masked gradient, bf16, box 64 x 128 (MMA A operand of the projection)
        MAP_G32,      // masked gradient, bf16, box 32 x 128, 64-byte swizzle (streaming tile of the fused update)
@@ -127,6 +127,8 @@ enum { MAP_G = 0,    // masked gradient, bf16, box 64 x 128 (MMA A operand of th
        MAP_M_MN,     // anchor momentum as an MN-major A operand: box 32 floats x 32 rows (one swizzle atom column)
        MAP_Y, MAP_Z, MAP_OMEGA,  // m x lp, n x lp, n x lp row-major fp32 as MN-major B operands: box 32 x 32
        MAP_Y2, MAP_Z2,           // the scratch twins of Y and Z (a single-round Cholesky QR leaves its result there)
+       MAP_GANC32,               // anchor gradient, bf16, box 32 x 128, 64-byte swizzle (rebuilt per anchor call)
+       MAP_M_F32,                // anchor momentum as plain fp32 (box 32 x 128): load and store of the fused EMA sweep
        MAP_SPARE };
 constexpr int kTileBytes = 128 * 128;   // 128 rows x 64 bf16
 
@@ -346,6 +348,154 @@ pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const C
         tmem_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + c, v);
         tmem_ld_wait();
         if (row < rows_out) {
+#pragma unroll
+          for (int j = 0; j < 16; j += 4)
+            *reinterpret_cast<float4*>(out + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_d, tmem_cols);
+}
+
+// =====================================================================================================
+// First sweep of the range finder fused with the anchor EMA (Eq. 1): the block streams its 128 rows of the OLD
+// momentum and of the bf16 anchor gradient, four warps form M_new = beta M + (1 - beta) G_anc in shared memory,
+// one thread sends the tile back with a TMA store while the MMA warp consumes the same tile for Y = M_new B.
+// The momentum is read once and written once for Eq. 1 and this sweep together.
+//   warp 0 producer | warp 1 MMA | warps 2-5 transform, later epilogue | warp 6 store
+// =====================================================================================================
+constexpr int kGancTile = 128 * 32 * 2;   // bf16, 128 rows x 32 columns
+
+__global__ void __launch_bounds__(224, 2)
+ema_pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const CUtensorMap* __restrict__ maps,
+                int b_map, int m, int n, int lp, int stages, uint32_t tmem_cols, float beta, unsigned* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int b_bytes = (lp / 32) * kAtomBytes;
+  const int stage_bytes = kTileBytes + kGancTile + b_bytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+  uint64_t* ready = full + stages;
+  uint64_t* empty = ready + stages;
+  uint64_t* accum = empty + stages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
+  const int row0 = blockIdx.x * 128;
+  const int nchunks = (n + kPassK - 1) / kPassK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&ready[s], 4); mbar_init(&empty[s], 2); }
+    mbar_init(accum, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_d = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const CUtensorMap* bmap = mp + b_map;
+      tensormap_acquire(mp + MAP_M_F32); tensormap_acquire(mp + MAP_GANC32); tensormap_acquire(bmap);
+      for (int i = 0; i < nchunks; ++i) {
+        const int s = i % stages;
+        if (!mbar_wait(&empty[s], ((i / stages) & 1) ^ 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
+        uint8_t* st = smem + (size_t)s * stage_bytes;
+        mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
+        const int k0 = i * kPassK;
+        tma_load_2d(st, mp + MAP_M_F32, &full[s], k0, row0);
+        tma_load_2d(st + kTileBytes, mp + MAP_GANC32, &full[s], k0, row0);
+        for (int a = 0; a < lp / 32; ++a)
+          tma_load_2d(st + kTileBytes + kGancTile + a * kAtomBytes, bmap, &full[s], 32 * a, k0);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_tf32(lp, 0, 1);
+      for (int i = 0; i < nchunks; ++i) {
+        const int s = i % stages;
+        if (!mbar_wait(&ready[s], (i / stages) & 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
+        tc_fence_after();
+        const uint32_t a = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint32_t b = a + kTileBytes + kGancTile;
+#pragma unroll
+        for (int k = 0; k < kPassK / 8; ++k)
+          umma_tf32(tmem_d, umma_desc_k128(a + k * 32), umma_desc_mn128(b + k * 1024, kAtomBytes), idesc, (i | k) != 0);
+        umma_commit(&empty[s]);
+      }
+      umma_commit(accum);
+    }
+    __syncwarp();
+  } else if (warp == 6) {
+    if (lane == 0) {
+      tensormap_acquire(mp + MAP_M_F32);
+      for (int i = 0; i < nchunks; ++i) {
+        const int s = i % stages;
+        if (!mbar_wait(&ready[s], (i / stages) & 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
+        tma_store_2d(mp + MAP_M_F32, smem + (size_t)s * stage_bytes, i * kPassK, row0);
+        tma_store_commit();
+        tma_store_wait_read<0>();
+        mbar_arrive(&empty[s]);
+      }
+      tma_store_wait_all();
+    }
+    __syncwarp();
+  } else {
+    // transform warps: one row per thread, 32 columns per chunk
+    const int q = warp & 3;
+    const int r = q * 32 + lane;
+    const float omb = 1.f - beta;
+    bool dead = false;
+    for (int i = 0; i < nchunks; ++i) {
+      const int s = i % stages;
+      if (!mbar_wait(&full[s], (i / stages) & 1, abort_flag)) { dead = true; break; }
+      uint8_t* st = smem + (size_t)s * stage_bytes;
+      float4* Ms = reinterpret_cast<float4*>(st);
+      const uint4* Gs = reinterpret_cast<const uint4*>(st + kTileBytes);
+#pragma unroll
+      for (int cg = 0; cg < 4; ++cg) {
+        const uint4 graw = Gs[r * 4 + (cg ^ ((r >> 1) & 3))];
+        const uint32_t gw[4] = {graw.x, graw.y, graw.z, graw.w};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int fidx = r * 8 + ((2 * cg + h) ^ (r & 7));
+          float4 mv = Ms[fidx];
+          const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gw[2 * h]);
+          const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&gw[2 * h + 1]);
+          mv.x = fmaf(beta, mv.x, omb * __low2float(g01));
+          mv.y = fmaf(beta, mv.y, omb * __high2float(g01));
+          mv.z = fmaf(beta, mv.z, omb * __low2float(g23));
+          mv.w = fmaf(beta, mv.w, omb * __high2float(g23));
+          Ms[fidx] = mv;
+        }
+      }
+      fence_proxy_async();          // the new tile must be visible to the MMA and to the TMA store
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ready[s]);
+    }
+    // epilogue: Y rows from the accumulator
+    bool ok = !dead && mbar_wait(accum, 0, abort_flag);
+    if (!ok && lane == 0) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
+    ok = __all_sync(0xffffffffu, ok) && !*abort_flag;
+    tc_fence_after();
+    if (ok) {
+      const int row = row0 + r;
+      float* out = md.Y + (size_t)row * lp;
+      for (int c = 0; c < lp; c += 16) {
+        float v[16];
+        tmem_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + c, v);
+        tmem_ld_wait();
+        if (row < m) {
 #pragma unroll
           for (int j = 0; j < 16; j += 4)
             *reinterpret_cast<float4*>(out + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -669,6 +819,7 @@ sc_status tc_init() {
   if (cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(fused_update_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kStreamSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(ema_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
     return SC_ERR_CUDA;
@@ -735,6 +886,8 @@ sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_
       ok = ok && encode_tf32(mp + MAP_Y, md.Y, lp, c.m, kPassK, true);
       ok = ok && encode_tf32(mp + MAP_Z, md.Z, lp, c.n, kPassK, true);
       ok = ok && encode_tf32(mp + MAP_OMEGA, md.omega, lp, c.n, kPassK, true);
+      ok = ok && encode2d(mp + MAP_M_F32, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, md.Manc, c.n, c.m, c.n, 32, 128,
+                          CU_TENSOR_MAP_SWIZZLE_128B);
       ok = ok && encode_tf32(mp + MAP_Y2, md.Y2, lp, c.m, kPassK, true);
       ok = ok && encode_tf32(mp + MAP_Z2, md.Z2, lp, c.n, kPassK, true);
       if (!ok) return SC_ERR_CUDA;
@@ -782,6 +935,41 @@ sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count
 
 sc_status tc_launch_wait_probe(sc_plan* p, int max_polls) {
   wait_probe_kernel<<<1, 32, 0, p->stream>>>(max_polls, p->status_dev);
+  ++g_kernel_launches;
+  return cuda_ok(cudaGetLastError());
+}
+
+// Tensor maps of the anchor gradients of one call (the matrices listed in ids), copied to the device.
+sc_status tc_encode_anchor(sc_plan* p, ShapeClass& c, const std::vector<int>& ids) {
+  CUtensorMap* dev = static_cast<CUtensorMap*>(c.tmaps);
+  for (int id : ids) {
+    const MatDev& md = p->host_tab[id];
+    CUtensorMap tm;
+    if (!encode2d(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, md.Ganc, c.n, c.m, c.n, 32, 128, CU_TENSOR_MAP_SWIZZLE_64B))
+      return SC_ERR_CUDA;
+    // pageable source: the runtime has taken its copy when this returns
+    if (cudaMemcpyAsync(dev + (size_t)md.inst * kMapsPerMat + MAP_GANC32, &tm, sizeof(tm), cudaMemcpyHostToDevice,
+                        p->stream) != cudaSuccess)
+      return SC_ERR_CUDA;
+  }
+  return SC_OK;
+}
+
+// Eq. 1 fused with the first sweep: M <- beta M + (1 - beta) G_anc and Y <- M_new B in one pass over M.
+sc_status tc_launch_ema_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, int b_field_off) {
+  const int lp = p->lp, m = (int)c.m, n = (int)c.n;
+  const int stage_bytes = kTileBytes + kGancTile + (lp / 32) * kAtomBytes;
+  const int stages = stages_for(stage_bytes, 6);
+  const size_t smem = (size_t)stages * stage_bytes + 1024 + 512;
+  uint32_t cols = 32;
+  while ((int)cols < lp) cols <<= 1;
+  int b_map;
+  if (b_field_off == (int)offsetof(MatDev, omega_t) || b_field_off == (int)offsetof(MatDev, omega)) b_map = MAP_OMEGA;
+  else if (b_field_off == (int)offsetof(MatDev, Z2)) b_map = MAP_Z2;
+  else return SC_ERR_INVALID_ARG;
+  dim3 grid((m + 127) / 128, 1, count);
+  ema_pass_kernel<<<grid, 224, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), b_map, m, n,
+                                                  lp, stages, cols, p->hp.beta_anc, p->status_dev);
   ++g_kernel_launches;
   return cuda_ok(cudaGetLastError());
 }
