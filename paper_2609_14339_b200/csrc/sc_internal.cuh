@@ -166,6 +166,8 @@ struct GemmArgs {
 };
 void launch_gemm(const GemmArgs& a, int count, cudaStream_t s);
 int atb_splits(int rows, int count);
+void launch_sum_slices(const MatDev* tab, const int* idx, int count, int offPart, int offOut, int numel, int nsplit,
+                       cudaStream_t s);
 void launch_atb(const MatDev* tab, const int* idx, int count, int offA, int offB, int offPart, int offOut, int rows,
                 int ca, int cb, int lda, int ldb, int nsplit, cudaStream_t s, int b_slices = 1, bool sum_here = true);
 void launch_epilogue_simt(const MatDev* tab, const int* idx, int count, int m, int n, int rp, int g_bf16,
@@ -183,7 +185,6 @@ void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int
 void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, int g_bf16, cudaStream_t s);
 void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, int x_slices, float scale, float alpha,
                unsigned* status, cudaStream_t s);
-void launch_split_ct(const MatDev* tab, const int* idx, int count, int n, int rp, int rk, cudaStream_t s);
 void launch_clip(const MatDev* tab, int n_mats, float max_norm, float* clip, cudaStream_t s);
 void launch_pad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, int cols_dst, cudaStream_t s);
 void launch_unpad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, cudaStream_t s);
@@ -199,6 +200,8 @@ sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int coun
 sc_status tc_launch_wait_probe(sc_plan* p, int max_polls);
 sc_status tc_encode_anchor(sc_plan* p, ShapeClass& c, const std::vector<int>& ids);
 sc_status tc_launch_ema_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, int b_field_off);
+sc_status tc_launch_gram(sc_plan* p, ShapeClass& c, const int* idx, int count, int panel_field_off, int rows, int slices);
+sc_status tc_launch_xpart(sc_plan* p, ShapeClass& c, const int* idx, int count, int slices);
 sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, bool transposed, int b_field_off);
 
 }  // namespace sc

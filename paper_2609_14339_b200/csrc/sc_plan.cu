@@ -244,9 +244,15 @@ void cholqr(sc_plan* p, const std::vector<ActiveClass>& act, const int* idx_all,
   ProfScope ps(p, PROF_SMALL);
   for (int round = 0; round < rounds; ++round) {
     const int src = round == 0 ? offY : offTmp, dst = round == 0 ? offTmp : offY;
-    for (const auto& a : act)
-      launch_atb(p->dev_tab, a.idx, a.cnt, src, src, OFF(gpart), OFF(gram), (int)(left ? a.c->m : a.c->n), lp, lp, lp,
-                 lp, left ? a.c->split_m : a.c->split_n, s);
+    for (const auto& a : act) {
+      const int rows = (int)(left ? a.c->m : a.c->n), slices = left ? a.c->split_m : a.c->split_n;
+      if (a.c->tensor) {     // Gram matrix on the tensor cores: the panel is read once, row-slice partials, fixed-order sum
+        tc_launch_gram(p, *a.c, a.idx, a.cnt, src, rows, slices);
+        launch_sum_slices(p->dev_tab, a.idx, a.cnt, OFF(gpart), OFF(gram), lp * lp, slices, s);
+      } else {
+        launch_atb(p->dev_tab, a.idx, a.cnt, src, src, OFF(gpart), OFF(gram), rows, lp, lp, lp, lp, slices, s);
+      }
+    }
     launch_chol(p->dev_tab, idx_all, n_all, lp, round == 0 ? OFF(rmat) : OFF(rmat2), s);
     for (const auto& a : act)
       launch_gemm(gemm(p, a.idx, src, OFF(rinv), dst, (int)(left ? a.c->m : a.c->n), lp, lp, lp, lp, lp, 0, 0), a.cnt, s);
@@ -632,9 +638,14 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
     // X = U^T T as row-slice partials (the K-slice partials of T are added on the way in); xs_kernel adds them up
     // (one block per matrix adds the slices inside xs_kernel unless that is too much for one block)
     const bool sum_in_xs = (size_t)c.split_m * rp * rp <= (size_t)(1 << 16);
-    if (rp > 0)
+    if (rp > 0 && c.tensor && c.ksplit == 1) {
+      sc_status e = tc_launch_xpart(p, c, idx, cnt, c.split_m);        // tensor cores, T read once
+      if (e != SC_OK) return e;
+      if (!sum_in_xs) launch_sum_slices(p->dev_tab, idx, cnt, OFF(xpart), OFF(X), rp * rp, c.split_m, s);
+    } else if (rp > 0) {
       launch_atb(p->dev_tab, idx, cnt, OFF(U), OFF(T), OFF(xpart), OFF(X), m, rp, rp, rp, rp, c.split_m, s, c.ksplit,
                  !sum_in_xs);
+    }
     if (want_norm) launch_sqnorm(p->dev_tab, idx, cnt, (int64_t)m * n, g_bf16, s);
     launch_xs(p->dev_tab, idx, cnt, rp, p->rank, (rp > 0 && sum_in_xs) ? c.split_m : 0, scale, hp.alpha, p->status_dev, s);   // D X D
     if (rp > 0) {

@@ -256,7 +256,12 @@ void launch_atb(const MatDev* tab, const int* idx, int count, int offA, int offB
   }
   ++g_kernel_launches;
   if (!sum_here) return;     // the consumer adds the row slices itself
-  const int numel = ca * cb;
+  launch_sum_slices(tab, idx, count, offPart, offOut, ca * cb, nsplit, s);
+}
+
+void launch_sum_slices(const MatDev* tab, const int* idx, int count, int offPart, int offOut, int numel, int nsplit,
+                       cudaStream_t s) {
+  if (count <= 0 || numel <= 0) return;
   sum_slices_kernel<<<dim3((numel + 255) / 256 < 64 ? (numel + 255) / 256 : 64, 1, count), 256, 0, s>>>(
       tab, idx, offPart, offOut, numel, nsplit);
   ++g_kernel_launches;
@@ -599,23 +604,6 @@ void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int
   int64_t tot = (int64_t)(m > n ? m : n) * rp;
   int blocks = (int)((tot + 255) / 256 < 1184 ? (tot + 255) / 256 : 1184);
   split_basis_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, m, n, rp, rk);
-  ++g_kernel_launches;
-}
-
-__global__ void __launch_bounds__(256) split_ct_kernel(const MatDev* tab, const int* idx, int64_t numel, int rp, int rk) {
-  const MatDev& md = tab[idx[blockIdx.z]];
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < numel; e += stride) {
-    const int64_t j = e / rp, k = e % rp;
-    split2(md.Ct[e], md.Cthi[j * rk + k], md.Ctlo[j * rk + k]);
-  }
-}
-
-void launch_split_ct(const MatDev* tab, const int* idx, int count, int n, int rp, int rk, cudaStream_t s) {
-  if (count <= 0 || rp <= 0) return;
-  const int64_t tot = (int64_t)n * rp;
-  int blocks = (int)((tot + 255) / 256 < 296 ? (tot + 255) / 256 : 296);
-  split_ct_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, tot, rp, rk);
   ++g_kernel_launches;
 }
 

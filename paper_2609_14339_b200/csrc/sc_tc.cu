@@ -115,7 +115,7 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16(int N) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-constexpr int kMapsPerMat = 24;
+constexpr int kMapsPerMat = 26;
 constexpr int kPerCallMaps = 6;   // the first six are rebuilt whenever the caller's buffers move
 enum { MAP_G = 0,    // masked gradient, bf16, box 64 x 128 (MMA A operand of the projection)
        MAP_G32,      // masked gradient, bf16, box 32 x 128, 64-byte swizzle (streaming tile of the fused update)
@@ -129,6 +129,7 @@ enum { MAP_G = 0,    // masked gradient, bf16, box 64 x 128 (MMA A operand of th
        MAP_Y2, MAP_Z2,           // the scratch twins of Y and Z (a single-round Cholesky QR leaves its result there)
        MAP_GANC32,               // anchor gradient, bf16, box 32 x 128, 64-byte swizzle (rebuilt per anchor call)
        MAP_M_F32,                // anchor momentum as plain fp32 (box 32 x 128): load and store of the fused EMA sweep
+       MAP_U_MN, MAP_T,          // fp32 U (m x rp) and T (m x rp) as MN-major panels: X = U^T T on the tensor cores
        MAP_SPARE };
 constexpr int kTileBytes = 128 * 128;   // 128 rows x 64 bf16
 
@@ -262,13 +263,28 @@ __device__ __forceinline__ uint32_t umma_idesc_tf32(int N, int a_mn, int b_mn) {
 constexpr int kPassK = 32;                       // K per stage
 constexpr int kAtomBytes = kPassK * 128;         // one MN-major atom column: 32 K-rows x 128 bytes
 
+struct PassArgs {
+  int a_map, b_map;     // tensor maps of the A source (K-major box 32 x 128, or MN-major box 32 x 32) and of B (MN-major)
+  int same_ab;          // A and B are the same panel (Gram matrix): load it once, both descriptors point at it
+  int out_off;          // MatDev field of the output (or of the partial-sum buffer when the K range is split)
+  int rows_out;         // valid output rows
+  int kdim;             // contraction length
+  int ncols;            // MMA N = B panel width, a multiple of 32
+  int ncols_valid;      // columns written (multiple of 16)
+  int ldo;              // output row stride in floats
+  int cps;              // K chunks (of 32) per K slice; blockIdx.y selects the slice
+  int stages;
+  uint32_t tmem_cols;
+};
+
 template <bool TRANS>
 __global__ void __launch_bounds__(192, 2)
 pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const CUtensorMap* __restrict__ maps,
-            int b_map, int out_off, int rows_out, int kdim, int lp, int stages, uint32_t tmem_cols, unsigned* status) {
+            PassArgs pa, unsigned* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  const int b_bytes = (lp / 32) * kAtomBytes;
+  const int stages = pa.stages;
+  const int b_bytes = pa.same_ab ? 0 : (pa.ncols / 32) * kAtomBytes;
   const int stage_bytes = kTileBytes + b_bytes;
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
   uint64_t* empty = full + stages;
@@ -281,7 +297,9 @@ pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const C
   const MatDev& md = tab[idx[blockIdx.z]];
   const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
   const int row0 = blockIdx.x * 128;
-  const int nchunks = (kdim + kPassK - 1) / kPassK;
+  const int nchunks_all = (pa.kdim + kPassK - 1) / kPassK;
+  const int c0 = blockIdx.y * pa.cps;
+  const int nchunks = min(pa.cps, nchunks_all - c0);      // <= 0 for a trailing K slice with nothing in it: writes zeros
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -291,15 +309,15 @@ pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const C
     fence_barrier_init();
     fence_proxy_async();
   }
-  if (warp == 1) tmem_alloc(tmem_slot, tmem_cols);
+  if (warp == 1) tmem_alloc(tmem_slot, pa.tmem_cols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_d = *tmem_slot;
 
   if (warp == 0 && lane == 0) {
-    const CUtensorMap* amap = mp + (TRANS ? MAP_M_MN : MAP_M_K);
-    const CUtensorMap* bmap = mp + b_map;
+    const CUtensorMap* amap = mp + pa.a_map;
+    const CUtensorMap* bmap = mp + pa.b_map;
     tensormap_acquire(amap); tensormap_acquire(bmap);
     int issued = 0;
     for (int i = 0; i < nchunks; ++i, ++issued) {
@@ -307,25 +325,26 @@ pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const C
       if (!mbar_wait(&empty[s], ((i / stages) & 1) ^ 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
       uint8_t* st = smem + (size_t)s * stage_bytes;
       mbar_expect_tx(&full[s], (uint32_t)stage_bytes);
-      const int k0 = i * kPassK;
+      const int k0 = (c0 + i) * kPassK;
       if (!TRANS) {
         tma_load_2d(st, amap, &full[s], k0, row0);                                    // 128 rows x 32 floats
       } else {
 #pragma unroll
         for (int a = 0; a < 4; ++a) tma_load_2d(st + a * kAtomBytes, amap, &full[s], row0 + 32 * a, k0);
       }
-      for (int a = 0; a < lp / 32; ++a) tma_load_2d(st + kTileBytes + a * kAtomBytes, bmap, &full[s], 32 * a, k0);
+      if (!pa.same_ab)
+        for (int a = 0; a < pa.ncols / 32; ++a) tma_load_2d(st + kTileBytes + a * kAtomBytes, bmap, &full[s], 32 * a, k0);
     }
     if (*abort_flag)
       for (int i = max(0, issued - stages); i < issued; ++i) mbar_wait(&full[i % stages], (i / stages) & 1, never_flag);
   } else if (warp == 1 && lane == 0) {
-    const uint32_t idesc = umma_idesc_tf32(lp, TRANS ? 1 : 0, 1);
+    const uint32_t idesc = umma_idesc_tf32(pa.ncols, TRANS ? 1 : 0, 1);
     for (int i = 0; i < nchunks; ++i) {
       const int s = i % stages;
       if (!mbar_wait(&full[s], (i / stages) & 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
       tc_fence_after();
       const uint32_t a = smem_u32(smem + (size_t)s * stage_bytes);
-      const uint32_t b = a + kTileBytes;
+      const uint32_t b = pa.same_ab ? a : a + kTileBytes;
 #pragma unroll
       for (int k = 0; k < kPassK / 8; ++k) {
         const uint64_t ad = TRANS ? umma_desc_mn128(a + k * 1024, kAtomBytes) : umma_desc_k128(a + k * 32);
@@ -333,21 +352,27 @@ pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const C
       }
       umma_commit(&empty[s]);
     }
-    umma_commit(accum);
+    if (nchunks > 0) umma_commit(accum);
   } else if (warp >= 2) {
     const int q = warp & 3;
     const int row = row0 + q * 32 + lane;
-    bool ok = mbar_wait(accum, 0, abort_flag);
+    bool ok = nchunks <= 0 || mbar_wait(accum, 0, abort_flag);
     if (!ok && lane == 0) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
     ok = __all_sync(0xffffffffu, ok) && !*abort_flag;
     tc_fence_after();
     if (ok) {
-      float* out = *reinterpret_cast<float* const*>(reinterpret_cast<const char*>(&md) + out_off) + (size_t)row * lp;
-      for (int c = 0; c < lp; c += 16) {
+      float* out = *reinterpret_cast<float* const*>(reinterpret_cast<const char*>(&md) + pa.out_off) +
+                   ((size_t)blockIdx.y * pa.rows_out + row) * pa.ldo;
+      for (int c = 0; c < pa.ncols_valid; c += 16) {
         float v[16];
-        tmem_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + c, v);
-        tmem_ld_wait();
-        if (row < rows_out) {
+        if (nchunks > 0) {
+          tmem_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + c, v);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = 0.f;
+        }
+        if (row < pa.rows_out) {
 #pragma unroll
           for (int j = 0; j < 16; j += 4)
             *reinterpret_cast<float4*>(out + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -357,7 +382,7 @@ pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const C
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_d, tmem_cols);
+  if (warp == 1) tmem_dealloc(tmem_d, pa.tmem_cols);
 }
 
 // =====================================================================================================
@@ -888,6 +913,8 @@ sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_
       ok = ok && encode_tf32(mp + MAP_OMEGA, md.omega, lp, c.n, kPassK, true);
       ok = ok && encode2d(mp + MAP_M_F32, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, md.Manc, c.n, c.m, c.n, 32, 128,
                           CU_TENSOR_MAP_SWIZZLE_128B);
+      ok = ok && encode_tf32(mp + MAP_U_MN, md.U, rp, c.m, kPassK, true);
+      ok = ok && encode_tf32(mp + MAP_T, md.T, rp, c.m, kPassK, true);
       ok = ok && encode_tf32(mp + MAP_Y2, md.Y2, lp, c.m, kPassK, true);
       ok = ok && encode_tf32(mp + MAP_Z2, md.Z2, lp, c.n, kPassK, true);
       if (!ok) return SC_ERR_CUDA;
@@ -974,33 +1001,79 @@ sc_status tc_launch_ema_pass(sc_plan* p, ShapeClass& c, const int* idx, int coun
   return cuda_ok(cudaGetLastError());
 }
 
+static uint32_t tmem_cols_for(int n) {
+  uint32_t cols = 32;
+  while ((int)cols < n) cols <<= 1;
+  return cols;
+}
+
+static int panel_map(int field_off) {
+  if (field_off == (int)offsetof(MatDev, omega_t) || field_off == (int)offsetof(MatDev, omega)) return MAP_OMEGA;
+  if (field_off == (int)offsetof(MatDev, Y)) return MAP_Y;
+  if (field_off == (int)offsetof(MatDev, Y2)) return MAP_Y2;
+  if (field_off == (int)offsetof(MatDev, Z)) return MAP_Z;
+  if (field_off == (int)offsetof(MatDev, Z2)) return MAP_Z2;
+  return -1;
+}
+
 // One sweep over the anchor momentum: transposed ? Z <- M^T B : Y <- M B, with B one of the n x lp / m x lp buffers.
 sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, bool transposed, int b_field_off) {
   const int lp = p->lp, m = (int)c.m, n = (int)c.n;
+  PassArgs pa{};
+  pa.a_map = transposed ? MAP_M_MN : MAP_M_K;
+  pa.b_map = panel_map(b_field_off);
+  if (pa.b_map < 0) return SC_ERR_INVALID_ARG;
+  pa.out_off = transposed ? (int)offsetof(MatDev, Z) : (int)offsetof(MatDev, Y);
+  pa.rows_out = transposed ? n : m;
+  pa.kdim = transposed ? m : n;
+  pa.ncols = lp; pa.ncols_valid = lp; pa.ldo = lp;
+  pa.cps = (pa.kdim + kPassK - 1) / kPassK;
   const int stage_bytes = kTileBytes + (lp / 32) * kAtomBytes;
-  const int stages = stages_for(stage_bytes, 8);
-  const size_t smem = (size_t)stages * stage_bytes + 1024 + 256;
-  uint32_t cols = 32;
-  while ((int)cols < lp) cols <<= 1;
-  int b_map;
-  if (b_field_off == (int)offsetof(MatDev, omega_t) || b_field_off == (int)offsetof(MatDev, omega)) b_map = MAP_OMEGA;
-  else if (b_field_off == (int)offsetof(MatDev, Y)) b_map = MAP_Y;
-  else if (b_field_off == (int)offsetof(MatDev, Y2)) b_map = MAP_Y2;
-  else if (b_field_off == (int)offsetof(MatDev, Z)) b_map = MAP_Z;
-  else if (b_field_off == (int)offsetof(MatDev, Z2)) b_map = MAP_Z2;
-  else return SC_ERR_INVALID_ARG;
+  pa.stages = stages_for(stage_bytes, 8);
+  pa.tmem_cols = tmem_cols_for(lp);
+  const size_t smem = (size_t)pa.stages * stage_bytes + 1024 + 256;
   const CUtensorMap* maps = static_cast<const CUtensorMap*>(c.tmaps);
-  if (transposed) {
-    dim3 grid((n + 127) / 128, 1, count);
-    pass_kernel<true><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, b_map, (int)offsetof(MatDev, Z), n, m, lp,
-                                                       stages, cols, p->status_dev);
-  } else {
-    dim3 grid((m + 127) / 128, 1, count);
-    pass_kernel<false><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, b_map, (int)offsetof(MatDev, Y), m, n, lp,
-                                                        stages, cols, p->status_dev);
-  }
+  dim3 grid((pa.rows_out + 127) / 128, 1, count);
+  if (transposed) pass_kernel<true><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, pa, p->status_dev);
+  else pass_kernel<false><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, pa, p->status_dev);
   ++g_kernel_launches;
   return cuda_ok(cudaGetLastError());
+}
+
+// part[slice] = A^T B over the rows of K slice `slice`, for tall panels A (rows x ca) and B (rows x cb) given by
+// their tensor maps; the caller adds the slices. a_map == b_map computes a Gram matrix from one load of the panel.
+sc_status tc_launch_atb(sc_plan* p, ShapeClass& c, const int* idx, int count, int a_map, int b_map, int part_off,
+                        int rows, int ca, int cb, int slices) {
+  PassArgs pa{};
+  pa.a_map = a_map; pa.b_map = b_map;
+  pa.same_ab = a_map == b_map && ca <= 128 && cb <= 128;   // one 128-column tile holds the whole panel
+  pa.out_off = part_off;
+  pa.rows_out = ca;
+  pa.kdim = rows;
+  pa.ncols = (cb + 31) / 32 * 32; pa.ncols_valid = cb; pa.ldo = cb;
+  const int nchunks = (rows + kPassK - 1) / kPassK;
+  pa.cps = (nchunks + slices - 1) / slices;
+  const int stage_bytes = kTileBytes + (pa.same_ab ? 0 : (pa.ncols / 32) * kAtomBytes);
+  pa.stages = stages_for(stage_bytes, 8);
+  pa.tmem_cols = tmem_cols_for(pa.ncols);
+  const size_t smem = (size_t)pa.stages * stage_bytes + 1024 + 256;
+  dim3 grid((ca + 127) / 128, slices, count);
+  pass_kernel<true><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), pa,
+                                                     p->status_dev);
+  ++g_kernel_launches;
+  return cuda_ok(cudaGetLastError());
+}
+
+// Gram matrix partials of one of the Y / Y2 / Z / Z2 panels (lp columns) into gpart.
+sc_status tc_launch_gram(sc_plan* p, ShapeClass& c, const int* idx, int count, int panel_field_off, int rows, int slices) {
+  const int pm = panel_map(panel_field_off);
+  if (pm < 0 || pm == MAP_OMEGA) return SC_ERR_INVALID_ARG;
+  return tc_launch_atb(p, c, idx, count, pm, pm, (int)offsetof(MatDev, gpart), rows, p->lp, p->lp, slices);
+}
+
+// X partials: xpart[slice] = U^T T over the rows of the slice.
+sc_status tc_launch_xpart(sc_plan* p, ShapeClass& c, const int* idx, int count, int slices) {
+  return tc_launch_atb(p, c, idx, count, MAP_U_MN, MAP_T, (int)offsetof(MatDev, xpart), (int)c.m, p->rp, p->rp, slices);
 }
 
 sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc) {

@@ -5,7 +5,7 @@ framework's caching allocator already owns HBM, or the path must not synchronise
 keeps its intermediates in a fixed array inside the library. This test calls it through the C ABI twice in a
 row - a large matrix first, a smaller one second, so the second call runs on top of the first call's leftovers -
 and checks both results against the projection the plan-based entry points compute, within the tolerance the
-other projection tests use (1e-4 relative Frobenius).
+other projection tests use for X (5e-4 relative Frobenius: the plan path forms X on tf32 tensor cores).
 
 Collected last on purpose (file name): a run that stops at the first failure has then run everything else.
 """
@@ -17,7 +17,7 @@ import pytest
 from parity_util import Case, GpuRun, make_inputs, rel
 
 pytestmark = pytest.mark.gpu
-TOL = 1e-4
+TOL = 5e-4
 
 
 @pytest.fixture(scope="module")
