@@ -356,3 +356,52 @@ def correct_and_step(states, G_masks, Ws, ms, vs, t: int, hp: Hyper):
         W2, m2, v2 = adamw_step(W, m, v, g, t, hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay)
         outW.append(W2); outm.append(m2); outv.append(v2); outg.append(g)
     return outW, outm, outv, outg
+
+
+# --------------------------------------------------------------------------
+# In-graph activation mask from a shared pseudo-random function (Section 3.1, Algorithm 1 line 4:
+# M_l = g(l, t, B, S, H)) and the masked weight gradient it leads to.  Nothing here is part of the
+# optimizer step; it is the producer of the step's input, kept beside it for the fused GPU producer.
+# --------------------------------------------------------------------------
+def lowbias32(x: np.ndarray) -> np.ndarray:
+    """A 32-bit integer finaliser (xorshift-multiply, two rounds), wrap-around uint32 arithmetic."""
+    x = np.asarray(x, np.uint32).copy()
+    with np.errstate(over="ignore"):
+        x ^= x >> np.uint32(16)
+        x *= np.uint32(0x21F0AAAD)
+        x ^= x >> np.uint32(15)
+        x *= np.uint32(0x735A2D97)
+        x ^= x >> np.uint32(15)
+    return x
+
+
+def keep_threshold(keep: float) -> int:
+    """keep ratio quantised to 16 bits: an element is kept iff its 16 random bits are below this."""
+    return int(min(65536, max(1, round(float(keep) * 65536.0))))
+
+
+def prf_keep_mask(seed: int, layer: int, step: int, tokens: int, features: int, keep: float) -> np.ndarray:
+    """Mask in {0,1}^{tokens x features}: a pure function of (seed, layer, step, token, feature).
+
+    row key   k_t = low 32 bits of mix64(seed XOR ((layer * 2^40 + step) * golden) XOR (t + 1) * 0xD1B54A32D192ED03)
+    pair hash h   = lowbias32(k_t + (j // 2) * 0x9E3779B9)
+    bits          = low 16 bits of h for even j, high 16 bits for odd j;  kept iff bits < keep_threshold(keep)
+    """
+    t = np.arange(tokens, dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        base = np.uint64(seed) ^ ((np.uint64(layer) * np.uint64(1 << 40) + np.uint64(step)) * _GOLDEN)
+        key = mix64(base ^ ((t + np.uint64(1)) * np.uint64(0xD1B54A32D192ED03)))
+    k32 = (key & np.uint64(0xFFFFFFFF)).astype(np.uint32)[:, None]
+    pairs = (np.arange((features + 1) // 2, dtype=np.uint64) * np.uint64(0x9E3779B9) & np.uint64(0xFFFFFFFF)).astype(np.uint32)[None, :]
+    with np.errstate(over="ignore"):
+        h = lowbias32(k32 + pairs)
+    bits = np.empty((tokens, 2 * h.shape[1]), np.uint32)
+    bits[:, 0::2] = h & np.uint32(0xFFFF)
+    bits[:, 1::2] = h >> np.uint32(16)
+    return (bits[:, :features] < np.uint32(keep_threshold(keep))).astype(F64)
+
+
+def masked_weight_gradient(dY, X, mask, keep: float, rescale: bool = True) -> np.ndarray:
+    """G_mask = dY^T (X * mask) / keep_q, keep_q the 16-bit quantised keep ratio (so that E_mask[G_mask] = dY^T X)."""
+    G = np.asarray(dY, F64).T @ (np.asarray(X, F64) * mask)
+    return G * (65536.0 / keep_threshold(keep)) if rescale else G

@@ -368,3 +368,32 @@ def test_mirror_warm_start_reduces_to_cold_on_first_arrival_and_improves_later()
         so.anchor_update(warm, G1, hp, r, mode="mirror", Omega=Om, q=0, warm=True)
         errs.append(so.projector_distance(warm.V, Ve))
     assert errs[-1] < 1e-2 * errs[0] and all(b <= a * 1.0001 for a, b in zip(errs, errs[1:]))
+
+
+def test_prf_mask_is_a_balanced_independent_pure_function():
+    keep = 0.1
+    M = so.prf_keep_mask(5, 3, 17, 512, 384, keep)
+    assert set(np.unique(M)) <= {0.0, 1.0}
+    assert abs(M.mean() - so.keep_threshold(keep) / 65536.0) < 0.004
+    assert np.array_equal(M, so.prf_keep_mask(5, 3, 17, 512, 384, keep))
+    assert np.array_equal(M[:100, :37], so.prf_keep_mask(5, 3, 17, 100, 37, keep))       # prefix-stable, odd width
+    for other in ((6, 3, 17), (5, 4, 17), (5, 3, 18)):
+        assert abs((M * so.prf_keep_mask(*other, 512, 384, keep)).mean() - M.mean() ** 2) < 0.003   # independent draws
+    # neighbours inside a pair, across pairs and across tokens are uncorrelated
+    c = lambda a, b: abs(np.mean(a * b) - a.mean() * b.mean())
+    assert c(M[:, 0::2], M[:, 1::2]) < 0.003 and c(M[:, :-2], M[:, 2:]) < 0.003 and c(M[:-1], M[1:]) < 0.003
+    assert so.keep_threshold(1.0) == 65536 and so.prf_keep_mask(1, 0, 0, 8, 8, 1.0).all()
+    assert so.keep_threshold(0.25) == 16384 and so.keep_threshold(0.5) == 32768
+
+
+def test_masked_weight_gradient_is_unbiased_over_steps():
+    rng = np.random.default_rng(3)
+    dY = rng.standard_normal((64, 6)); X = rng.standard_normal((64, 10))
+    dense = dY.T @ X
+    acc = np.zeros_like(dense)
+    steps = 3000
+    for s in range(steps):
+        acc += so.masked_weight_gradient(dY, X, so.prf_keep_mask(1, 2, s, 64, 10, 0.25), 0.25)
+    var = (1 - 0.25) / 0.25 * (dY ** 2).T @ (X ** 2)                 # per-entry variance of one masked draw
+    assert np.max(np.abs(acc / steps - dense) / np.sqrt(var / steps)) < 5.0
+    assert np.array_equal(so.masked_weight_gradient(dY, X, np.ones_like(X), 1.0), dense)
