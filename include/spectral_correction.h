@@ -177,6 +177,15 @@ SC_API sc_status sc_correct_and_step_host(sc_plan* plan, const void* const* host
                                           void* const* params, const sc_opt_state* state, int64_t step,
                                           sc_mat_stats* stats_out, float* clip_out);
 
+/* sc_apply_prf_mask - the in-graph activation mask of Section 3.1 / Algorithm 1 line 4: out = X * M (times
+ * 65536 / round(keep * 65536) when rescale != 0), M a pure function of (seed, layer, step, token, feature), so every
+ * pipeline stage regenerates it and nothing is transmitted. Stand-alone (no plan).
+ *   X_dev, out_dev   device: tokens x features bf16 row-major, 16-byte aligned (out may alias X); features % 8 == 0
+ *   keep             keep ratio 1 - p_mask in (0, 1], quantised to 16 bits
+ * The masked weight gradient of the step is then the plain product dY^T out. */
+SC_API sc_status sc_apply_prf_mask(const void* X_dev, void* out_dev, int64_t tokens, int64_t features, float keep,
+                                   uint64_t seed, uint32_t layer, uint64_t step, int rescale, void* stream);
+
 /* ---- inspection / test hooks ------------------------------------------------------------------------- */
 
 /* Copy matrix `mat`'s cached basis into caller device buffers (any may be NULL):
