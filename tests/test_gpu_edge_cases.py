@@ -1,0 +1,149 @@
+"""Degenerate and boundary cases of the method on the GPU, both engines, against the oracle."""
+import numpy as np
+import pytest
+
+from oracle import spectral_oracle as so
+from parity_util import Case, GpuRun, OracleRun, compare_basis, compare_step, make_inputs, make_plan, rel, to_dev
+from synth import generator as gen
+
+pytestmark = pytest.mark.gpu
+ENGINES = [0, 1]
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    return torch
+
+
+def _tol(engine):
+    return 2e-3 if engine == 0 else 2e-5
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_zero_anchor_gradient_gives_an_empty_basis(torch, engine):
+    """G_anc = 0 -> M = 0 -> every direction is dropped: s = d = 0 and G_proj = alpha g, nothing non-finite."""
+    case = Case(shapes=[(256, 384)], rank=16, tokens=128, engine=engine)
+    inp = make_inputs(case)
+    inp["anchors"][0][0] = np.zeros_like(inp["anchors"][0][0])
+    g = GpuRun(case, inp, torch)
+    assert g.dev_status == 0
+    U, s, V = g.basis[0]
+    assert np.all(s == 0) and np.all(np.isfinite(U)) and np.all(np.isfinite(V))
+    G = gen.stored_to_f64(inp["G"][0], case.dtype)
+    assert rel(g.gproj[0], 0.3 * G) < 1e-6
+    assert np.all(np.isfinite(g.W[0]))
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_rank_deficient_anchor_momentum(torch, engine):
+    """rank(M) = 3 < r = 8: the five missing directions are dropped (s = 0, d = 0); the rest matches the exact SVD."""
+    rng = np.random.default_rng(4)
+    m, n, true_rank = 256, 384, 3
+    # small-integer factors and beta_anc = 1/2: G_anc and M are exact in bf16 / fp32, so the rank really is 3
+    Ganc = (rng.integers(-2, 3, (m, true_rank)) @ rng.integers(-2, 3, (true_rank, n))).astype(np.float32)
+    case = Case(shapes=[(m, n)], rank=8, tokens=128, tau_p=0.5, beta_anc=0.5, engine=engine, q=2)
+    inp = make_inputs(case)
+    inp["anchors"][0][0] = gen.round_to(Ganc, case.dtype)
+    g = GpuRun(case, inp, torch)
+    assert g.dev_status == 0
+    U, s, V = g.basis[0]
+    assert np.all(s[true_rank:] == 0) and np.all(s[:true_rank] > 0)
+    assert np.all(U[:, true_rank:] == 0)
+    oe = OracleRun(case, inp, "exact")
+    st = oe.states[0]
+    tol = _tol(engine) * 5
+    assert rel(s[:true_rank], st.s[:true_rank]) < tol
+    assert so.projector_distance(U[:, :true_rank], st.U[:, :true_rank]) < tol
+    assert so.projector_distance(V[:, :true_rank], st.V[:, :true_rank]) < tol
+    # the exact SVD's trailing singular values are ~1e-13, its d = s/(s+tau) ~ 0 there: G_proj agrees
+    es = compare_step(g, oe)
+    assert max(es["gproj"], es["m"], es["dW"]) < tol, es
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("alpha", [0.0, 1.0])
+def test_blend_limits_on_the_gpu(torch, engine, alpha):
+    case = Case(shapes=[(256, 384)], rank=16, tokens=128, alpha=alpha, tau_p=20.0, engine=engine)
+    inp = make_inputs(case)
+    g = GpuRun(case, inp, torch)
+    o = OracleRun(case, inp, "mirror")
+    if alpha == 1.0:                                   # masked-only training: the gradient passes through untouched
+        assert np.array_equal(g.gproj[0], gen.stored_to_f64(inp["G"][0], case.dtype))
+    es = compare_step(g, o)
+    assert max(es["gproj"], es["m"], es["v"], es["dW"]) < _tol(engine), es
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_keep_one_and_full_rank_is_the_identity(torch, engine):
+    """keep = 1 (no masking), r = min(m, n) on a square matrix, tau_p = 0: P = I, so G_proj = g for any alpha."""
+    case = Case(shapes=[(64, 64)], rank=64, tokens=256, keep=1.0, tau_p=0.0, engine=engine, q=2)
+    inp = make_inputs(case)
+    g = GpuRun(case, inp, torch)
+    assert g.dev_status == 0
+    G = gen.stored_to_f64(inp["G"][0], case.dtype)
+    assert rel(g.gproj[0], G) < (1e-3 if engine == 0 else 1e-4)
+
+
+def test_smaller_than_one_tile_on_the_tensor_engine(torch):
+    """Matrices smaller than the 128-row / 64-column tiles: everything is TMA out-of-bounds fill and clipped stores."""
+    case = Case(shapes=[(16, 64), (40, 72), (129, 200)], rank=8, tokens=96, tau_p=10.0, planted=2)
+    inp = make_inputs(case)
+    g = GpuRun(case, inp, torch)
+    assert g.uses_tc and g.dev_status == 0
+    o = OracleRun(case, inp, "mirror")
+    eb, es = compare_basis(g, o), compare_step(g, o)
+    assert max(eb["PU"], eb["PV"], eb["s"]) < 2e-3, eb
+    assert max(es["gproj"], es["m"], es["v"], es["dW"]) < 2e-3, es
+
+
+def test_two_plans_on_two_streams_do_not_interfere(torch):
+    case = Case(shapes=[(256, 384), (384, 256)], rank=16, tokens=128, planted=4, tau_p=20.0)
+    inp = make_inputs(case)
+    ref = GpuRun(case, inp, torch)
+    import paper_2609_14339_b200 as sc
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    plans, bufs = [], []
+    for st in streams:
+        hp = sc.Hparams.default(tau_p=20.0, lr=1e-2, weight_decay=0.01, collect_stats=1)
+        plans.append(sc.Plan(case.shapes, 16, case.keep, hp, stream=st))
+    torch.cuda.synchronize()
+    for plan, st in zip(plans, streams):
+        with torch.cuda.stream(st):
+            n = len(case.shapes)
+            A = [to_dev(inp["anchors"][i][0], "bf16", torch, "cuda:0") for i in range(n)]
+            G = [to_dev(inp["G"][i], "bf16", torch, "cuda:0") for i in range(n)]
+            W = [torch.from_numpy(inp["W"][i].copy()).cuda() for i in range(n)]
+            m = [torch.from_numpy(inp["m"][i].copy()).cuda() for i in range(n)]
+            v = [torch.from_numpy(inp["v"][i].copy()).cuda() for i in range(n)]
+            plan.anchor_update(A, 0)
+            plan.correct_and_step(G, W, m, v, 100)
+            bufs.append((A, G, W, m, v))
+    torch.cuda.synchronize()
+    for (_, _, W, m, v) in bufs:
+        for i in range(len(case.shapes)):
+            assert np.array_equal(W[i].double().cpu().numpy(), ref.W[i]) and np.array_equal(m[i].double().cpu().numpy(), ref.m[i])
+
+
+def test_many_steps_stay_deterministic_and_finite(torch):
+    """Ten steps with an anchor arrival every third step, run twice: bit-identical (fixed-order reductions)."""
+    case = Case(shapes=[(256, 384), (200, 136)], rank=12, tokens=128, planted=4, tau_p=20.0, warm=True)
+    inp = make_inputs(case)
+    outs = []
+    for _ in range(2):
+        plan = make_plan(case, torch)
+        n = len(case.shapes)
+        A = [to_dev(inp["anchors"][i][0], "bf16", torch, "cuda:0") for i in range(n)]
+        G = [to_dev(inp["G"][i], "bf16", torch, "cuda:0") for i in range(n)]
+        W = [torch.from_numpy(inp["W"][i].copy()).cuda() for i in range(n)]
+        m = [torch.from_numpy(inp["m"][i].copy()).cuda() for i in range(n)]
+        v = [torch.from_numpy(inp["v"][i].copy()).cuda() for i in range(n)]
+        for t in range(10):
+            if t % 3 == 0:
+                plan.anchor_update(A, t)
+            plan.correct_and_step(G, W, m, v, 100 + t)
+        torch.cuda.synchronize()
+        assert plan.get_device_status() == 0
+        outs.append([x.clone() for x in W + m + v])
+    assert all(torch.equal(a, b) for a, b in zip(*outs))
+    assert all(bool(torch.isfinite(x).all()) for x in outs[0])
