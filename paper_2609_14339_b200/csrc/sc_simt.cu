@@ -396,13 +396,19 @@ void launch_sketch_rowmajor(float* omega, int64_t rows, int width, uint64_t seed
 // A pivot that has cancelled to (numerically) nothing marks a column that lies in the span of the earlier
 // ones: that direction is dropped (its column of R^-1 is zero) instead of dividing by ~0.
 // =====================================================================================================
+// kSmem: the factor and its inverse are built in shared memory (2 lp^2 floats, lp <= 128) and copied out at the end;
+// otherwise they are built in place in global memory.
+template <bool kSmem>
 __global__ void __launch_bounds__(256) chol_kernel(const MatDev* tab, const int* idx, int lp, int offR) {
+  extern __shared__ __align__(16) float chol_smem[];
   __shared__ float invd[kMaxRank];
   __shared__ float piv_inv;
   const MatDev& md = tab[idx[blockIdx.x]];
   const float* G = md.gram;
-  float* R = field<float>(md, offR);
-  float* Ri = md.rinv;
+  float* Rg = field<float>(md, offR);
+  float* Rig = md.rinv;
+  float* R = kSmem ? chol_smem : Rg;
+  float* Ri = kSmem ? chol_smem + (size_t)lp * lp : Rig;
   const int t = threadIdx.x;
   for (int j = 0; j < lp; ++j) {
     const int i = t;
@@ -452,11 +458,21 @@ __global__ void __launch_bounds__(256) chol_kernel(const MatDev* tab, const int*
       Ri[(size_t)i * lp + c] = -((s0 + s1) + (s2 + s3)) * invd[i];
     }
   }
+  if (kSmem) {
+    __syncthreads();
+    for (int e = t; e < lp * lp; e += 256) { Rg[e] = R[e]; Rig[e] = Ri[e]; }
+  }
 }
 
 void launch_chol(const MatDev* tab, const int* idx, int count, int lp, int offR, cudaStream_t s) {
   if (count <= 0 || lp <= 0) return;
-  chol_kernel<<<count, 256, 0, s>>>(tab, idx, lp, offR);
+  if (lp <= 128) {
+    const size_t smem = (size_t)2 * lp * lp * sizeof(float);
+    cudaFuncSetAttribute(chol_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 128 * 128 * 4);
+    chol_kernel<true><<<count, 256, smem, s>>>(tab, idx, lp, offR);
+  } else {
+    chol_kernel<false><<<count, 256, 0, s>>>(tab, idx, lp, offR);
+  }
   ++g_kernel_launches;
 }
 
@@ -469,14 +485,16 @@ void launch_chol(const MatDev* tab, const int* idx, int count, int lp, int offR,
 // =====================================================================================================
 constexpr int kJacobiThreads = 512;
 
+template <bool kSmem>
 __global__ void __launch_bounds__(kJacobiThreads) jacobi_kernel(const MatDev* tab, const int* idx, int lp, int rp,
                                                                 int rank, float tau_p) {
+  extern __shared__ __align__(16) float jac_smem[];   // kSmem: both l x l work arrays live here (lp <= 128)
   __shared__ float nrm[kMaxRank];
   __shared__ int order[kMaxRank];
   __shared__ int rotated;
   const MatDev& md = tab[idx[blockIdx.x]];
-  float* Kc = md.jk;
-  float* Jc = md.jv;
+  float* Kc = kSmem ? jac_smem : md.jk;
+  float* Jc = kSmem ? jac_smem + (size_t)lp * lp : md.jv;
   const float* R = md.racc;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kJacobiThreads / 32;
   for (int e = tid; e < lp * lp; e += kJacobiThreads) {
@@ -558,7 +576,13 @@ __global__ void __launch_bounds__(kJacobiThreads) jacobi_kernel(const MatDev* ta
 void launch_jacobi(const MatDev* tab, const int* idx, int count, int lp, int rp, int rank, float tau_p,
                    cudaStream_t s) {
   if (count <= 0 || lp <= 0 || rp <= 0) return;
-  jacobi_kernel<<<count, kJacobiThreads, 0, s>>>(tab, idx, lp, rp, rank, tau_p);
+  if (lp <= 128) {
+    const size_t smem = (size_t)2 * lp * lp * sizeof(float);
+    cudaFuncSetAttribute(jacobi_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 128 * 128 * 4);
+    jacobi_kernel<true><<<count, kJacobiThreads, smem, s>>>(tab, idx, lp, rp, rank, tau_p);
+  } else {
+    jacobi_kernel<false><<<count, kJacobiThreads, 0, s>>>(tab, idx, lp, rp, rank, tau_p);
+  }
   ++g_kernel_launches;
 }
 

@@ -332,7 +332,8 @@ ema_pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, con
     if (lane == 0) {
       const CUtensorMap* bmap = mp + b_map;
       tensormap_acquire(mp + MAP_M_F32); tensormap_acquire(mp + MAP_GANC32); tensormap_acquire(bmap);
-      for (int i = 0; i < nchunks; ++i) {
+      int issued = 0;
+      for (int i = 0; i < nchunks; ++i, ++issued) {
         const int s = i % stages;
         if (!mbar_wait(&empty[s], ((i / stages) & 1) ^ 1, abort_flag)) { atomicOr(status, kDevTimeout); *abort_flag = 1; break; }
         uint8_t* st = smem + (size_t)s * stage_bytes;
@@ -342,6 +343,10 @@ ema_pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, con
         tma_load_2d(st + kTileBytes, mp + MAP_GANC32, &full[s], k0, row0);
         for (int a = 0; a < lp / 32; ++a)
           tma_load_2d(st + kTileBytes + kGancTile + a * kAtomBytes, bmap, &full[s], 32 * a, k0);
+      }
+      if (*abort_flag) {   // let the copies already in flight land before the block's shared memory goes away
+        volatile int never = 0;
+        for (int i = max(0, issued - stages); i < issued; ++i) mbar_wait(&full[i % stages], (i / stages) & 1, &never);
       }
     }
     __syncwarp();
@@ -570,7 +575,15 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
           }
         }
       }
-      if (dead) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
+      if (dead) {
+        atomicOr(status, kDevTimeout);
+        *abort_flag = 1;
+        // let the copies already in flight land before this block's shared memory goes away (bounded waits)
+        volatile int never = 0;
+        for (uint32_t u = unit_it > kStreamStages ? unit_it - kStreamStages : 0; u < unit_it; ++u)
+          mbar_wait(&bars->full[u % kStreamStages], (u / kStreamStages) & 1, &never);
+        if (op_it > 0) mbar_wait(&bars->opnd_full, (op_it - 1) & 1, &never);
+      }
     }
     __syncwarp();
   } else if (warp == 1) {
