@@ -21,6 +21,8 @@
  *     says otherwise, are owned by the caller, must be 16-byte aligned and must stay valid until the
  *     work queued on the plan's stream has finished.
  *   - All calls queue work on the stream given to sc_plan_create and return without waiting for it.
+ *   - A plan is not thread-safe: calls on ONE plan must come from one thread at a time. Different plans (on the
+ *     same or different streams) are independent.
  *   - Every function returns an sc_status; nothing throws or aborts across this boundary.
  *     Conditions the device detects (a bounded wait that ran out, non-finite values) are latched in a
  *     status word that sc_get_device_status reads back.

@@ -6,6 +6,7 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <vector>
 
 #include "spectral_correction.h"
@@ -147,7 +148,7 @@ struct sc_plan {
 namespace sc {
 
 // ---- host helpers (sc_plan.cu) -------------------------------------------------------------------------
-extern long long g_kernel_launches;   // kernels this library has launched in this process (all plans)
+extern std::atomic<long long> g_kernel_launches;   // kernels this library has launched in this process (all plans)
 sc_status upload_table(sc_plan* p);
 sc_status cuda_ok(cudaError_t e);
 

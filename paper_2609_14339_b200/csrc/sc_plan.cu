@@ -279,7 +279,7 @@ sc_status check_ptr_array(const void* const* arr, int n, bool allow_null_entries
 
 namespace sc {
 
-long long g_kernel_launches = 0;
+std::atomic<long long> g_kernel_launches{0};
 
 sc_status cuda_ok(cudaError_t e) { return e == cudaSuccess ? SC_OK : SC_ERR_CUDA; }
 
@@ -933,7 +933,7 @@ sc_status sc_get_profile(sc_plan* p, sc_profile* out) {
   return SC_OK;
 }
 
-int64_t sc_kernel_launch_count(void) { return (int64_t)g_kernel_launches; }
+int64_t sc_kernel_launch_count(void) { return (int64_t)g_kernel_launches.load(); }
 
 int sc_plan_uses_tensor_cores(const sc_plan* p) { return p && p->tensor_any ? 1 : 0; }
 
