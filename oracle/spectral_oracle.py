@@ -405,3 +405,29 @@ def masked_weight_gradient(dY, X, mask, keep: float, rescale: bool = True) -> np
     """G_mask = dY^T (X * mask) / keep_q, keep_q the 16-bit quantised keep ratio (so that E_mask[G_mask] = dY^T X)."""
     G = np.asarray(dY, F64).T @ (np.asarray(X, F64) * mask)
     return G * (65536.0 / keep_threshold(keep)) if rescale else G
+
+
+def prf_exact_k_mask(seed: int, layer: int, step: int, tokens: int, features: int, keep: float) -> np.ndarray:
+    """The per-token variant of the shared-PRF mask (Section 3.1: "retaining K = round((1-p) H) dimensions per
+    token"): every token keeps exactly K features, those with the K smallest composite keys
+        key(t, j) = lowbias32(k_t + j * 0x9E3779B9) * 2^16 + j        (k_t as in prf_keep_mask; j < 65536),
+    which are distinct by construction, so the selection is unique.
+    """
+    K = exact_k(features, keep)
+    t = np.arange(tokens, dtype=np.uint64)
+    with np.errstate(over="ignore"):
+        base = np.uint64(seed) ^ ((np.uint64(layer) * np.uint64(1 << 40) + np.uint64(step)) * _GOLDEN)
+        key = mix64(base ^ ((t + np.uint64(1)) * np.uint64(0xD1B54A32D192ED03)))
+    k32 = (key & np.uint64(0xFFFFFFFF)).astype(np.uint32)[:, None]
+    j = np.arange(features, dtype=np.uint64)
+    jm = ((j * np.uint64(0x9E3779B9)) & np.uint64(0xFFFFFFFF)).astype(np.uint32)[None, :]
+    with np.errstate(over="ignore"):
+        h = lowbias32(k32 + jm)
+    comp = (h.astype(np.uint64) << np.uint64(16)) | j[None, :]
+    kth = np.partition(comp, K - 1, axis=1)[:, K - 1:K]
+    return (comp <= kth).astype(F64)
+
+
+def exact_k(features: int, keep: float) -> int:
+    """K = round(keep * H), at least 1 and at most H."""
+    return int(min(features, max(1, round(float(keep) * features))))

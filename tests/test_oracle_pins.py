@@ -397,3 +397,17 @@ def test_masked_weight_gradient_is_unbiased_over_steps():
     var = (1 - 0.25) / 0.25 * (dY ** 2).T @ (X ** 2)                 # per-entry variance of one masked draw
     assert np.max(np.abs(acc / steps - dense) / np.sqrt(var / steps)) < 5.0
     assert np.array_equal(so.masked_weight_gradient(dY, X, np.ones_like(X), 1.0), dense)
+
+
+def test_exact_k_mask_keeps_exactly_k_per_token_and_is_unbiased():
+    H, T, keep = 200, 300, 0.1
+    M = so.prf_exact_k_mask(4, 1, 9, T, H, keep)
+    K = so.exact_k(H, keep)
+    assert K == 20 and np.all(M.sum(axis=1) == K)                       # exactly K per token
+    assert np.array_equal(M, so.prf_exact_k_mask(4, 1, 9, T, H, keep))
+    assert not np.array_equal(M, so.prf_exact_k_mask(4, 1, 10, T, H, keep))
+    # every feature is kept with probability K/H: column means over many tokens
+    big = so.prf_exact_k_mask(4, 1, 9, 4000, H, keep)
+    assert np.max(np.abs(big.mean(axis=0) - K / H)) < 5 * np.sqrt(0.1 * 0.9 / 4000)
+    assert so.exact_k(4096, 0.05) == 205 and so.exact_k(8, 0.01) == 1 and so.exact_k(8, 1.0) == 8
+    assert so.prf_exact_k_mask(1, 0, 0, 5, 8, 1.0).all()
