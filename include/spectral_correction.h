@@ -188,6 +188,14 @@ SC_API sc_status sc_correct_and_step_host(sc_plan* plan, const void* const* host
 SC_API sc_status sc_apply_prf_mask(const void* X_dev, void* out_dev, int64_t tokens, int64_t features, float keep,
                                    uint64_t seed, uint32_t layer, uint64_t step, int rescale, void* stream);
 
+/* sc_apply_prf_mask_exact_k - the per-token form of the same mask (Section 3.1: "retaining K = round((1 - p) H)
+ * dimensions per token"): every token keeps exactly K = round(keep * features) features, chosen by the K smallest
+ * values of a per-(token, feature) hash (ties impossible by construction); rescale multiplies by features / K.
+ * Same layouts as sc_apply_prf_mask; features <= 65536, no multiple-of-8 requirement. */
+SC_API sc_status sc_apply_prf_mask_exact_k(const void* X_dev, void* out_dev, int64_t tokens, int64_t features,
+                                           float keep, uint64_t seed, uint32_t layer, uint64_t step, int rescale,
+                                           void* stream);
+
 /* ---- inspection / test hooks ------------------------------------------------------------------------- */
 
 /* Copy matrix `mat`'s cached basis into caller device buffers (any may be NULL):

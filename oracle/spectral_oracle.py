@@ -377,7 +377,8 @@ def lowbias32(x: np.ndarray) -> np.ndarray:
 
 def keep_threshold(keep: float) -> int:
     """keep ratio quantised to 16 bits: an element is kept iff its 16 random bits are below this."""
-    return int(min(65536, max(1, round(float(keep) * 65536.0))))
+    x = np.float32(keep) * np.float32(65536.0)           # the keep ratio crosses the C ABI as a float
+    return int(min(65536, max(1, int(np.floor(np.float64(x) + 0.5)))))
 
 
 def prf_keep_mask(seed: int, layer: int, step: int, tokens: int, features: int, keep: float) -> np.ndarray:
@@ -429,5 +430,6 @@ def prf_exact_k_mask(seed: int, layer: int, step: int, tokens: int, features: in
 
 
 def exact_k(features: int, keep: float) -> int:
-    """K = round(keep * H), at least 1 and at most H."""
-    return int(min(features, max(1, round(float(keep) * features))))
+    """K = round(keep * H) (halves round up; the product is formed in fp32 as the C ABI does), at least 1, at most H."""
+    x = np.float32(keep) * np.float32(features)
+    return int(min(features, max(1, int(np.floor(np.float64(x) + 0.5)))))

@@ -79,6 +79,8 @@ EXPORTS = {
                                            C.POINTER(C.c_float)]),
     "sc_apply_prf_mask": (C.c_int, [_VP, _VP, C.c_int64, C.c_int64, C.c_float, C.c_uint64, C.c_uint32, C.c_uint64, C.c_int,
                                     _VP]),
+    "sc_apply_prf_mask_exact_k": (C.c_int, [_VP, _VP, C.c_int64, C.c_int64, C.c_float, C.c_uint64, C.c_uint32, C.c_uint64,
+                                            C.c_int, _VP]),
     "sc_export_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
     "sc_import_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
     "sc_export_projection": (C.c_int, [_VP, C.c_int, _VP, _VP]),
@@ -181,10 +183,22 @@ def project_static(G, U, V, X_out=None, stream=None):
     return X_out
 
 
-def apply_prf_mask(X, keep: float, seed: int, layer: int, step: int, rescale: bool = True, out=None, stream=None):
-    """h~ = h * M(seed, layer, step) (/ keep): the shared-PRF activation mask, bf16 tokens x features on the GPU."""
+def apply_prf_mask(X, keep: float, seed: int, layer: int, step: int, rescale: bool = True, out=None, stream=None,
+                   exact_k: bool = False):
+    """h~ = h * M(seed, layer, step) (/ keep): the shared-PRF activation mask, bf16 tokens x features on the GPU.
+    exact_k=True keeps exactly round(keep * features) features per token instead of independent coin flips."""
     import torch
     lib = load_library()
+    if exact_k:
+        assert X.is_cuda and X.is_contiguous() and X.dtype == torch.bfloat16 and X.dim() == 2
+        if out is None:
+            out = torch.empty_like(X)
+        st = stream if stream is not None else torch.cuda.current_stream(X.device)
+        with torch.cuda.device(X.device):
+            _check(lib.sc_apply_prf_mask_exact_k(X.data_ptr(), out.data_ptr(), X.shape[0], X.shape[1], float(keep),
+                                                 int(seed), int(layer), int(step), int(bool(rescale)), st.cuda_stream),
+                   "sc_apply_prf_mask_exact_k")
+        return out
     assert X.is_cuda and X.is_contiguous() and X.dtype == torch.bfloat16 and X.dim() == 2
     if out is None:
         out = torch.empty_like(X)

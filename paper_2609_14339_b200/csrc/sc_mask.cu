@@ -55,7 +55,73 @@ __global__ void __launch_bounds__(256) prf_mask_kernel(const uint4* __restrict__
   }
 }
 
+// Exactly-K-per-token variant: one block per token. Composite keys (hash << 16 | j) are distinct, so the K smallest
+// are found exactly by a radix select over their 48 bits, most significant byte first: in each of six rounds the
+// block histograms the current byte of the keys that still match the prefix and keeps the bin the K-th key falls in.
+__global__ void __launch_bounds__(256) prf_exact_k_kernel(const sc::bf16* __restrict__ in, sc::bf16* __restrict__ out,
+                                                          int features, int K, uint64_t base, float scale,
+                                                          int do_scale) {
+  __shared__ unsigned hist[256];
+  __shared__ unsigned long long prefix_s;
+  __shared__ unsigned remaining_s;
+  const int64_t t = blockIdx.x;
+  const uint32_t key = (uint32_t)mix64(base ^ (((uint64_t)t + 1ull) * 0xD1B54A32D192ED03ull));
+  unsigned long long prefix = 0;      // the leading bytes of the K-th smallest key found so far
+  unsigned remaining = (unsigned)K;   // its rank among the keys that share this prefix (1-based)
+  for (int round = 0; round < 6; ++round) {
+    const int shift = 40 - 8 * round;
+    hist[threadIdx.x] = 0;
+    __syncthreads();
+    for (int j = threadIdx.x; j < features; j += 256) {
+      const unsigned long long c = ((unsigned long long)lowbias32(key + (uint32_t)j * 0x9E3779B9u) << 16) | (unsigned)j;
+      if (round == 0 || (c >> (shift + 8)) == prefix) atomicAdd(&hist[(unsigned)(c >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      unsigned acc = 0;
+      int b = 0;
+      for (; b < 256; ++b) {
+        if (acc + hist[b] >= remaining) break;
+        acc += hist[b];
+      }
+      prefix_s = (prefix << 8) | (unsigned)b;
+      remaining_s = remaining - acc;
+    }
+    __syncthreads();
+    prefix = prefix_s;
+    remaining = remaining_s;
+    __syncthreads();
+  }
+  // prefix is now the K-th smallest composite key: keep everything at or below it
+  const sc::bf16 zero = __float2bfloat16_rn(0.f);
+  for (int j = threadIdx.x; j < features; j += 256) {
+    const unsigned long long c = ((unsigned long long)lowbias32(key + (uint32_t)j * 0x9E3779B9u) << 16) | (unsigned)j;
+    const size_t o = (size_t)t * features + j;
+    sc::bf16 v = in[o];
+    if (c > prefix) v = zero;
+    else if (do_scale) v = __float2bfloat16_rn(__bfloat162float(v) * scale);
+    out[o] = v;
+  }
+}
+
 }  // namespace
+
+extern "C" sc_status sc_apply_prf_mask_exact_k(const void* X_dev, void* out_dev, int64_t tokens, int64_t features,
+                                               float keep, uint64_t seed, uint32_t layer, uint64_t step, int rescale,
+                                               void* stream) {
+  if (!X_dev || !out_dev) return SC_ERR_INVALID_ARG;
+  if (tokens <= 0 || features <= 0) return SC_ERR_SHAPE;
+  if (features > 65536 || tokens > (1ll << 31) - 1) return SC_ERR_TOO_LARGE;
+  if (!(keep > 0.f && keep <= 1.f)) return SC_ERR_INVALID_ARG;
+  long K = lroundf(keep * (float)features);
+  K = K < 1 ? 1 : (K > features ? (long)features : K);
+  const uint64_t base = seed ^ ((((uint64_t)layer << 40) + step) * 0x9E3779B97F4A7C15ull);
+  prf_exact_k_kernel<<<(unsigned)tokens, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const sc::bf16*>(X_dev), static_cast<sc::bf16*>(out_dev), (int)features, (int)K, base,
+      (float)features / (float)K, rescale != 0);
+  ++sc::g_kernel_launches;
+  return cudaGetLastError() == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+}
 
 extern "C" sc_status sc_apply_prf_mask(const void* X_dev, void* out_dev, int64_t tokens, int64_t features, float keep,
                                        uint64_t seed, uint32_t layer, uint64_t step, int rescale, void* stream) {

@@ -61,3 +61,20 @@ def test_rejects_bad_arguments(torch):
     assert lib.sc_apply_prf_mask(p, p, 4, 16, 0.0, 0, 0, 0, 0, None) == -1
     assert lib.sc_apply_prf_mask(None, p, 4, 16, 0.5, 0, 0, 0, 0, None) == -1
     assert lib.sc_apply_prf_mask(p + 2, p, 4, 16, 0.5, 0, 0, 0, 0, None) == -4
+
+
+@pytest.mark.parametrize("tokens,features,keep", [(200, 264, 0.1), (64, 4096, 0.05), (33, 37, 0.5), (8, 16, 1.0)])
+def test_exact_k_mask_is_bit_exact(torch, tokens, features, keep):
+    import paper_2609_14339_b200 as sc
+    rng = np.random.default_rng(2)
+    X = (rng.standard_normal((tokens, features)) + 3.0).astype(np.float32)
+    Xb = torch.from_numpy(X).cuda().to(torch.bfloat16)
+    out = sc.apply_prf_mask(Xb, keep, seed=31, layer=2, step=7, rescale=False, exact_k=True)
+    M = so.prf_exact_k_mask(31, 2, 7, tokens, features, keep)
+    got = out.float().cpu().numpy()
+    assert np.array_equal(got != 0, M != 0)
+    assert np.all((got != 0).sum(axis=1) == so.exact_k(features, keep))
+    assert np.array_equal(got, Xb.float().cpu().numpy() * M)
+    out2 = sc.apply_prf_mask(Xb, keep, seed=31, layer=2, step=7, rescale=True, exact_k=True)
+    want = Xb.double().cpu().numpy() * M * (features / so.exact_k(features, keep))
+    assert rel(out2.double().cpu().numpy(), want) < 3e-3
