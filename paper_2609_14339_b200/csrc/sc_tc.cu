@@ -850,7 +850,7 @@ sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_
 // Two blocks per SM when three stages of each fit (their prologues and epilogues then overlap the other block's
 // streaming); otherwise one block with as many stages as fit.
 static int stages_for(int stage_bytes, int max_one_block) {
-  if (3 * stage_bytes + 2048 <= 110 * 1024) {
+  if (2 * stage_bytes + 2048 <= 110 * 1024) {
     const int s = (110 * 1024 - 2048) / stage_bytes;
     return s > 4 ? 4 : s;
   }
