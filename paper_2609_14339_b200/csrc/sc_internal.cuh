@@ -54,6 +54,7 @@ struct MatDev {
   float* Z;      // n x lp
   float* Z2;     // n x lp
   float* gram;   // lp x lp
+  float* spart;  // sweep_split x max(m, n) x lp   K-slice partials of a sweep (plans with few matrices only)
   float* gpart;  // kAtbMaxSplits x lp x lp   row-slice partials of the Gram matrix
   float* rmat;   // lp x lp   Cholesky factor (upper), first pass
   float* rmat2;  // lp x lp   second pass
@@ -90,6 +91,7 @@ struct ShapeClass {
   int* idx_dyn2 = nullptr; // device: subset list written per call (anchor arrivals, warm starts)
   bool tensor = false;     // served by the tcgen05 kernels
   int ksplit = 1;
+  int sweep_split_n = 1, sweep_split_t = 1;   // K slices of the plain / transposed sweeps over the momentum
   int split_m = 1, split_n = 1;   // row slices of A^T B products over m / n rows (fixed at plan creation)
   void* tmaps = nullptr;   // device: per-instance tensor maps (tensor engine only)
 };

@@ -148,13 +148,15 @@ size_t layout(sc_plan* p, bool assign) {
     float* gram = cv.take<float>((size_t)lp * lp); float* rmat = cv.take<float>((size_t)lp * lp);
     const ShapeClass& cls = p->classes[p->class_of[i]];
     float* gpart = cv.take<float>((size_t)std::max(cls.split_m, cls.split_n) * lp * lp);
+    const int ssp = std::max(cls.sweep_split_n, cls.sweep_split_t);
+    float* spart = ssp > 1 ? cv.take<float>((size_t)ssp * std::max(m, n) * lp) : nullptr;
     float* rmat2 = cv.take<float>((size_t)lp * lp); float* rinv = cv.take<float>((size_t)lp * lp);
     float* racc = cv.take<float>((size_t)lp * lp); float* jk = cv.take<float>((size_t)lp * lp);
     float* jv = cv.take<float>((size_t)lp * lp);
     float* ub = cv.take<float>((size_t)lp * rp); float* wb = cv.take<float>((size_t)lp * rp);
     if (assign) {
       MatDev& md = p->host_tab[i];
-      md.Y = Y; md.Y2 = Y2; md.Z = Z; md.Z2 = Z2; md.gram = gram; md.gpart = gpart; md.rmat = rmat; md.rmat2 = rmat2;
+      md.Y = Y; md.Y2 = Y2; md.Z = Z; md.Z2 = Z2; md.gram = gram; md.gpart = gpart; md.spart = spart; md.rmat = rmat; md.rmat2 = rmat2;
       md.rinv = rinv; md.racc = racc; md.jk = jk; md.jv = jv; md.ub = ub; md.wb = wb;
     }
   }
@@ -173,6 +175,17 @@ void fill_plan_basics(sc_plan* p, const sc_shape* shapes, int n_mats, int rank, 
     c.tensor = hp->engine == SC_ENGINE_AUTO && hp->grad_dtype == SC_DTYPE_BF16 && rank > 0 &&
                tc_shape_supported(c.m, c.n, d.rp);
     c.ksplit = c.tensor ? choose_ksplit(c) : 1;
+    if (c.tensor) {
+      // sweeps: one block per 128 output rows and matrix; split K when that leaves most SMs idle (slices >= 1024 long)
+      auto sweep_split = [&](int64_t rows_out, int64_t kdim) {
+        const int64_t tiles = (rows_out + 127) / 128 * (int64_t)c.mats.size();
+        int s = 1;
+        while (s < 8 && tiles * s < 148 && kdim / (s * 2) >= 1024) s *= 2;
+        return s;
+      };
+      c.sweep_split_n = sweep_split(c.m, c.n);
+      c.sweep_split_t = sweep_split(c.n, c.m);
+    }
     c.split_m = atb_splits((int)c.m, (int)c.mats.size());
     c.split_n = atb_splits((int)c.n, (int)c.mats.size());
     p->tensor_any = p->tensor_any || c.tensor;

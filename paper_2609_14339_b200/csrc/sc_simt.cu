@@ -262,7 +262,7 @@ void launch_atb(const MatDev* tab, const int* idx, int count, int offA, int offB
 void launch_sum_slices(const MatDev* tab, const int* idx, int count, int offPart, int offOut, int numel, int nsplit,
                        cudaStream_t s) {
   if (count <= 0 || numel <= 0) return;
-  sum_slices_kernel<<<dim3((numel + 255) / 256 < 64 ? (numel + 255) / 256 : 64, 1, count), 256, 0, s>>>(
+  sum_slices_kernel<<<dim3((numel + 255) / 256 < 592 ? (numel + 255) / 256 : 592, 1, count), 256, 0, s>>>(
       tab, idx, offPart, offOut, numel, nsplit);
   ++g_kernel_launches;
 }

@@ -941,16 +941,23 @@ sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, b
   pa.rows_out = transposed ? n : m;
   pa.kdim = transposed ? m : n;
   pa.ncols = lp; pa.ncols_valid = lp; pa.ldo = lp;
-  pa.cps = (pa.kdim + kPassK - 1) / kPassK;
+  // few output tiles (a plan with one or two matrices): split the contraction over K slices into spart, add them up
+  const int slices = transposed ? c.sweep_split_t : c.sweep_split_n;
+  const int nchunks = (pa.kdim + kPassK - 1) / kPassK;
+  pa.cps = (nchunks + slices - 1) / slices;
+  const int out_final = pa.out_off;
+  if (slices > 1) pa.out_off = (int)offsetof(MatDev, spart);
   const int stage_bytes = kTileBytes + (lp / 32) * kAtomBytes;
   pa.stages = stages_for(stage_bytes, 8);
   pa.tmem_cols = tmem_cols_for(lp);
   const size_t smem = (size_t)pa.stages * stage_bytes + 1024 + 256;
   const CUtensorMap* maps = static_cast<const CUtensorMap*>(c.tmaps);
-  dim3 grid((pa.rows_out + 127) / 128, 1, count);
+  dim3 grid((pa.rows_out + 127) / 128, slices, count);
   if (transposed) pass_kernel<true><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, pa, p->status_dev);
   else pass_kernel<false><<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, maps, pa, p->status_dev);
   ++g_kernel_launches;
+  if (slices > 1)
+    launch_sum_slices(p->dev_tab, idx, count, (int)offsetof(MatDev, spart), out_final, pa.rows_out * lp, slices, p->stream);
   return cuda_ok(cudaGetLastError());
 }
 
