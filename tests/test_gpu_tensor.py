@@ -173,3 +173,19 @@ def test_factored_anchor_gradient(torch, engine):
     import paper_2609_14339_b200 as sc
     with pytest.raises(sc.SCError):
         plan.anchor_update_factored([None, torch.zeros((200, 4), device="cuda")], [torch.zeros((256, 4), device="cuda"), None], 9)
+
+
+def test_global_clipping_and_in_step_rescale_on_the_tensor_engine(torch):
+    """max_grad_norm on: projections of all classes first, one clip factor from the closed-form norms, then the
+    updates; grads_prescaled = 0: the step applies 1/keep itself."""
+    case = Case(shapes=[(256, 384), (384, 256), (256, 384)], rank=16, tokens=128, keep=0.25, prescaled=False,
+                max_grad_norm=0.2, tau_p=30.0, planted=4)
+    inp = make_inputs(case)
+    g = GpuRun(case, inp, torch)
+    assert g.uses_tc and g.dev_status == 0
+    o = OracleRun(case, inp, "mirror")
+    es = compare_step(g, o)
+    assert max(es["gproj"], es["m"], es["v"], es["dW"]) < TOL, es
+    total = sum(np.sum(x * x) for x in g.gproj)
+    assert abs(np.sqrt(total) - 0.2) < 2e-4
+    assert 0.0 < g.clip < 1.0
