@@ -135,10 +135,173 @@ __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs a, EpiAdamW epi) {
   }
 }
 
+// =====================================================================================================
+// Tall-skinny product  C = alpha * A * op(B) [+ beta_c * C]  for row-major fp32 A (M x K, K a few dozen to a
+// few hundred): the shape of Y R^-1, U = Q Ub, V = Qb Wb and C^T = V Xs^T. A is streamed once through a
+// two-deep ring of 128 x 32 chunks filled by cp.async (16 bytes per copy when base, row stride and K allow
+// it, 4 bytes otherwise); B is small, comes from L2 and is prefetched into registers one chunk ahead.
+// Thread (ty, tx) owns rows ty + 16 i (i < 8) and columns 4 tx .. 4 tx + 3; the sum over k runs in
+// increasing k with one fmaf per term, exactly like gemm_kernel, so both give the same bits.
+// =====================================================================================================
+constexpr int TS_BM = 128, TS_BN = 64, TS_KC = 32;
+constexpr int TS_AP = TS_KC + 4;   // row pitch of the A chunk (floats): 16-byte rows, no bank conflicts on float4 reads
+constexpr int TS_BP = TS_BN + 4;
+constexpr int TS_SMEM = (2 * TS_BM * TS_AP + 2 * TS_KC * TS_BP) * (int)sizeof(float);
+
+__device__ __forceinline__ void cp_async16(float* dst, const float* src, bool valid) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst);
+  const int bytes = valid ? 16 : 0;   // 0 source bytes: the 16 destination bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async4(float* dst, const float* src, bool valid) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst);
+  const int bytes = valid ? 4 : 0;
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+}
+
+__global__ void __launch_bounds__(256, 2) tsgemm_kernel(GemmArgs a) {
+  extern __shared__ __align__(16) float ts_smem[];
+  float(*As)[TS_BM][TS_AP] = reinterpret_cast<float(*)[TS_BM][TS_AP]>(ts_smem);
+  float(*Bs)[TS_KC][TS_BP] = reinterpret_cast<float(*)[TS_KC][TS_BP]>(ts_smem + 2 * TS_BM * TS_AP);
+  const MatDev& md = a.tab[a.idx[blockIdx.z]];
+  const float* __restrict__ A = field<const float>(md, a.offA);
+  const float* __restrict__ B = field<const float>(md, a.offB);
+  const int row0 = blockIdx.y * TS_BM, col0 = blockIdx.x * TS_BN;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const bool vec = ((reinterpret_cast<uintptr_t>(A) & 15) == 0) && (a.lda % 4 == 0) && (a.K % 4 == 0);
+  const int nchunks = (a.K + TS_KC - 1) / TS_KC;
+
+  auto issue_a = [&](int stage, int k0) {
+    if (vec) {
+#pragma unroll
+      for (int j = 0; j < (TS_BM * TS_KC / 4) / 256; ++j) {
+        const int e = tid + 256 * j, r = e >> 3, q = e & 7;
+        const int gr = row0 + r, gk = k0 + 4 * q;
+        const bool ok = gr < a.M && gk < a.K;
+        cp_async16(&As[stage][r][4 * q], ok ? A + (size_t)gr * a.lda + gk : A, ok);
+      }
+    } else {
+      for (int e = tid; e < TS_BM * TS_KC; e += 256) {
+        const int r = e / TS_KC, k = e % TS_KC;
+        const int gr = row0 + r, gk = k0 + k;
+        const bool ok = gr < a.M && gk < a.K;
+        cp_async4(&As[stage][r][k], ok ? A + (size_t)gr * a.lda + gk : A, ok);
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  float breg[TS_KC * TS_BN / 256];
+  auto load_b = [&](int k0) {
+#pragma unroll
+    for (int j = 0; j < TS_KC * TS_BN / 256; ++j) {
+      const int e = tid + 256 * j;
+      int k, c;
+      if (!a.transB) { k = e / TS_BN; c = e % TS_BN; } else { c = e / TS_KC; k = e % TS_KC; }
+      const int gk = k0 + k, gc = col0 + c;
+      float v = 0.f;
+      if (gk < a.K && gc < a.N) v = a.transB ? B[(size_t)gc * a.ldb + gk] : B[(size_t)gk * a.ldb + gc];
+      breg[j] = v;
+    }
+  };
+  auto store_b = [&](int stage) {
+#pragma unroll
+    for (int j = 0; j < TS_KC * TS_BN / 256; ++j) {
+      const int e = tid + 256 * j;
+      int k, c;
+      if (!a.transB) { k = e / TS_BN; c = e % TS_BN; } else { c = e / TS_KC; k = e % TS_KC; }
+      Bs[stage][k][c] = breg[j];
+    }
+  };
+
+  float acc[8][4] = {};
+  issue_a(0, 0);
+  load_b(0);
+  store_b(0);
+  for (int c = 0; c < nchunks; ++c) {
+    const int st = c & 1;
+    const bool more = c + 1 < nchunks;
+    if (more) {
+      issue_a(st ^ 1, (c + 1) * TS_KC);
+      load_b((c + 1) * TS_KC);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kq = 0; kq < TS_KC / 4; ++kq) {
+      float4 av[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) av[i] = *reinterpret_cast<const float4*>(&As[st][i * 16 + ty][4 * kq]);
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        const float4 b = *reinterpret_cast<const float4*>(&Bs[st][4 * kq + kk][tx * 4]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const float x = kk == 0 ? av[i].x : kk == 1 ? av[i].y : kk == 2 ? av[i].z : av[i].w;
+          acc[i][0] = fmaf(x, b.x, acc[i][0]);
+          acc[i][1] = fmaf(x, b.y, acc[i][1]);
+          acc[i][2] = fmaf(x, b.z, acc[i][2]);
+          acc[i][3] = fmaf(x, b.w, acc[i][3]);
+        }
+      }
+    }
+    __syncthreads();
+    if (more) store_b(st ^ 1);
+  }
+
+  float* C = field<float>(md, a.offC);
+  bf16* Chi = a.offHi ? field<bf16>(md, a.offHi) : nullptr;
+  bf16* Clo = a.offHi ? field<bf16>(md, a.offLo) : nullptr;
+  const int gc0 = col0 + tx * 4;
+  const bool vec_c = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && (a.ldc % 4 == 0) && gc0 + 3 < a.N;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int gr = row0 + i * 16 + ty;
+    if (gr >= a.M) continue;
+    float val[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) val[j] = a.alpha * acc[i][j];
+    float* crow = C + (size_t)gr * a.ldc;
+    if (vec_c) {
+      if (a.beta_c != 0.f) {
+        const float4 o = *reinterpret_cast<const float4*>(crow + gc0);
+        val[0] = fmaf(a.beta_c, o.x, val[0]); val[1] = fmaf(a.beta_c, o.y, val[1]);
+        val[2] = fmaf(a.beta_c, o.z, val[2]); val[3] = fmaf(a.beta_c, o.w, val[3]);
+      }
+      *reinterpret_cast<float4*>(crow + gc0) = make_float4(val[0], val[1], val[2], val[3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (gc0 + j >= a.N) continue;
+        if (a.beta_c != 0.f) val[j] = fmaf(a.beta_c, crow[gc0 + j], val[j]);
+        crow[gc0 + j] = val[j];
+      }
+    }
+    if (Chi) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (gc0 + j >= a.N) continue;
+        bf16 hi, lo;
+        split2(val[j], hi, lo);
+        Chi[(size_t)gr * a.ld_split + gc0 + j] = hi;
+        Clo[(size_t)gr * a.ld_split + gc0 + j] = lo;
+      }
+    }
+  }
+}
+
 void launch_gemm(const GemmArgs& a, int count, cudaStream_t s) {
   if (count <= 0 || a.M <= 0 || a.N <= 0) return;
-  dim3 grid((a.N + BN - 1) / BN, (a.M + BM - 1) / BM, count);
-  gemm_kernel<false><<<grid, 256, 0, s>>>(a, EpiAdamW{});
+  if (!a.transA && !a.a_bf16) {
+    static const cudaError_t attr = cudaFuncSetAttribute(tsgemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TS_SMEM);
+    (void)attr;
+    dim3 grid((a.N + TS_BN - 1) / TS_BN, (a.M + TS_BM - 1) / TS_BM, count);
+    tsgemm_kernel<<<grid, 256, TS_SMEM, s>>>(a);
+  } else {
+    dim3 grid((a.N + BN - 1) / BN, (a.M + BM - 1) / BM, count);
+    gemm_kernel<false><<<grid, 256, 0, s>>>(a, EpiAdamW{});
+  }
   ++g_kernel_launches;
 }
 
