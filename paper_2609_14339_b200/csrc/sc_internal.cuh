@@ -127,6 +127,7 @@ struct sc_plan {
   int staging_next = 0;
   float* clip_dev = nullptr;          // clip factor applied to G_proj
   unsigned* status_dev = nullptr;     // latched device status bits
+  unsigned* work_dev = nullptr;       // work-item counter of the streaming update kernel (zeroed before each launch)
   float* stats_dev = nullptr;         // n_mats * kStatsFloats
   char* ws = nullptr;
   size_t ws_bytes = 0;

@@ -97,8 +97,9 @@ size_t layout(sc_plan* p, bool assign) {
   MatDev* tab = cv.take<MatDev>(n_mats);
   float* clip = cv.take<float>(1);
   unsigned* status = cv.take<unsigned>(1);
+  unsigned* work = cv.take<unsigned>(1);
   float* stats = cv.take<float>((size_t)n_mats * kStatsFloats);
-  if (assign) { p->dev_tab = tab; p->clip_dev = clip; p->status_dev = status; p->stats_dev = stats; }
+  if (assign) { p->dev_tab = tab; p->clip_dev = clip; p->status_dev = status; p->work_dev = work; p->stats_dev = stats; }
   for (auto& c : p->classes) {
     int* a = cv.take<int>(c.mats.size());
     int* b = cv.take<int>(c.mats.size());

@@ -442,6 +442,22 @@ ema_pass_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, con
 // =====================================================================================================
 // AdamW on four elements of G_proj = clip * (alpha_s * G + R), R = the low-rank part from the tensor cores.
 // =====================================================================================================
+// Square root and quotient without the special-case branches of the IEEE expansions: those branches end the
+// basic block after every element, so the sixteen element chains of a thread would run one after another.
+// sqrt.approx is within 1 ulp; the quotient takes the hardware reciprocal (1 ulp) and one residual correction,
+// which leaves it within 1 ulp of the rounded quotient. den >= eps > 0 and vo >= 0 always hold here.
+__device__ __forceinline__ float sqrt_nobranch(float x) {
+  float y;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float div_nobranch(float a, float b) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(b));
+  const float q = a * r;
+  return fmaf(fmaf(-b, q, a), r, q);
+}
+
 __device__ __forceinline__ void adamw4(const StepScalars& s, float clip, const float g_raw[4], const float4& r,
                                        float4& w, float4& m1, float4& m2, float4& gp) {
   const float rr[4] = {r.x, r.y, r.z, r.w};
@@ -451,8 +467,8 @@ __device__ __forceinline__ void adamw4(const StepScalars& s, float clip, const f
     const float g = clip * fmaf(s.alpha_s, g_raw[j], rr[j]);
     const float mo = fmaf(s.beta1, M1[j], s.one_m_beta1 * g);
     const float vo = fmaf(s.beta2, M2[j], s.one_m_beta2 * g * g);
-    const float den = fmaf(sqrtf(vo), s.inv_sqrt_bc2, s.eps);
-    W[j] = fmaf(-s.step_size, mo / den, W[j] * s.decay);
+    const float den = fmaf(sqrt_nobranch(vo), s.inv_sqrt_bc2, s.eps);
+    W[j] = fmaf(-s.step_size, div_nobranch(mo, den), W[j] * s.decay);
     M1[j] = mo; M2[j] = vo; GP[j] = g;
   }
 }
@@ -477,10 +493,18 @@ constexpr int kOpndU = 2 * kTileBytes;                       // U hi + lo, 128 r
 constexpr int kOpndC = 2 * (kTileN * 128);                   // C^T hi + lo, 64 rows x 64 bf16 each
 constexpr int kStreamSmem = kStreamStages * kStreamStageBytes + kOpndU + kOpndC;
 
+// Work items are handed out by an atomic counter: blocks do not run at the same speed (the slowest of a static split
+// finished 7% after the median), so each block's producer draws the next item when it needs one and passes the index
+// to the MMA issuer and the consumers through a small ring in shared memory. The producer can be at most three
+// units, i.e. fewer than kItemSlots items, ahead of the consumers, so a slot is never rewritten while still in use.
+constexpr int kItemSlots = 8;
+
 struct StreamBars {
   uint64_t full[kStreamStages], empty[kStreamStages];
   uint64_t opnd_full, opnd_empty;
   uint64_t acc_full[2], acc_empty[2];
+  uint64_t item_ready[kItemSlots];
+  int item_slot[kItemSlots];
   uint32_t tmem_slot;
   int abort_flag;
 };
@@ -503,7 +527,7 @@ __device__ __forceinline__ void decode_item(const StreamGeom& g, int item, int& 
 __global__ void __launch_bounds__(320, 1)
 fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx,
                            const CUtensorMap* __restrict__ maps, StreamGeom g, StepScalars sc,
-                           const float* __restrict__ clip_ptr, unsigned* status) {
+                           const float* __restrict__ clip_ptr, unsigned* status, unsigned* work_counter) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* opnd = smem + kStreamStages * kStreamStageBytes;
@@ -517,6 +541,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
     mbar_init(&bars->opnd_full, 1);
     mbar_init(&bars->opnd_empty, 1);
     for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 8); }
+    for (int k = 0; k < kItemSlots; ++k) mbar_init(&bars->item_ready[k], 1);
     bars->abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
@@ -533,7 +558,16 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
       uint32_t unit_it = 0, op_it = 0;
       int last_inst = -1, last_panel = -1;
       bool dead = false;
-      for (int item = blockIdx.x; item < g.n_items && !dead; item += gridDim.x) {
+      uint32_t item_it = 0;
+      int next_item = (int)atomicAdd(work_counter, 1u);
+      while (!dead) {
+        const int item = next_item < g.n_items ? next_item : -1;
+        volatile int* slot = &bars->item_slot[item_it % kItemSlots];
+        *slot = item;
+        mbar_arrive(&bars->item_ready[item_it % kItemSlots]);   // release: the slot is visible to whoever sees this phase
+        ++item_it;
+        if (item < 0) break;
+        next_item = (int)atomicAdd(work_counter, 1u);           // drawn one item ahead, so its latency is hidden
         int inst, rt, ct0, ct1;
         decode_item(g, item, inst, rt, ct0, ct1);
         const MatDev& md = tab[idx[inst]];
@@ -593,7 +627,10 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
       const uint32_t uh = smem_u32(opnd), ul = uh + kTileBytes, ch = uh + kOpndU, cl = ch + kTileN * 128;
       uint32_t op_it = 0, t = 0;
       bool dead = false;
-      for (int item = blockIdx.x; item < g.n_items && !dead; item += gridDim.x) {
+      for (uint32_t item_it = 0; !dead; ++item_it) {
+        if (!mbar_wait(&bars->item_ready[item_it % kItemSlots], (item_it / kItemSlots) & 1, abort_flag)) { dead = true; break; }
+        const int item = *reinterpret_cast<volatile int*>(&bars->item_slot[item_it % kItemSlots]);
+        if (item < 0) break;
         int inst, rt, ct0, ct1;
         decode_item(g, item, inst, rt, ct0, ct1);
         for (int ct = ct0; ct < ct1 && !dead; ++ct, ++t) {
@@ -630,7 +667,10 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
     uint32_t unit_it = 0, t = 0;
     int last_inst = -1;
     bool dead = false;
-    for (int item = blockIdx.x; item < g.n_items && !dead; item += gridDim.x) {
+    for (uint32_t item_it = 0; !dead; ++item_it) {
+      if (!mbar_wait(&bars->item_ready[item_it % kItemSlots], (item_it / kItemSlots) & 1, abort_flag)) { dead = true; break; }
+      const int item = *reinterpret_cast<volatile int*>(&bars->item_slot[item_it % kItemSlots]);
+      if (item < 0) break;
       int inst, rt, ct0, ct1;
       decode_item(g, item, inst, rt, ct0, ct1);
       const MatDev& md = tab[idx[inst]];
@@ -659,37 +699,49 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
           float4* M1s = reinterpret_cast<float4*>(st + kUnitF32);
           float4* M2s = reinterpret_cast<float4*>(st + 2 * kUnitF32);
           uint4* Gs = reinterpret_cast<uint4*>(st + 3 * kUnitF32);
-          float gout[16];
-          uint4 wb_pk[2];
+          // all of this thread's 16 elements are read first, so that the 16 AdamW chains are independent work for
+          // the scheduler; results go back in place afterwards
+          int fidx[4], gidx[2];
+          float4 w[4], m1[4], m2[4], gp[4];
+          uint4 graw[2];
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
-            const int gidx = r * 4 + ((2 * h + j) ^ ((r >> 1) & 3));
-            const uint4 graw = Gs[gidx];
-            const uint32_t gw[4] = {graw.x, graw.y, graw.z, graw.w};
-            uint32_t wbw[4];
+            gidx[j] = r * 4 + ((2 * h + j) ^ ((r >> 1) & 3));
+            graw[j] = Gs[gidx[j]];
+          }
 #pragma unroll
-            for (int i2 = 0; i2 < 2; ++i2) {
-              const int i = 2 * j + i2;            // 16-byte chunk of the fp32 rows
-              const int fidx = r * 8 + ((4 * h + i) ^ (r & 7));
-              float4 w = Ws[fidx], m1 = M1s[fidx], m2 = M2s[fidx], gp;
-              const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&gw[2 * i2]);
-              const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&gw[2 * i2 + 1]);
-              const float g4[4] = {__low2float(g01), __high2float(g01), __low2float(g23), __high2float(g23)};
-              const float4 rr = make_float4(rv[4 * i], rv[4 * i + 1], rv[4 * i + 2], rv[4 * i + 3]);
-              adamw4(sc, clip, g4, rr, w, m1, m2, gp);
-              Ws[fidx] = w; M1s[fidx] = m1; M2s[fidx] = m2;
-              gout[4 * i] = gp.x; gout[4 * i + 1] = gp.y; gout[4 * i + 2] = gp.z; gout[4 * i + 3] = gp.w;
-              __nv_bfloat162 b01 = __floats2bfloat162_rn(w.x, w.y), b23 = __floats2bfloat162_rn(w.z, w.w);
-              wbw[2 * i2] = *reinterpret_cast<uint32_t*>(&b01);
-              wbw[2 * i2 + 1] = *reinterpret_cast<uint32_t*>(&b23);
-            }
-            wb_pk[j] = make_uint4(wbw[0], wbw[1], wbw[2], wbw[3]);
-            Gs[gidx] = wb_pk[j];
+          for (int i = 0; i < 4; ++i) {
+            fidx[i] = r * 8 + ((4 * h + i) ^ (r & 7));
+            w[i] = Ws[fidx[i]]; m1[i] = M1s[fidx[i]]; m2[i] = M2s[fidx[i]];
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint4& gq = graw[i >> 1];
+            const uint32_t lo = (i & 1) ? gq.z : gq.x, hi = (i & 1) ? gq.w : gq.y;
+            const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162*>(&lo);
+            const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&hi);
+            const float g4[4] = {__low2float(g01), __high2float(g01), __low2float(g23), __high2float(g23)};
+            const float4 rr = make_float4(rv[4 * i], rv[4 * i + 1], rv[4 * i + 2], rv[4 * i + 3]);
+            adamw4(sc, clip, g4, rr, w[i], m1[i], m2[i], gp[i]);
+          }
+          float gout[16];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            Ws[fidx[i]] = w[i]; M1s[fidx[i]] = m1[i]; M2s[fidx[i]] = m2[i];
+            gout[4 * i] = gp[i].x; gout[4 * i + 1] = gp[i].y; gout[4 * i + 2] = gp[i].z; gout[4 * i + 3] = gp[i].w;
+          }
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            const __nv_bfloat162 b0 = __floats2bfloat162_rn(w[2 * j].x, w[2 * j].y), b1 = __floats2bfloat162_rn(w[2 * j].z, w[2 * j].w);
+            const __nv_bfloat162 b2 = __floats2bfloat162_rn(w[2 * j + 1].x, w[2 * j + 1].y), b3 = __floats2bfloat162_rn(w[2 * j + 1].z, w[2 * j + 1].w);
+            Gs[gidx[j]] = make_uint4(*reinterpret_cast<const uint32_t*>(&b0), *reinterpret_cast<const uint32_t*>(&b1),
+                                     *reinterpret_cast<const uint32_t*>(&b2), *reinterpret_cast<const uint32_t*>(&b3));
           }
           const int x = ct * kTileN + u * kUnitW;
           if (gp_dbg) {   // test hook: plain stores, one row per thread
             const int row = row0 + r, col = x + h * 16;
             if (row < g.m)
+#pragma unroll
               for (int e = 0; e < 16; ++e)
                 if (col + e < g.n) gp_dbg[(size_t)row * g.n + col + e] = gout[e];
           }
@@ -1004,16 +1056,16 @@ sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int coun
   g.m = m; g.n = n; g.rp = p->rp;
   g.row_tiles = (m + 127) / 128;
   g.col_tiles = (n + kTileN - 1) / kTileN;
-  int csplit = 1;
-  // enough work items that the last, partly filled round of the persistent blocks costs a few percent at most
-  while ((long long)count * g.row_tiles * csplit < 16LL * n_sm && g.col_tiles / (csplit * 2) >= 2) csplit *= 2;
-  g.tiles_per_chunk = (g.col_tiles + csplit - 1) / csplit;
+  // small items (two 128 x 64 tiles), neighbouring column chunks next to each other in the item order: blocks that
+  // run side by side then touch the same rows of DRAM, and the atomic hand-out has something to balance with
+  g.tiles_per_chunk = 2 < g.col_tiles ? 2 : g.col_tiles;
   g.csplit = (g.col_tiles + g.tiles_per_chunk - 1) / g.tiles_per_chunk;
   g.n_items = count * g.row_tiles * g.csplit;
   const int grid = g.n_items < n_sm ? g.n_items : n_sm;
   const size_t smem = kStreamSmem + sizeof(StreamBars) + 1024;
+  if (cudaMemsetAsync(p->work_dev, 0, sizeof(unsigned), p->stream) != cudaSuccess) return SC_ERR_CUDA;
   fused_update_stream_kernel<<<grid, 320, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps),
-                                                             g, sc, p->clip_dev, p->status_dev);
+                                                             g, sc, p->clip_dev, p->status_dev, p->work_dev);
   ++g_kernel_launches;
   return cuda_ok(cudaGetLastError());
 }
