@@ -652,7 +652,9 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
     // X = U^T T as row-slice partials (the K-slice partials of T are added on the way in); xs_kernel adds them up
     // (one block per matrix adds the slices inside xs_kernel unless that is too much for one block)
     const bool sum_in_xs = (size_t)c.split_m * rp * rp <= (size_t)(1 << 16);
-    if (rp > 0 && c.tensor && c.ksplit == 1) {
+    if (rp > 0 && c.tensor) {
+      // plans with few matrices split K in the projection: add those partials of T up first (in place, slice 0)
+      launch_reduce_partials(p->dev_tab, idx, cnt, (int64_t)m * rp, c.ksplit, s);
       sc_status e = tc_launch_xpart(p, c, idx, cnt, c.split_m);        // tensor cores, T read once
       if (e != SC_OK) return e;
       if (!sum_in_xs) launch_sum_slices(p->dev_tab, idx, cnt, OFF(xpart), OFF(X), rp * rp, c.split_m, s);
@@ -762,9 +764,7 @@ sc_status sc_export_projection(sc_plan* p, int mat, void* T_dev, void* X_dev) {
   const int r = p->rank, rp = p->rp;
   if (r == 0) return SC_OK;
   if (T_dev) {
-    // the tensor-core projection leaves K-slice partials: add them up first (the next step rewrites them anyway)
-    ShapeClass& c = p->classes[p->class_of[mat]];
-    launch_reduce_partials(p->dev_tab, c.idx_all + p->inst_of[mat], 1, (int64_t)md.m * rp, c.ksplit, p->stream);
+    // the step has already added the K-slice partials of the tensor-core projection into slice 0
     launch_unpad_copy(static_cast<float*>(T_dev), r, md.T, rp, md.m, r, p->stream);
   }
   if (X_dev) launch_unpad_copy(static_cast<float*>(X_dev), r, md.X, rp, r, r, p->stream);
