@@ -188,6 +188,21 @@ SC_API sc_status sc_correct_and_step_host(sc_plan* plan, const void* const* host
 SC_API sc_status sc_apply_prf_mask(const void* X_dev, void* out_dev, int64_t tokens, int64_t features, float keep,
                                    uint64_t seed, uint32_t layer, uint64_t step, int rescale, void* stream);
 
+/* sc_masked_weight_grad - the fast circuit's weight gradient of one linear layer from masked activations
+ * (Section 3.1, Algorithm 1 lines 4-5): G = dY^T (X * M) * 65536 / round(keep * 65536), M the mask of sc_apply_prf_mask
+ * for the same (seed, layer, step). Two launches on `stream`: the mask pass X -> Xm and a dense bf16 GEMM over the
+ * token dimension on the tensor cores (fp32 accumulation, the rescale applied in fp32 before the result is rounded).
+ * Stand-alone (no plan), asynchronous.
+ *   dY_dev      device: tokens x rows bf16 row-major (gradient with respect to the layer's output), read only
+ *   X_dev       device: tokens x cols bf16 row-major (the layer's input, unmasked), read only
+ *   Xm_dev      device: tokens x cols bf16, caller-owned; receives X * M (unscaled). May alias X_dev.
+ *   G_dev       device: rows x cols row-major, out_dtype (SC_DTYPE_BF16 or SC_DTYPE_FP32), overwritten
+ *   status_dev  device: one uint32 that receives bit 0 if a bounded device-side wait runs out, or NULL
+ * All pointers 16-byte aligned; rows % 8 == 0 and cols % 8 == 0 (SC_ERR_SHAPE otherwise); tokens is unrestricted. */
+SC_API sc_status sc_masked_weight_grad(const void* dY_dev, const void* X_dev, void* Xm_dev, void* G_dev, int out_dtype,
+                                       int64_t tokens, int64_t rows, int64_t cols, float keep, uint64_t seed,
+                                       uint32_t layer, uint64_t step, void* status_dev, void* stream);
+
 /* sc_apply_prf_mask_exact_k - the per-token form of the same mask (Section 3.1: "retaining K = round((1 - p) H)
  * dimensions per token"): every token keeps exactly K = round(keep * features) features, chosen by the K smallest
  * values of a per-(token, feature) hash (ties impossible by construction); rescale multiplies by features / K.

@@ -79,6 +79,8 @@ EXPORTS = {
                                            C.POINTER(C.c_float)]),
     "sc_apply_prf_mask": (C.c_int, [_VP, _VP, C.c_int64, C.c_int64, C.c_float, C.c_uint64, C.c_uint32, C.c_uint64, C.c_int,
                                     _VP]),
+    "sc_masked_weight_grad": (C.c_int, [_VP, _VP, _VP, _VP, C.c_int, C.c_int64, C.c_int64, C.c_int64, C.c_float,
+                                        C.c_uint64, C.c_uint32, C.c_uint64, _VP, _VP]),
     "sc_apply_prf_mask_exact_k": (C.c_int, [_VP, _VP, C.c_int64, C.c_int64, C.c_float, C.c_uint64, C.c_uint32, C.c_uint64,
                                             C.c_int, _VP]),
     "sc_export_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
@@ -181,6 +183,32 @@ def project_static(G, U, V, X_out=None, stream=None):
         _check(lib.sc_project_static(G.data_ptr(), dt, U.data_ptr(), V.data_ptr(), rows, cols, r, X_out.data_ptr(),
                                      st.cuda_stream), "sc_project_static")
     return X_out
+
+
+def masked_weight_grad(dY, X, keep: float, seed: int, layer: int, step: int, out_dtype=None, Xm=None, out=None,
+                       status=None, stream=None):
+    """G = dY^T (X * M(seed, layer, step)) / keep for one linear layer: the mask pass and a tensor-core GEMM over the
+    tokens. dY: tokens x rows, X: tokens x cols, both bf16 on the GPU. Returns (G, Xm); Xm holds X * M (unscaled)."""
+    import torch
+    lib = load_library()
+    assert dY.is_cuda and X.is_cuda and dY.is_contiguous() and X.is_contiguous()
+    assert dY.dtype == torch.bfloat16 and X.dtype == torch.bfloat16 and dY.dim() == 2 and X.dim() == 2
+    assert dY.shape[0] == X.shape[0]
+    tokens, rows, cols = X.shape[0], dY.shape[1], X.shape[1]
+    out_dtype = torch.bfloat16 if out_dtype is None else out_dtype
+    if Xm is None:
+        Xm = torch.empty_like(X)
+    if out is None:
+        out = torch.empty((rows, cols), device=X.device, dtype=out_dtype)
+    assert out.is_contiguous() and out.shape == (rows, cols) and out.dtype in (torch.bfloat16, torch.float32)
+    st = stream if stream is not None else torch.cuda.current_stream(X.device)
+    with torch.cuda.device(X.device):
+        _check(lib.sc_masked_weight_grad(dY.data_ptr(), X.data_ptr(), Xm.data_ptr(), out.data_ptr(),
+                                         0 if out.dtype == torch.bfloat16 else 1, tokens, rows, cols, float(keep),
+                                         int(seed), int(layer), int(step),
+                                         status.data_ptr() if status is not None else None, st.cuda_stream),
+               "sc_masked_weight_grad")
+    return out, Xm
 
 
 def apply_prf_mask(X, keep: float, seed: int, layer: int, step: int, rescale: bool = True, out=None, stream=None,

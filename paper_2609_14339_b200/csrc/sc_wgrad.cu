@@ -1,0 +1,263 @@
+// sc_masked_weight_grad: the fast circuit's weight gradient of one linear layer from masked activations
+// (Section 3.1; Algorithm 1 lines 4-5):  G = dY^T (X . M) * 65536 / round(keep * 65536),  M the shared-PRF mask.
+//
+// Two launches on the caller's stream: the mask pass (sc_apply_prf_mask, X -> Xm, one HBM pass over the activation)
+// and a dense bf16 GEMM over the token dimension on the tensor cores. The mask is applied once, not inside the GEMM's
+// operand load: every activation tile is an operand of all row tiles of the output, so hashing at load time would
+// repeat the same work rows/128 times and turn a tensor-bound kernel into an issue-bound one.
+//
+// GEMM: G[rows x cols] = scale * A^T B with A = dY (tokens x rows) and B = Xm (tokens x cols), both row-major, i.e.
+// both operands are MN-major for the tensor core (the contraction index is the slow one in memory). Persistent blocks,
+// one per SM, tiles of 128 x 256 in row-tile-fastest order (blocks running side by side share the activation panel in
+// L2), K advancing 64 tokens per pipeline stage:
+//   warp 0   TMA producer: two 64 x 64 boxes of dY and four of Xm per stage (128-byte swizzle), 4-stage ring
+//   warp 1   tcgen05.mma kind::f16 issuer, M = 128, N = 256, fp32 accumulators, two 256-column buffers in TMEM
+//   warps 2-5  epilogue: TMEM -> registers -> scale -> bf16 or fp32 -> global
+// Every mbarrier wait is bounded; a wait that runs out latches SC_ERR_TIMEOUT in *status_dev and the block winds down.
+#include <cuda.h>
+
+#include "sc_internal.cuh"
+#include "sc_ptx.cuh"
+
+namespace sc {
+namespace {
+
+constexpr int kWgBM = 128, kWgBN = 256, kWgBK = 64, kWgStages = 4;
+constexpr int kWgBox = 64 * kWgBK * 2;                     // one 64 (MN) x 64 (K) bf16 box: 8 KB
+constexpr int kWgABytes = (kWgBM / 64) * kWgBox;           // 16 KB
+constexpr int kWgBBytes = (kWgBN / 64) * kWgBox;           // 32 KB
+constexpr int kWgStageBytes = kWgABytes + kWgBBytes;       // 48 KB
+
+struct WgBars {
+  uint64_t full[kWgStages], empty[kWgStages];
+  uint64_t acc_full[2], acc_empty[2];
+  uint32_t tmem_slot;
+  int abort_flag;
+  int never_flag;
+};
+
+// MN-major bf16 operand, 128-byte swizzle: atoms of 64 (MN, contiguous 128 bytes) x 8 (K rows); consecutive K groups
+// of 8 rows are 1024 bytes apart (SBO), consecutive 64-wide MN blocks `lbo` bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_mn_bf16(uint32_t saddr, uint32_t lbo) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// bf16 x bf16 -> fp32, both operands MN-major, M = 128.
+__device__ __forceinline__ uint32_t umma_idesc_bf16_mn(int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(128 >> 4) << 24);
+}
+
+__global__ void __launch_bounds__(192, 1)
+wgrad_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x, void* __restrict__ G,
+             int out_f32, int tokens, int rows, int cols, float scale, unsigned* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  WgBars* bars = reinterpret_cast<WgBars*>(smem + kWgStages * kWgStageBytes);
+  volatile int* abort_flag = &bars->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_m = (rows + kWgBM - 1) / kWgBM, tiles_n = (cols + kWgBN - 1) / kWgBN;
+  const int tiles = tiles_m * tiles_n;
+  const int kchunks = (tokens + kWgBK - 1) / kWgBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kWgStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 4); }
+    bars->abort_flag = 0;
+    bars->never_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) tmem_alloc(&bars->tmem_slot, 512);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool dead = false;
+      for (int tile = blockIdx.x; tile < tiles && !dead; tile += gridDim.x) {
+        const int tm = tile % tiles_m, tn = tile / tiles_m;
+        for (int kc = 0; kc < kchunks; ++kc, ++it) {
+          const int s = it % kWgStages;
+          if (!mbar_wait(&bars->empty[s], ((it / kWgStages) & 1) ^ 1, abort_flag)) { dead = true; break; }
+          uint8_t* st = smem + (size_t)s * kWgStageBytes;
+          mbar_expect_tx(&bars->full[s], kWgStageBytes);
+          // tokens past the end and rows / columns past the edge come in as zeros
+          for (int b = 0; b < kWgBM / 64; ++b)
+            tma_load_2d(st + b * kWgBox, &map_dy, &bars->full[s], tm * kWgBM + b * 64, kc * kWgBK);
+          for (int b = 0; b < kWgBN / 64; ++b)
+            tma_load_2d(st + kWgABytes + b * kWgBox, &map_x, &bars->full[s], tn * kWgBN + b * 64, kc * kWgBK);
+        }
+      }
+      if (dead) {
+        if (status) atomicOr(status, kDevTimeout);
+        *abort_flag = 1;
+        for (uint32_t u = it > (uint32_t)kWgStages ? it - kWgStages : 0; u < it; ++u)
+          mbar_wait(&bars->full[u % kWgStages], (u / kWgStages) & 1, &bars->never_flag);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16_mn(kWgBN);
+      uint32_t it = 0, t = 0;
+      bool dead = false;
+      for (int tile = blockIdx.x; tile < tiles && !dead; tile += gridDim.x, ++t) {
+        const uint32_t ab = t & 1;
+        if (!mbar_wait(&bars->acc_empty[ab], ((t >> 1) & 1) ^ 1, abort_flag)) { dead = true; break; }
+        tc_fence_after();
+        const uint32_t d = tmem_base + ab * kWgBN;
+        for (int kc = 0; kc < kchunks; ++kc, ++it) {
+          const int s = it % kWgStages;
+          if (!mbar_wait(&bars->full[s], (it / kWgStages) & 1, abort_flag)) { dead = true; break; }
+          tc_fence_after();
+          const uint32_t a0 = smem_u32(smem + (size_t)s * kWgStageBytes), b0 = a0 + kWgABytes;
+#pragma unroll
+          for (int k = 0; k < kWgBK / 16; ++k) {   // 16 tokens = two 8-row K groups = 2048 bytes per step
+            umma_bf16(d, umma_desc_mn_bf16(a0 + k * 2048, kWgBox), umma_desc_mn_bf16(b0 + k * 2048, kWgBox), idesc,
+                      (kc | k) != 0);
+          }
+          umma_commit(&bars->empty[s]);
+        }
+        if (dead) break;
+        umma_commit(&bars->acc_full[ab]);
+      }
+      if (dead) {
+        if (status) atomicOr(status, kDevTimeout);
+        *abort_flag = 1;
+      }
+    }
+    __syncwarp();
+  } else {
+    const int q = warp & 3;
+    uint32_t t = 0;
+    bool dead = false;
+    for (int tile = blockIdx.x; tile < tiles && !dead; tile += gridDim.x, ++t) {
+      const int tm = tile % tiles_m, tn = tile / tiles_m;
+      const uint32_t ab = t & 1;
+      if (!mbar_wait(&bars->acc_full[ab], (t >> 1) & 1, abort_flag)) { dead = true; break; }
+      tc_fence_after();
+      const int row = tm * kWgBM + q * 32 + lane;
+      const uint32_t d = tmem_base + ab * kWgBN + ((uint32_t)(q * 32) << 16);
+      for (int c = 0; c < kWgBN; c += 16) {
+        float v[16];
+        tmem_ld16(d + c, v);
+        tmem_ld_wait();
+        const int col = tn * kWgBN + c;
+        if (row < rows && col < cols) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] *= scale;
+          if (out_f32) {
+            float* o = static_cast<float*>(G) + (size_t)row * cols + col;
+#pragma unroll
+            for (int j = 0; j < 16; j += 8) {
+              if (col + j < cols) {     // cols is a multiple of 8
+                *reinterpret_cast<float4*>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                *reinterpret_cast<float4*>(o + j + 4) = make_float4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
+              }
+            }
+          } else {
+            bf16* o = static_cast<bf16*>(G) + (size_t)row * cols + col;
+#pragma unroll
+            for (int j = 0; j < 16; j += 8) {
+              if (col + j < cols) {
+                const __nv_bfloat162 p0 = __floats2bfloat162_rn(v[j], v[j + 1]), p1 = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
+                const __nv_bfloat162 p2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]), p3 = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
+                *reinterpret_cast<uint4*>(o + j) =
+                    make_uint4(*reinterpret_cast<const uint32_t*>(&p0), *reinterpret_cast<const uint32_t*>(&p1),
+                               *reinterpret_cast<const uint32_t*>(&p2), *reinterpret_cast<const uint32_t*>(&p3));
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->acc_empty[ab]);
+    }
+    if (dead && lane == 0) {
+      if (status) atomicOr(status, kDevTimeout);
+      *abort_flag = 1;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, 512);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// tokens x width bf16 row-major -> boxes of 64 (width) x 64 (tokens), 128-byte swizzle
+bool encode_mn(CUtensorMap* out, const void* base, int64_t tokens, int64_t width) {
+  EncodeTiledFn enc = encode_fn();
+  if (!enc) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)width, (cuuint64_t)tokens};
+  cuuint64_t strides[1] = {(cuuint64_t)width * 2};
+  cuuint32_t box[2] = {64, (cuuint32_t)kWgBK};
+  cuuint32_t estr[2] = {1, 1};
+  return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+}  // namespace sc
+
+using namespace sc;
+
+extern "C" sc_status sc_masked_weight_grad(const void* dY_dev, const void* X_dev, void* Xm_dev, void* G_dev,
+                                           int out_dtype, int64_t tokens, int64_t rows, int64_t cols, float keep,
+                                           uint64_t seed, uint32_t layer, uint64_t step, void* status_dev,
+                                           void* stream) {
+  if (!dY_dev || !X_dev || !Xm_dev || !G_dev) return SC_ERR_INVALID_ARG;
+  if (tokens <= 0 || rows <= 0 || cols <= 0 || tokens > (1 << 30) || rows > (1 << 30) || cols > (1 << 30))
+    return SC_ERR_INVALID_ARG;
+  if ((rows % 8) != 0 || (cols % 8) != 0) return SC_ERR_SHAPE;              // 16-byte row strides for TMA
+  if (out_dtype != SC_DTYPE_BF16 && out_dtype != SC_DTYPE_FP32) return SC_ERR_DTYPE;
+  if (!(keep > 0.f) || keep > 1.f) return SC_ERR_INVALID_ARG;
+  const uintptr_t al = reinterpret_cast<uintptr_t>(dY_dev) | reinterpret_cast<uintptr_t>(X_dev) |
+                       reinterpret_cast<uintptr_t>(Xm_dev) | reinterpret_cast<uintptr_t>(G_dev);
+  if (al & 15) return SC_ERR_ALIGNMENT;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  // Algorithm 1 line 4: Xm = X . M (unscaled; the 1 / keep goes into the GEMM's fp32 epilogue)
+  sc_status st = sc_apply_prf_mask(X_dev, Xm_dev, tokens, cols, keep, seed, layer, step, 0, stream);
+  if (st != SC_OK) return st;
+  long thr = lroundf(keep * 65536.f);
+  if (thr < 1) thr = 1;
+  if (thr > 65536) thr = 65536;
+  const float scale = 65536.f / (float)thr;
+
+  CUtensorMap map_dy, map_x;
+  if (!encode_mn(&map_dy, dY_dev, tokens, rows) || !encode_mn(&map_x, Xm_dev, tokens, cols)) return SC_ERR_CUDA;
+  int dev = 0, n_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return SC_ERR_CUDA;
+  const size_t smem = (size_t)kWgStages * kWgStageBytes + sizeof(WgBars) + 1024;
+  if (cudaFuncSetAttribute(wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return SC_ERR_CUDA;
+  const long long tiles = ((rows + kWgBM - 1) / kWgBM) * ((cols + kWgBN - 1) / kWgBN);
+  const int grid = tiles < n_sm ? (int)tiles : n_sm;
+  wgrad_kernel<<<grid, 192, smem, s>>>(map_dy, map_x, G_dev, out_dtype == SC_DTYPE_FP32, (int)tokens, (int)rows, (int)cols,
+                                       scale, static_cast<unsigned*>(status_dev));
+  ++g_kernel_launches;
+  return cudaGetLastError() == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+}
