@@ -8,8 +8,8 @@
 //
 // GEMM: G[rows x cols] = scale * A^T B with A = dY (tokens x rows) and B = Xm (tokens x cols), both row-major, i.e.
 // both operands are MN-major for the tensor core (the contraction index is the slow one in memory). Persistent blocks,
-// one per SM, tiles of 128 x 256 in row-tile-fastest order (blocks running side by side share the activation panel in
-// L2), K advancing 64 tokens per pipeline stage:
+// one per SM, tiles of 128 x 256 ordered so that the smaller of the two operands is the one the blocks running side by
+// side have in common (it stays in L2; the larger one is streamed once), K advancing 64 tokens per pipeline stage:
 //   warp 0   TMA producer: two 64 x 64 boxes of dY and four of Xm per stage (128-byte swizzle), 4-stage ring
 //   warp 1   tcgen05.mma kind::f16 issuer, M = 128, N = 256, fp32 accumulators, two 256-column buffers in TMEM
 //   warps 2-5  epilogue: TMEM -> registers -> scale -> bf16 or fp32 -> global
@@ -50,7 +50,7 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16_mn(int N) {
 
 __global__ void __launch_bounds__(192, 1)
 wgrad_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x, void* __restrict__ G,
-             int out_f32, int tokens, int rows, int cols, float scale, unsigned* status) {
+             int out_f32, int tokens, int rows, int cols, float scale, int n_fastest, unsigned* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   WgBars* bars = reinterpret_cast<WgBars*>(smem + kWgStages * kWgStageBytes);
@@ -79,7 +79,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
       uint32_t it = 0;
       bool dead = false;
       for (int tile = blockIdx.x; tile < tiles && !dead; tile += gridDim.x) {
-        const int tm = tile % tiles_m, tn = tile / tiles_m;
+        const int tm = n_fastest ? tile / tiles_n : tile % tiles_m, tn = n_fastest ? tile % tiles_n : tile / tiles_m;
         for (int kc = 0; kc < kchunks; ++kc, ++it) {
           const int s = it % kWgStages;
           if (!mbar_wait(&bars->empty[s], ((it / kWgStages) & 1) ^ 1, abort_flag)) { dead = true; break; }
@@ -136,7 +136,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
     uint32_t t = 0;
     bool dead = false;
     for (int tile = blockIdx.x; tile < tiles && !dead; tile += gridDim.x, ++t) {
-      const int tm = tile % tiles_m, tn = tile / tiles_m;
+      const int tm = n_fastest ? tile / tiles_n : tile % tiles_m, tn = n_fastest ? tile % tiles_n : tile / tiles_m;
       const uint32_t ab = t & 1;
       if (!mbar_wait(&bars->acc_full[ab], (t >> 1) & 1, abort_flag)) { dead = true; break; }
       tc_fence_after();
@@ -257,7 +257,7 @@ extern "C" sc_status sc_masked_weight_grad(const void* dY_dev, const void* X_dev
   const long long tiles = ((rows + kWgBM - 1) / kWgBM) * ((cols + kWgBN - 1) / kWgBN);
   const int grid = tiles < n_sm ? (int)tiles : n_sm;
   wgrad_kernel<<<grid, 192, smem, s>>>(map_dy, map_x, G_dev, out_dtype == SC_DTYPE_FP32, (int)tokens, (int)rows, (int)cols,
-                                       scale, static_cast<unsigned*>(status_dev));
+                                       scale, rows >= cols ? 1 : 0, static_cast<unsigned*>(status_dev));
   ++g_kernel_launches;
   return cudaGetLastError() == cudaSuccess ? SC_OK : SC_ERR_CUDA;
 }
