@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--workload", default="llama8b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--short", action="store_true", help="with --wgrad: time exactly --steps passes (profiler runs)")
+    ap.add_argument("--wgrad", action="store_true",
+                    help="time the masked weight gradients of one 8B-shaped layer (mask pass + tensor-core GEMM)")
     ap.add_argument("--sweep", action="store_true",
                     help="config 4: one 14336x4096 matrix, rank x keep grid; prints one JSON line with a 'cells' list")
     return ap.parse_args()
@@ -51,8 +54,9 @@ def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         d = json.load(open(path))
-        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]), source="measured")
-    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", 0.0)) or None, source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
 
 
 # ------------------------------------------------------------------------------------------ clocks
@@ -396,8 +400,89 @@ def run_sweep(args):
                       "cells": cells}), flush=True)
 
 
+def run_wgrad(args):
+    """The step before the hot path (Algorithm 1 lines 4-5): masked weight gradients of one 8B-shaped layer
+    (q, k, v, o, gate, up, down; 4096 tokens, keep 0.1) through sc_masked_weight_grad, i.e. the PRF mask pass plus
+    the tcgen05 GEMM over the tokens. Tensor-bound: the roofline is the measured bf16 GEMM peak."""
+    import torch
+    import paper_2609_14339_b200 as sc
+    from paper_2609_14339_b200 import build as _build
+    _build.build()
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    peaks = measured_peaks()
+    T, keep = 4096, 0.1
+    # (name, rows of W = width of dY, cols of W = width of X); q/k/v share X, gate/up share X
+    layers = [("q", 4096, 4096), ("k", 1024, 4096), ("v", 1024, 4096), ("o", 4096, 4096), ("gate", 14336, 4096),
+              ("up", 14336, 4096), ("down", 4096, 14336)]
+    g = torch.Generator(device=device); g.manual_seed(3)
+    X = {4096: torch.randn((T, 4096), generator=g, device=device).to(torch.bfloat16),
+         14336: torch.randn((T, 14336), generator=g, device=device).to(torch.bfloat16)}
+    Xm = {k: torch.empty_like(v) for k, v in X.items()}
+    dY = {r: torch.randn((T, r), generator=g, device=device).to(torch.bfloat16) for r in (1024, 4096, 14336)}
+    G = {nm: torch.empty((r, c), device=device, dtype=torch.bfloat16) for nm, r, c in layers}
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)      # larger than L2
+
+    def layer_pass(step):
+        for li, (nm, r, c) in enumerate(layers):
+            sc.masked_weight_grad(dY[r], X[c], keep, seed=1, layer=li, step=step, Xm=Xm[c], out=G[nm], status=status)
+
+    def mask_pass(step):
+        for li, (nm, r, c) in enumerate(layers):
+            sc.apply_prf_mask(X[c], keep, seed=1, layer=li, step=step, rescale=False, out=Xm[c])
+
+    for i in range(max(args.warmup, 3)):
+        layer_pass(i)
+    lib = sc.load_library()
+    launches0 = lib.sc_kernel_launch_count()
+    sampler = ClockSampler(0)
+    times, mask_times = [], []
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    steps = max(args.steps, 100) if not args.short else args.steps     # long enough for the clock sampler to see it
+    for i in range(steps):
+        flush.zero_()
+        e[0].record(); layer_pass(100 + i); e[1].record(); torch.cuda.synchronize()
+        times.append(e[0].elapsed_time(e[1]))
+    launches = lib.sc_kernel_launch_count() - launches0
+    clocks = sampler.stop()
+    for i in range(args.steps):
+        flush.zero_()
+        e[0].record(); mask_pass(100 + i); e[1].record(); torch.cuda.synchronize()
+        mask_times.append(e[0].elapsed_time(e[1]))
+    assert int(status.item()) == 0, "device status %d" % int(status.item())
+    ms, ms_mask = statistics.median(times), statistics.median(mask_times)
+    flops = sum(2.0 * T * r * c for _, r, c in layers)
+    gemm_tflops = flops / ((ms - ms_mask) * 1e-3) / 1e12
+    ref_times = []
+    for i in range(3 + args.steps):                                        # library GEMM on the same operands: context
+        flush.zero_()
+        e[0].record()
+        for nm, r, c in layers:
+            torch.matmul(dY[r].T, Xm[c], out=G[nm])
+        e[1].record(); torch.cuda.synchronize()
+        ref_times.append(e[0].elapsed_time(e[1]))
+    print(json.dumps({
+        "metric": "masked weight gradients of one 8B-shaped layer (7 matrices, 4096 tokens): TFLOP/s incl. the mask pass",
+        "value": flops / (ms * 1e-3) / 1e12, "unit": "TFLOP/s", "n_gpus": 1, "steps": steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "wgrad_llama8b_layer", "tokens": T, "keep": keep, "matrices": len(layers),
+                   "flops_per_step": flops, "l2": "256 MB buffer rewritten between timed iterations"},
+        "gpu_launches": launches, "mask_pass_ms": ms_mask,
+        "roofline": {"bound": "tensor", "kernel": "wgrad_kernel", "achieved": gemm_tflops, "peak": peaks["bf16_tflops"],
+                     "unit": "TFLOP/s", "frac": gemm_tflops / peaks["bf16_tflops"], "traffic": None,
+                     "peak_source": peaks["source"], "peak_sustained": peaks["bf16_tflops_sustained"],
+                     "note": "achieved = flops / (step time - mask pass time), both CUDA events; peak is the burst figure"},
+        "context": {"torch_matmul_tflops": flops / (statistics.median(ref_times[3:]) * 1e-3) / 1e12},
+        "clocks": clocks}), flush=True)
+
+
 def main():
     args = parse_args()
+    if args.wgrad:
+        run_wgrad(args)
+        return
     if args.sweep:
         run_sweep(args)
         return
