@@ -16,6 +16,8 @@
 // Every mbarrier wait is bounded; a wait that runs out latches SC_ERR_TIMEOUT in *status_dev and the block winds down.
 #include <cuda.h>
 
+#include <cstdlib>
+
 #include "sc_internal.cuh"
 #include "sc_ptx.cuh"
 
@@ -188,6 +190,215 @@ wgrad_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__
   if (warp == 1) tmem_dealloc(tmem_base, 512);
 }
 
+// -----------------------------------------------------------------------------------------------------------------
+// The same GEMM with two blocks (a cluster of two SMs) on one 256 x 256 tile: tcgen05.mma cta_group::2. Block t of the
+// pair loads rows t*128.. of the dY tile and columns t*128.. of the Xm tile, i.e. half the activation tile each, and the
+// tensor cores of both SMs read the two halves, so per SM and stage 32 KB go into shared memory instead of 48 KB for
+// the same number of flops; with one block per tile the tensor pipe waits for shared memory (75% busy). Block 0 (the
+// leader) issues the MMAs for both; its full barriers collect the bytes of both blocks' loads; its commits arrive on
+// the empty and accumulator barriers of both blocks; the epilogue warps of both blocks release the accumulator
+// through the leader's barrier. No multicast loads anywhere.
+// -----------------------------------------------------------------------------------------------------------------
+constexpr int kW2Stages = 6;
+constexpr int kW2ABytes = 2 * kWgBox, kW2BBytes = 2 * kWgBox;          // 128 rows of dY^T, 128 columns of Xm per block
+constexpr int kW2StageBytes = kW2ABytes + kW2BBytes;                   // 32 KB per block and stage
+
+struct W2Bars {
+  uint64_t full[kW2Stages], empty[kW2Stages];
+  uint64_t acc_full[2], acc_empty[2];
+  uint32_t tmem_slot;
+  int abort_flag;
+  int never_flag;
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in block `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load of the pair: the bytes are counted on the leader's barrier
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const void* map, uint32_t leader_bar, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(smem_u32(dst)), "l"(map), "r"(leader_bar), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc), "r"(0u)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {   // arrives on `bar` in both blocks of the pair
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"((uint16_t)3)
+               : "memory");
+}
+__device__ __forceinline__ uint32_t umma_idesc_bf16_mn_pair(int N) {   // M = 256 over the two blocks
+  return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(N >> 3) << 17) |
+         ((uint32_t)(256 >> 4) << 24);
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1)
+wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x,
+                  void* __restrict__ G, int out_f32, int tokens, int rows, int cols, float scale, int n_fastest,
+                  unsigned* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  W2Bars* bars = reinterpret_cast<W2Bars*>(smem + kW2Stages * kW2StageBytes);
+  volatile int* abort_flag = &bars->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int tiles_m = (rows + 255) / 256, tiles_n = (cols + 255) / 256;
+  const int tiles = tiles_m * tiles_n;
+  const int kchunks = (tokens + kWgBK - 1) / kWgBK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kW2Stages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 8); }
+    bars->abort_flag = 0;
+    bars->never_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars->tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();            // the peer's barriers exist before anything is sent to them
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool dead = false;
+      for (int tile = pair; tile < tiles && !dead; tile += n_pairs) {
+        const int tm = n_fastest ? tile / tiles_n : tile % tiles_m, tn = n_fastest ? tile % tiles_n : tile / tiles_m;
+        for (int kc = 0; kc < kchunks; ++kc, ++it) {
+          const int s = it % kW2Stages;
+          if (!mbar_wait(&bars->empty[s], ((it / kW2Stages) & 1) ^ 1, abort_flag)) { dead = true; break; }
+          uint8_t* st = smem + (size_t)s * kW2StageBytes;
+          if (rank == 0) mbar_expect_tx(&bars->full[s], 2 * kW2StageBytes);      // both blocks' bytes
+          const uint32_t leader_bar = map_to_rank(smem_u32(&bars->full[s]), 0);
+          for (int b = 0; b < 2; ++b)
+            tma_load_2d_pair(st + b * kWgBox, &map_dy, leader_bar, tm * 256 + (int)rank * 128 + b * 64, kc * kWgBK);
+          for (int b = 0; b < 2; ++b)
+            tma_load_2d_pair(st + kW2ABytes + b * kWgBox, &map_x, leader_bar, tn * 256 + (int)rank * 128 + b * 64,
+                             kc * kWgBK);
+        }
+      }
+      if (dead) {
+        if (status) atomicOr(status, kDevTimeout);
+        *abort_flag = 1;
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = umma_idesc_bf16_mn_pair(256);
+      uint32_t it = 0, t = 0;
+      bool dead = false;
+      for (int tile = pair; tile < tiles && !dead; tile += n_pairs, ++t) {
+        const uint32_t ab = t & 1;
+        if (!mbar_wait(&bars->acc_empty[ab], ((t >> 1) & 1) ^ 1, abort_flag)) { dead = true; break; }
+        tc_fence_after();
+        const uint32_t d = tmem_base + ab * 256;
+        for (int kc = 0; kc < kchunks; ++kc, ++it) {
+          const int s = it % kW2Stages;
+          if (!mbar_wait(&bars->full[s], (it / kW2Stages) & 1, abort_flag)) { dead = true; break; }
+          tc_fence_after();
+          const uint32_t a0 = smem_u32(smem + (size_t)s * kW2StageBytes), b0 = a0 + kW2ABytes;
+#pragma unroll
+          for (int k = 0; k < kWgBK / 16; ++k)
+            umma_bf16_pair(d, umma_desc_mn_bf16(a0 + k * 2048, kWgBox), umma_desc_mn_bf16(b0 + k * 2048, kWgBox), idesc,
+                           (kc | k) != 0);
+          umma_commit_pair(&bars->empty[s]);
+        }
+        if (dead) break;
+        umma_commit_pair(&bars->acc_full[ab]);
+      }
+      if (dead) {
+        if (status) atomicOr(status, kDevTimeout);
+        *abort_flag = 1;
+      }
+    }
+    __syncwarp();
+  } else {
+    const int q = warp & 3;
+    uint32_t t = 0;
+    bool dead = false;
+    for (int tile = pair; tile < tiles && !dead; tile += n_pairs, ++t) {
+      const int tm = n_fastest ? tile / tiles_n : tile % tiles_m, tn = n_fastest ? tile % tiles_n : tile / tiles_m;
+      const uint32_t ab = t & 1;
+      if (!mbar_wait(&bars->acc_full[ab], (t >> 1) & 1, abort_flag)) { dead = true; break; }
+      tc_fence_after();
+      const int row = tm * 256 + (int)rank * 128 + q * 32 + lane;
+      const uint32_t d = tmem_base + ab * 256 + ((uint32_t)(q * 32) << 16);
+      for (int c = 0; c < 256; c += 16) {
+        float v[16];
+        tmem_ld16(d + c, v);
+        tmem_ld_wait();
+        const int col = tn * 256 + c;
+        if (row < rows && col < cols) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] *= scale;
+          if (out_f32) {
+            float* o = static_cast<float*>(G) + (size_t)row * cols + col;
+#pragma unroll
+            for (int j = 0; j < 16; j += 8) {
+              if (col + j < cols) {
+                *reinterpret_cast<float4*>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                *reinterpret_cast<float4*>(o + j + 4) = make_float4(v[j + 4], v[j + 5], v[j + 6], v[j + 7]);
+              }
+            }
+          } else {
+            bf16* o = static_cast<bf16*>(G) + (size_t)row * cols + col;
+#pragma unroll
+            for (int j = 0; j < 16; j += 8) {
+              if (col + j < cols) {
+                const __nv_bfloat162 p0 = __floats2bfloat162_rn(v[j], v[j + 1]), p1 = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
+                const __nv_bfloat162 p2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]), p3 = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
+                *reinterpret_cast<uint4*>(o + j) =
+                    make_uint4(*reinterpret_cast<const uint32_t*>(&p0), *reinterpret_cast<const uint32_t*>(&p1),
+                               *reinterpret_cast<const uint32_t*>(&p2), *reinterpret_cast<const uint32_t*>(&p3));
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_rank(smem_u32(&bars->acc_empty[ab]), 0));   // the leader's barrier
+    }
+    if (dead && lane == 0) {
+      if (status) atomicOr(status, kDevTimeout);
+      *abort_flag = 1;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();            // nothing of the peer is touched after this
+  if (warp == 1)
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -254,10 +465,23 @@ extern "C" sc_status sc_masked_weight_grad(const void* dY_dev, const void* X_dev
   const size_t smem = (size_t)kWgStages * kWgStageBytes + sizeof(WgBars) + 1024;
   if (cudaFuncSetAttribute(wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return SC_ERR_CUDA;
-  const long long tiles = ((rows + kWgBM - 1) / kWgBM) * ((cols + kWgBN - 1) / kWgBN);
-  const int grid = tiles < n_sm ? (int)tiles : n_sm;
-  wgrad_kernel<<<grid, 192, smem, s>>>(map_dy, map_x, G_dev, out_dtype == SC_DTYPE_FP32, (int)tokens, (int)rows, (int)cols,
-                                       scale, rows >= cols ? 1 : 0, static_cast<unsigned*>(status_dev));
+  static const bool pair_off = getenv("SC_WGRAD_ONE_CTA") != nullptr;       // test hook: force the one-block-per-tile kernel
+  const long long tiles2 = ((rows + 255) / 256) * ((cols + 255) / 256);
+  if (!pair_off && rows >= 256 && cols >= 256 && n_sm >= 2) {
+    // pairs of SMs on 256 x 256 tiles (tcgen05 cta_group::2)
+    const size_t smem2 = (size_t)kW2Stages * kW2StageBytes + sizeof(W2Bars) + 1024;
+    if (cudaFuncSetAttribute(wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
+      return SC_ERR_CUDA;
+    const int n_pairs = tiles2 < n_sm / 2 ? (int)tiles2 : n_sm / 2;
+    wgrad_pair_kernel<<<2 * n_pairs, 192, smem2, s>>>(map_dy, map_x, G_dev, out_dtype == SC_DTYPE_FP32, (int)tokens,
+                                                      (int)rows, (int)cols, scale, rows >= cols ? 1 : 0,
+                                                      static_cast<unsigned*>(status_dev));
+  } else {
+    const long long tiles = ((rows + kWgBM - 1) / kWgBM) * ((cols + kWgBN - 1) / kWgBN);
+    const int grid = tiles < n_sm ? (int)tiles : n_sm;
+    wgrad_kernel<<<grid, 192, smem, s>>>(map_dy, map_x, G_dev, out_dtype == SC_DTYPE_FP32, (int)tokens, (int)rows,
+                                         (int)cols, scale, rows >= cols ? 1 : 0, static_cast<unsigned*>(status_dev));
+  }
   ++g_kernel_launches;
   return cudaGetLastError() == cudaSuccess ? SC_OK : SC_ERR_CUDA;
 }
