@@ -470,7 +470,7 @@ def run_wgrad(args):
         "config": {"workload": "wgrad_llama8b_layer", "tokens": T, "keep": keep, "matrices": len(layers),
                    "flops_per_step": flops, "l2": "256 MB buffer rewritten between timed iterations"},
         "gpu_launches": launches, "mask_pass_ms": ms_mask,
-        "roofline": {"bound": "tensor", "kernel": "wgrad_kernel", "achieved": gemm_tflops, "peak": peaks["bf16_tflops"],
+        "roofline": {"bound": "tensor", "kernel": "wgrad_pair_kernel", "achieved": gemm_tflops, "peak": peaks["bf16_tflops"],
                      "unit": "TFLOP/s", "frac": gemm_tflops / peaks["bf16_tflops"], "traffic": None,
                      "peak_source": peaks["source"], "peak_sustained": peaks["bf16_tflops_sustained"],
                      "note": "achieved = flops / (step time - mask pass time), both CUDA events; peak is the burst figure"},
