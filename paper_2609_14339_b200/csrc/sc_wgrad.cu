@@ -8,12 +8,14 @@
 //
 // GEMM: G[rows x cols] = scale * A^T B with A = dY (tokens x rows) and B = Xm (tokens x cols), both row-major, i.e.
 // both operands are MN-major for the tensor core (the contraction index is the slow one in memory). Persistent blocks,
-// one per SM, tiles of 128 x 256 ordered so that the smaller of the two operands is the one the blocks running side by
-// side have in common (it stays in L2; the larger one is streamed once), K advancing 64 tokens per pipeline stage:
-//   warp 0   TMA producer: two 64 x 64 boxes of dY and four of Xm per stage (128-byte swizzle), 4-stage ring
-//   warp 1   tcgen05.mma kind::f16 issuer, M = 128, N = 256, fp32 accumulators, two 256-column buffers in TMEM
-//   warps 2-5  epilogue: TMEM -> registers -> scale -> bf16 or fp32 -> global
-// Every mbarrier wait is bounded; a wait that runs out latches SC_ERR_TIMEOUT in *status_dev and the block winds down.
+// tiles ordered so that the smaller of the two operands is the one the blocks running side by side have in common (it
+// stays in L2; the larger one is streamed once), K advancing 64 tokens per pipeline stage. Two kernels:
+//   wgrad_pair_kernel   outputs of at least 256 x 256: clusters of two SMs on 256 x 256 tiles, tcgen05 cta_group::2
+//   wgrad_kernel        anything smaller: one block per 128 x 256 tile
+// Warp roles in both: warp 0 TMA producer (64 x 64 boxes, 128-byte swizzle), warp 1 tcgen05.mma kind::f16 issuer with
+// fp32 accumulators in two 256-column TMEM buffers, warps 2-5 epilogue (TMEM -> registers -> scale -> bf16 or fp32 ->
+// global). Every mbarrier wait is bounded; a wait that runs out latches the time-out bit in *status_dev and the block
+// winds down.
 #include <cuda.h>
 
 #include <cstdlib>
