@@ -79,3 +79,38 @@ def test_rejects_bad_arguments(torch):
     assert lib.sc_masked_weight_grad(p, p, p, p + 2, 0, 16, 8, 8, 0.5, 0, 0, 0, None, None) == -4   # alignment
     assert lib.sc_masked_weight_grad(p, p, p, p, 0, 16, 8, 8, 1.5, 0, 0, 0, None, None) == -1       # keep
     assert lib.sc_masked_weight_grad(None, p, p, p, 0, 16, 8, 8, 0.5, 0, 0, 0, None, None) == -1
+
+
+def test_from_activations_to_the_corrected_step(torch):
+    """Algorithm 1 lines 4-14 on the GPU from the activations on: masked weight gradients from sc_masked_weight_grad
+    (anchor gradients from the same call with keep = 1 on an independent batch), then the anchor update and the
+    corrected AdamW step; the oracle forms its own gradients in fp64 from the same X, dY and the oracle's mask."""
+    import paper_2609_14339_b200 as sc
+    from parity_util import Case, GpuRun, OracleRun, compare_step, make_inputs
+    shapes = [(512, 256), (256, 512), (384, 384)]
+    case = Case(shapes=shapes, rank=16, tokens=384, keep=0.25, planted=8, seed=7, tau_p=50.0, prescaled=True)
+    inp_o = make_inputs(case)                     # optimizer state and specs; gradients are replaced below
+    inp_g = dict(inp_o, anchors=[None] * len(shapes), G=[None] * len(shapes))
+    inp_o = dict(inp_o, anchors=[None] * len(shapes), G=[None] * len(shapes))
+    bits = lambda t: t.view(torch.int16).cpu().numpy().view(np.uint16)
+    for i, spec in enumerate(inp_o["specs"]):
+        Xa, dYa = gen.batch(spec, 0)              # the anchor circuit's unmasked batch
+        X, dY = gen.batch(spec, 2)                # the fast circuit's batch
+        dev = lambda a: torch.from_numpy(a.astype(np.float32)).cuda().to(torch.bfloat16)
+        Xab, dYab, Xb, dYb = dev(Xa), dev(dYa), dev(X), dev(dY)
+        Ganc, _ = sc.masked_weight_grad(dYab, Xab, 1.0, seed=3, layer=i, step=0)
+        G, _ = sc.masked_weight_grad(dYb, Xb, case.keep, seed=3, layer=i, step=2)
+        torch.cuda.synchronize()
+        inp_g["anchors"][i] = [bits(Ganc)]
+        inp_g["G"][i] = bits(G)
+        f64 = lambda t: t.double().cpu().numpy()
+        M = so.prf_keep_mask(3, i, 2, case.tokens, spec.n, case.keep)
+        inp_o["anchors"][i] = [gen.round_to(f64(dYab).T @ f64(Xab), "bf16")]
+        inp_o["G"][i] = gen.round_to(so.masked_weight_gradient(f64(dYb), f64(Xb), M, case.keep), "bf16")
+        # the two sides' stored gradients differ only where the fp32 sum lands on the other side of a bf16 rounding point
+        assert rel(gen.stored_to_f64(inp_g["G"][i], "bf16"), gen.stored_to_f64(inp_o["G"][i], "bf16")) < 5e-4
+    g = GpuRun(case, inp_g, torch)
+    assert g.uses_tc and g.dev_status == 0
+    o = OracleRun(case, inp_o, "mirror")
+    es = compare_step(g, o)
+    assert max(es["gproj"], es["m"], es["v"], es["dW"]) < TOL_BF16, es
