@@ -189,3 +189,55 @@ def test_global_clipping_and_in_step_rescale_on_the_tensor_engine(torch):
     total = sum(np.sum(x * x) for x in g.gproj)
     assert abs(np.sqrt(total) - 0.2) < 2e-4
     assert 0.0 < g.clip < 1.0
+
+
+def test_every_tile_of_every_matrix_is_updated_exactly_once(torch):
+    """Thousands of work items over ten matrices of two shape classes (the update kernel hands them out through an
+    atomic counter): every element of every matrix against the CUDA-core engine run from the same basis, and a second
+    run of the tensor-core engine from the same state bit for bit."""
+    import paper_2609_14339_b200 as sc
+    dev = torch.device("cuda", 0)
+    shapes = [(1024, 2048)] * 6 + [(1536, 1024)] * 4
+    g = torch.Generator(device=dev); g.manual_seed(17)
+    rnd = lambda s, scale=1.0: torch.randn(s, generator=g, device=dev) * scale
+    # low-rank signal plus noise, so that the basis is well defined
+    def grad(s, seed_rank=8):
+        m, n = s
+        return (rnd((m, seed_rank)) @ rnd((seed_rank, n)) * 3.0 + rnd(s)).to(torch.bfloat16)
+    Ga = [grad(s) for s in shapes]
+    G = [grad(s) for s in shapes]
+    W0 = [rnd(s, 0.02) for s in shapes]
+    m0 = [rnd(s, 0.1) for s in shapes]
+    v0 = [torch.rand(s, generator=g, device=dev) * 4.0 + 0.1 for s in shapes]
+
+    def run(engine, bases=None):
+        hp = sc.Hparams.default(tau_p=60.0, lr=1e-2, weight_decay=0.01, engine=engine)
+        plan = sc.Plan(shapes, 32, 0.25, hp, device=dev)
+        plan.anchor_update(Ga, 0)
+        if bases is not None:
+            for i, (U, s, V) in enumerate(bases):
+                plan.import_basis(i, U, s, V)
+        W = [x.clone() for x in W0]; m = [x.clone() for x in m0]; v = [x.clone() for x in v0]
+        Wb = [torch.zeros(s, dtype=torch.bfloat16, device=dev) for s in shapes]
+        assert plan.correct_and_step(G, W, m, v, 50, params_bf16=Wb) == 0
+        torch.cuda.synchronize()
+        assert plan.get_device_status() == 0
+        out_bases = [plan.export_basis(i) for i in range(len(shapes))]
+        used_tc = plan.uses_tensor_cores()
+        plan.close()
+        return W, m, v, Wb, out_bases, used_tc
+
+    W1, m1, v1, Wb1, bases, tc1 = run(sc.SC_ENGINE_AUTO)
+    W2, m2, v2, Wb2, _, tc2 = run(sc.SC_ENGINE_AUTO)
+    assert tc1 and tc2
+    for a, b in zip(W1 + m1 + v1 + Wb1, W2 + m2 + v2 + Wb2):
+        assert torch.equal(a, b)
+    W3, m3, v3, Wb3, _, tc3 = run(sc.SC_ENGINE_SIMT, bases)
+    assert not tc3
+    for i in range(len(shapes)):
+        dW1 = (W1[i] - W0[i]).double(); dW3 = (W3[i] - W0[i]).double()
+        assert float((dW1 - dW3).norm() / dW3.norm()) < 1e-4, i
+        assert float((m1[i] - m3[i]).double().norm() / m3[i].double().norm()) < 1e-5, i
+        assert float((v1[i] - v3[i]).double().norm() / v3[i].double().norm()) < 1e-5, i
+        # element-wise as well: a tile applied twice or not at all moves dW by its whole size there
+        assert float((dW1 - dW3).abs().max()) < 2e-2 * float(dW3.abs().max()), i
