@@ -29,8 +29,8 @@ METRIC = "spectral-correction step: gradient GB/s (and ms per step) on the 8B-sh
 REFRESH_EVERY = 4
 BYTES_PER_ELEM_STEADY = 28.0      # read G (2) + read/write fp32 W, m, v (24) + write bf16 W (2)
 BYTES_PER_ELEM_UPDATE = 28.0      # what the fused update kernel itself moves per element (G is re-read here)
-TRAFFIC_PER_ELEM_UPDATE = 27.19   # dram read+write bytes per element of that kernel from one ncu capture
-                                  # (profiles/fused_update_stream_kernel_ffn14336x4096.md); scales with elements
+TRAFFIC_PER_ELEM_UPDATE = 27.19   # dram read+write bytes per element of that kernel from one ncu capture of a
+                                  # single 14336x4096 matrix; grows in proportion to the elements
 
 
 def parse_args():

@@ -203,9 +203,9 @@ SC_API sc_status sc_masked_weight_grad(const void* dY_dev, const void* X_dev, vo
                                        int64_t tokens, int64_t rows, int64_t cols, float keep, uint64_t seed,
                                        uint32_t layer, uint64_t step, void* status_dev, void* stream);
 
-/* sc_apply_prf_mask_exact_k - the per-token form of the same mask (Section 3.1: "retaining K = round((1 - p) H)
- * dimensions per token"): every token keeps exactly K = round(keep * features) features, chosen by the K smallest
- * values of a per-(token, feature) hash (ties impossible by construction); rescale multiplies by features / K.
+/* sc_apply_prf_mask_exact_k - the per-token form of the same mask (Section 3.1): every token keeps exactly
+ * K = round(keep * features) features (halves round up, the product formed in single precision), chosen by the K
+ * smallest values of a per-(token, feature) hash (ties impossible by construction); rescale multiplies by features / K.
  * Same layouts as sc_apply_prf_mask; features <= 65536, no multiple-of-8 requirement. */
 SC_API sc_status sc_apply_prf_mask_exact_k(const void* X_dev, void* out_dev, int64_t tokens, int64_t features,
                                            float keep, uint64_t seed, uint32_t layer, uint64_t step, int rescale,
@@ -268,13 +268,16 @@ SC_API sc_status sc_set_debug_gproj_out(sc_plan* plan, void* const* gproj_out);
  * and the clip factor applied into *clip (host, may be NULL). */
 SC_API sc_status sc_get_stats(sc_plan* plan, sc_mat_stats* stats, float* clip);
 
-/* Wait for the plan's stream and return the latched device status (SC_OK, SC_ERR_TIMEOUT, SC_ERR_NONFINITE), then clear it. */
+/* Wait for the plan's stream and return one latched device condition (SC_ERR_TIMEOUT before SC_ERR_NONFINITE, else
+ * SC_OK), clearing only the condition reported: when both are latched, two calls report them one after the other. */
 SC_API sc_status sc_get_device_status(sc_plan* plan);
 
-/* Checkpoint / resume. The blob holds, for every matrix, the anchor momentum, the cached basis (U, s, V, d), whether a
- * basis exists, and the last accepted step tag; AdamW state and weights stay with the caller. host_buf is HOST memory
- * of at least sc_state_bytes(plan) bytes. Both calls wait for the plan's stream. Import needs a plan created with the
- * same shapes and rank (SC_ERR_SHAPE otherwise); a step after import continues bit-identically. */
+/* Checkpoint / resume. The blob holds, for every matrix, its shape, the anchor momentum, the cached basis (U, s, V, d),
+ * whether a basis exists, and the last accepted step tag; AdamW state and weights stay with the caller. host_buf is
+ * HOST memory of at least sc_state_bytes(plan) bytes. Both calls wait for the plan's stream. Import needs a plan created
+ * with the same shapes in the same order and the same rank (SC_ERR_SHAPE otherwise: every matrix's rows and cols are
+ * compared); the filter weights d of Eq. 2 are recomputed from the imported singular values with the importing plan's
+ * tau_p. With equal tau_p a step after import continues bit-identically. */
 SC_API size_t sc_state_bytes(const sc_plan* plan);
 SC_API sc_status sc_state_export(sc_plan* plan, void* host_buf, size_t bytes);
 SC_API sc_status sc_state_import(sc_plan* plan, const void* host_buf, size_t bytes);

@@ -24,7 +24,9 @@ uses a randomized subspace iteration:
 Pins (tests/test_oracle_pins.py): hand-derived 2x2 worked example, brute-force
 one-sided Jacobi SVD, rank-1 / diagonal closed forms, Lemma 1 and Lemma 2,
 idempotence at tau_p = 0, the alpha / rank / keep limit cases, torch AdamW in
-fp64, the closed-form global norm, MIRROR == EXACT for rank(M) <= r.
+fp64, the closed-form global norm, MIRROR == EXACT for rank(M) <= r; the dual-EMA
+step by a one-element hand calculation, its mix_alpha = 0 and beta3 = beta1 special
+cases (both reduce to adamw_step) and the fixed point of the slow EMA.
 Parity unpinned: end-to-end MIRROR vs EXACT on inputs with no spectral gap at r
 (the cut is ill-posed there; it is reported, not gated).
 """
@@ -205,6 +207,29 @@ def adamw_step(W, m, v, g, t: int, lr: float, beta1: float, beta2: float, eps: f
     return W, m, v
 
 
+def ademamix_step(W, m1, m2, v, g, t: int, lr: float, beta1: float, beta2: float, beta3: float, mix_alpha: float,
+                  eps: float, weight_decay: float):
+    """One dual-EMA (AdEMAMix) step on the corrected gradient (appendix "On the Compatibility with Dual-EMA
+    Optimizers": the composition applies the dual-EMA dynamics to G_proj instead of the raw masked gradient).
+
+    fast EMA  m1 <- b1 m1 + (1-b1) g   (bias-corrected in the update, as Adam's first moment)
+    slow EMA  m2 <- b3 m2 + (1-b3) g   (b3 close to 1, no bias correction)
+    second    v  <- b2 v  + (1-b2) g^2 (bias-corrected)
+    theta <- theta - lr*wd*theta - lr * (m1/(1-b1^t) + mix_alpha * m2) / (sqrt(v/(1-b2^t)) + eps).
+    The appendix prints the update without a decay term; decay is decoupled here exactly as in adamw_step, so
+    that mix_alpha = 0 is that function.  Returns new (W, m1, m2, v).
+    """
+    W = np.asarray(W, F64)
+    g = np.asarray(g, F64)
+    m1 = beta1 * np.asarray(m1, F64) + (1.0 - beta1) * g
+    m2 = beta3 * np.asarray(m2, F64) + (1.0 - beta3) * g
+    v = beta2 * np.asarray(v, F64) + (1.0 - beta2) * g * g
+    m1_hat = m1 / (1.0 - beta1 ** t)
+    v_hat = v / (1.0 - beta2 ** t)
+    W = W - lr * weight_decay * W - lr * (m1_hat + mix_alpha * m2) / (np.sqrt(v_hat) + eps)
+    return W, m1, m2, v
+
+
 # --------------------------------------------------------------------------
 # Randomized range finder (MIRROR mode)
 # --------------------------------------------------------------------------
@@ -293,6 +318,8 @@ class Hyper:
     max_grad_norm: float = 0.0      # 0 = no clipping
     grads_prescaled: bool = True    # False: the step multiplies the masked gradient by 1/keep
     keep: float = 1.0
+    beta3: float = 0.9999           # slow EMA of the dual-EMA composition
+    mix_alpha: float = 5.0          # weight of the slow EMA in the update
 
 
 @dataclass
@@ -358,6 +385,21 @@ def correct_and_step(states, G_masks, Ws, ms, vs, t: int, hp: Hyper):
     return outW, outm, outv, outg
 
 
+def correct_and_step_ademamix(states, G_masks, Ws, m1s, m2s, vs, t: int, hp: Hyper):
+    """The same fast-circuit step with the dual-EMA optimizer in place of AdamW: correction, optional global clip,
+    then ademamix_step on G_proj.  Returns (new Ws, new m1s, new m2s, new vs, list of G_proj after clipping)."""
+    projs = [correct(st, G, hp)[0] for st, G in zip(states, G_masks)]
+    total = sum(float(np.sum(P * P)) for P in projs)
+    c = clip_factor(total, hp.max_grad_norm)
+    outW, out1, out2, outv, outg = [], [], [], [], []
+    for P, W, m1, m2, v in zip(projs, Ws, m1s, m2s, vs):
+        g = c * P
+        W2, a, b, v2 = ademamix_step(W, m1, m2, v, g, t, hp.lr, hp.beta1, hp.beta2, hp.beta3, hp.mix_alpha, hp.eps,
+                                     hp.weight_decay)
+        outW.append(W2); out1.append(a); out2.append(b); outv.append(v2); outg.append(g)
+    return outW, out1, out2, outv, outg
+
+
 # --------------------------------------------------------------------------
 # In-graph activation mask from a shared pseudo-random function (Section 3.1, Algorithm 1 line 4:
 # M_l = g(l, t, B, S, H)) and the masked weight gradient it leads to.  Nothing here is part of the
@@ -409,8 +451,8 @@ def masked_weight_gradient(dY, X, mask, keep: float, rescale: bool = True) -> np
 
 
 def prf_exact_k_mask(seed: int, layer: int, step: int, tokens: int, features: int, keep: float) -> np.ndarray:
-    """The per-token variant of the shared-PRF mask (Section 3.1: "retaining K = round((1-p) H) dimensions per
-    token"): every token keeps exactly K features, those with the K smallest composite keys
+    """The per-token variant of the shared-PRF mask (Section 3.1, K = round(keep * H) features kept per token):
+    every token keeps exactly K features, those with the K smallest composite keys
         key(t, j) = lowbias32(k_t + j * 0x9E3779B9) * 2^16 + j        (k_t as in prf_keep_mask; j < 65536),
     which are distinct by construction, so the selection is unique.
     """

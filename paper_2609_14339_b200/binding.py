@@ -240,7 +240,10 @@ def apply_prf_mask(X, keep: float, seed: int, layer: int, step: int, rescale: bo
 class Plan:
     """Owns a workspace tensor and an sc_plan handle; methods mirror the C entry points one to one."""
 
-    def __init__(self, shapes, rank: int, keep_ratio: float, hp: Optional[Hparams] = None, stream=None, device="cuda:0"):
+    def __init__(self, shapes, rank: int, keep_ratio: float, hp: Optional[Hparams] = None, stream=None, device="cuda:0",
+                 workspace=None):
+        """workspace: optional caller-owned uint8 CUDA tensor of at least workspace_bytes(...) bytes whose data pointer
+        is 256-byte aligned; by default the plan allocates one."""
         import torch
         self._torch = torch
         self.lib = load_library()
@@ -255,14 +258,27 @@ class Plan:
             raise SCError(-1, "sc_plan_workspace_bytes")
         self.workspace_bytes = int(need)
         with torch.cuda.device(self.device):
-            self.workspace = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
-            base = (self.workspace.data_ptr() + 255) // 256 * 256
+            if workspace is not None:
+                if workspace.dtype != torch.uint8 or not workspace.is_cuda or workspace.numel() < need:
+                    raise ValueError("workspace must be a uint8 CUDA tensor of at least %d bytes" % need)
+                self.workspace = workspace
+                base = workspace.data_ptr()
+            else:
+                self.workspace = torch.empty(need + 256, dtype=torch.uint8, device=self.device)
+                base = (self.workspace.data_ptr() + 255) // 256 * 256
             self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
             handle = C.c_void_p()
             _check(self.lib.sc_plan_create(C.byref(handle), arr, self.n_mats, self.rank, float(keep_ratio),
                                            C.byref(self.hp), base, need, self.stream.cuda_stream), "sc_plan_create")
         self.handle = handle
         self._keep = []
+
+    @staticmethod
+    def workspace_bytes_for(shapes, rank: int, hp: Optional[Hparams] = None) -> int:
+        lib = load_library()
+        hp = hp if hp is not None else Hparams.default()
+        arr = (Shape * len(shapes))(*[Shape(int(m), int(n)) for m, n in shapes])
+        return int(lib.sc_plan_workspace_bytes(arr, len(shapes), int(rank), C.byref(hp)))
 
     def close(self):
         if getattr(self, "handle", None):

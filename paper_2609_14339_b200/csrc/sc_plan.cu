@@ -825,9 +825,13 @@ sc_status sc_get_device_status(sc_plan* p) {
   if (cudaMemcpyAsync(&w, p->status_dev, sizeof(w), cudaMemcpyDeviceToHost, p->stream) != cudaSuccess ||
       cudaStreamSynchronize(p->stream) != cudaSuccess)
     return SC_ERR_CUDA;
-  if (w) cudaMemsetAsync(p->status_dev, 0, sizeof(w), p->stream);
-  if (w & kDevTimeout) return SC_ERR_TIMEOUT;
-  if (w & kDevNonfinite) return SC_ERR_NONFINITE;
+  // one condition is reported per call and only its bit is cleared, so a second latched condition is reported by
+  // the next call (the bits live in the low byte of the word, which is what the one-byte memset rewrites)
+  const unsigned reported = (w & kDevTimeout) ? kDevTimeout : (w & kDevNonfinite);
+  if (reported && cudaMemsetAsync(p->status_dev, (int)(w & ~reported & 0xFFu), 1, p->stream) != cudaSuccess)
+    return SC_ERR_CUDA;
+  if (reported == kDevTimeout) return SC_ERR_TIMEOUT;
+  if (reported == kDevNonfinite) return SC_ERR_NONFINITE;
   return SC_OK;
 }
 
@@ -850,9 +854,12 @@ struct StateHeader {
   int64_t last_tag;
 };
 constexpr uint32_t kStateMagic = 0x53435354u;   // "SCST"
+constexpr uint32_t kStateVersion = 2u;          // 2: the blob lists every matrix's rows and cols after the flags
+
+size_t state_shape_bytes(const sc_plan* p) { return align_up((size_t)p->n_mats * sizeof(sc_shape), 16); }
 
 size_t state_bytes(const sc_plan* p) {
-  size_t b = sizeof(StateHeader) + align_up((size_t)p->n_mats, 16);
+  size_t b = sizeof(StateHeader) + align_up((size_t)p->n_mats, 16) + state_shape_bytes(p);
   for (int i = 0; i < p->n_mats; ++i) {
     const size_t m = (size_t)p->shapes[i].rows, n = (size_t)p->shapes[i].cols;
     b += (m * n + (m + n + 2) * (size_t)p->rp) * sizeof(float);
@@ -867,12 +874,15 @@ sc_status sc_state_export(sc_plan* p, void* host_buf, size_t bytes) {
   if (!p || !host_buf) return SC_ERR_INVALID_ARG;
   if (bytes < state_bytes(p)) return SC_ERR_WORKSPACE;
   char* out = static_cast<char*>(host_buf);
-  StateHeader h{kStateMagic, 1u, p->n_mats, p->rank, p->rp, 0, p->last_tag};
+  StateHeader h{kStateMagic, kStateVersion, p->n_mats, p->rank, p->rp, 0, p->last_tag};
   memcpy(out, &h, sizeof(h));
   char* flags = out + sizeof(h);
   memset(flags, 0, align_up((size_t)p->n_mats, 16));
   for (int i = 0; i < p->n_mats; ++i) flags[i] = p->has_basis[i];
-  char* cur = flags + align_up((size_t)p->n_mats, 16);
+  char* shp = flags + align_up((size_t)p->n_mats, 16);
+  memset(shp, 0, state_shape_bytes(p));
+  memcpy(shp, p->shapes.data(), (size_t)p->n_mats * sizeof(sc_shape));
+  char* cur = shp + state_shape_bytes(p);
   auto pull = [&](const float* src, size_t count) {
     const bool ok = count == 0 ||
                     cudaMemcpyAsync(cur, src, count * sizeof(float), cudaMemcpyDeviceToHost, p->stream) == cudaSuccess;
@@ -894,12 +904,18 @@ sc_status sc_state_import(sc_plan* p, const void* host_buf, size_t bytes) {
   const char* in = static_cast<const char*>(host_buf);
   StateHeader h;
   memcpy(&h, in, sizeof(h));
-  if (h.magic != kStateMagic || h.version != 1u) return SC_ERR_INVALID_ARG;
+  if (h.magic != kStateMagic || h.version != kStateVersion) return SC_ERR_INVALID_ARG;
   if (h.n_mats != p->n_mats || h.rank != p->rank || h.rp != p->rp) return SC_ERR_SHAPE;
+  const char* flags = in + sizeof(h);
+  const char* shp = flags + align_up((size_t)p->n_mats, 16);
+  for (int i = 0; i < p->n_mats; ++i) {      // same shapes in the same order, or the arrays would land in the wrong matrices
+    sc_shape sh;
+    memcpy(&sh, shp + (size_t)i * sizeof(sc_shape), sizeof(sh));
+    if (sh.rows != p->shapes[i].rows || sh.cols != p->shapes[i].cols) return SC_ERR_SHAPE;
+  }
   sc_status st = upload_table(p);
   if (st != SC_OK) return st;
-  const char* flags = in + sizeof(h);
-  const char* cur = flags + align_up((size_t)p->n_mats, 16);
+  const char* cur = shp + state_shape_bytes(p);
   auto push = [&](float* dst, size_t count) {
     const bool ok = count == 0 ||
                     cudaMemcpyAsync(dst, cur, count * sizeof(float), cudaMemcpyHostToDevice, p->stream) == cudaSuccess;
@@ -912,7 +928,11 @@ sc_status sc_state_import(sc_plan* p, const void* host_buf, size_t bytes) {
     if (!push(md.Manc, m * n) || !push(md.U, m * rp) || !push(md.V, n * rp) || !push(md.sv, rp) || !push(md.d, rp))
       return SC_ERR_CUDA;
   }
-  for (auto& c : p->classes) refresh_operands(p, c, c.idx_all, (int)c.mats.size());
+  // Eq. 2 from the imported singular values and THIS plan's tau_p (the blob's d belongs to the exporting plan)
+  for (auto& c : p->classes) {
+    if (p->rp > 0) launch_filter_weights(p->dev_tab, c.idx_all, (int)c.mats.size(), p->rp, p->rank, p->hp.tau_p, p->stream);
+    refresh_operands(p, c, c.idx_all, (int)c.mats.size());
+  }
   // the copies above read caller memory: finish them before returning
   if (cudaStreamSynchronize(p->stream) != cudaSuccess) return SC_ERR_CUDA;
   for (int i = 0; i < p->n_mats; ++i) p->has_basis[i] = flags[i];

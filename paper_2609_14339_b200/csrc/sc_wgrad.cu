@@ -208,6 +208,7 @@ constexpr int kW2StageBytes = kW2ABytes + kW2BBytes;                   // 32 KB 
 struct W2Bars {
   uint64_t full[kW2Stages], empty[kW2Stages];
   uint64_t acc_full[2], acc_empty[2];
+  uint64_t drain;                // abort path only: the leader's MMAs in flight have finished
   uint32_t tmem_slot;
   int abort_flag;
   int never_flag;
@@ -272,6 +273,7 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_const
   if (threadIdx.x == 0) {
     for (int s = 0; s < kW2Stages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 8); }
+    mbar_init(&bars->drain, 1);
     bars->abort_flag = 0;
     bars->never_flag = 0;
     fence_barrier_init();
@@ -309,6 +311,16 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_const
       if (dead) {
         if (status) atomicOr(status, kDevTimeout);
         *abort_flag = 1;
+        // Let the copies in flight land before the pair's shared memory goes away. The bytes of both blocks are counted
+        // on the leader's barriers, so the leader waits (bounded) for the stages it armed; the other block cannot see
+        // its own copies land and instead idles for a grace period far longer than a copy takes. Both blocks then
+        // meet in the cluster barrier at the end of the kernel, so neither leaves before the leader has drained.
+        if (rank == 0) {
+          for (uint32_t u = it > (uint32_t)kW2Stages ? it - kW2Stages : 0; u < it; ++u)
+            mbar_wait(&bars->full[u % kW2Stages], (u / kW2Stages) & 1, &bars->never_flag);
+        } else {
+          for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        }
       }
     }
     __syncwarp();
@@ -339,6 +351,10 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_const
       if (dead) {
         if (status) atomicOr(status, kDevTimeout);
         *abort_flag = 1;
+        // MMAs already issued still read shared memory and write TMEM of both blocks: wait (bounded) until they are done
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                     ::"r"(smem_u32(&bars->drain)) : "memory");
+        mbar_wait(&bars->drain, 0, &bars->never_flag);
       }
     }
     __syncwarp();

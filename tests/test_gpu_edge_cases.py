@@ -17,7 +17,8 @@ def torch():
 
 
 def _tol(engine):
-    return 2e-3 if engine == 0 else 2e-5
+    """The stated bars: 2e-3 with bf16 operands on the tensor cores, 1e-5 for the fp32 CUDA-core engine."""
+    return 2e-3 if engine == 0 else 1e-5
 
 
 @pytest.mark.parametrize("engine", ENGINES)
@@ -52,7 +53,7 @@ def test_rank_deficient_anchor_momentum(torch, engine):
     assert np.all(U[:, true_rank:] == 0)
     oe = OracleRun(case, inp, "exact")
     st = oe.states[0]
-    tol = _tol(engine) * 5
+    tol = _tol(engine)
     assert rel(s[:true_rank], st.s[:true_rank]) < tol
     assert so.projector_distance(U[:, :true_rank], st.U[:, :true_rank]) < tol
     assert so.projector_distance(V[:, :true_rank], st.V[:, :true_rank]) < tol

@@ -63,7 +63,9 @@ def test_rejects_bad_arguments(torch):
     assert lib.sc_apply_prf_mask(p + 2, p, 4, 16, 0.5, 0, 0, 0, 0, None) == -4
 
 
-@pytest.mark.parametrize("tokens,features,keep", [(200, 264, 0.1), (64, 4096, 0.05), (33, 37, 0.5), (8, 16, 1.0)])
+# the last four cases sit on rounding ties of K = round(keep * features): halves round up, product in single precision
+@pytest.mark.parametrize("tokens,features,keep", [(200, 264, 0.1), (64, 4096, 0.05), (33, 37, 0.5), (8, 16, 1.0),
+                                                  (9, 8, 0.3125), (9, 10, 0.25), (9, 5, 0.7), (9, 6, 0.75)])
 def test_exact_k_mask_is_bit_exact(torch, tokens, features, keep):
     import paper_2609_14339_b200 as sc
     rng = np.random.default_rng(2)

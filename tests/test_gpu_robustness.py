@@ -77,3 +77,38 @@ def test_state_export_import_continues_bit_identically(torch, engine):
     with pytest.raises(sc.SCError) as e:
         other.state_import(blob)
     assert e.value.status in (-2, -5)
+    # the same shapes in another order (equal totals, equal rank) are refused too: SC_ERR_SHAPE
+    perm = make_plan(Case(**{**case.__dict__, "shapes": [case.shapes[1], case.shapes[0], case.shapes[2]]}), torch)
+    with pytest.raises(sc.SCError) as e:
+        perm.state_import(blob)
+    assert e.value.status == -2
+    # a plan with another tau_p gets its own filter weights from the imported singular values (Eq. 2), not the blob's
+    c2 = make_plan(Case(**{**case.__dict__, "tau_p": 5.0}), torch)
+    c2.state_import(blob)
+    _, s0, _ = c2.export_basis(0)
+    gp = [torch.zeros(sh, dtype=torch.float32, device="cuda:0") for sh in case.shapes]
+    c2.set_debug_gproj_out(gp)
+    W3, m3, v3 = [x.clone() for x in W2], [x.clone() for x in m2], [x.clone() for x in v2]
+    c2.correct_and_step(G, W3, m3, v3, 101)
+    fresh = make_plan(Case(**{**case.__dict__, "tau_p": 5.0}), torch)
+    fresh.anchor_update([A[0], None, A[2]], 7)
+    gq = [torch.zeros(sh, dtype=torch.float32, device="cuda:0") for sh in case.shapes]
+    fresh.set_debug_gproj_out(gq)
+    W4, m4, v4 = [x.clone() for x in W2], [x.clone() for x in m2], [x.clone() for x in v2]
+    fresh.correct_and_step(G, W4, m4, v4, 101)
+    torch.cuda.synchronize()
+    assert all(torch.equal(x, y) for x, y in zip(gp, gq))
+
+
+def test_two_latched_conditions_are_reported_one_after_the_other(torch):
+    case = Case(shapes=[(256, 384)], rank=16, tokens=128)
+    inp = make_inputs(case)
+    plan = make_plan(case, torch)
+    G, A, W, m, v = _tensors(case, inp, torch)
+    plan.anchor_update(A, 0)
+    G[0][3, 5] = float("inf")
+    plan.correct_and_step(G, W, m, v, 100)           # latches the non-finite bit
+    plan.debug_wait_probe(1024)                      # latches the time-out bit as well
+    assert plan.get_device_status() == -9
+    assert plan.get_device_status() == -10
+    assert plan.get_device_status() == 0

@@ -411,3 +411,103 @@ def test_exact_k_mask_keeps_exactly_k_per_token_and_is_unbiased():
     assert np.max(np.abs(big.mean(axis=0) - K / H)) < 5 * np.sqrt(0.1 * 0.9 / 4000)
     assert so.exact_k(4096, 0.05) == 205 and so.exact_k(8, 0.01) == 1 and so.exact_k(8, 1.0) == 8
     assert so.prf_exact_k_mask(1, 0, 0, 5, 8, 1.0).all()
+
+
+def _golden_lines(name):
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", name)
+    return [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+
+
+def test_exact_k_and_keep_threshold_at_ties_hand_computed():
+    """Halves round up and the product is formed in single precision (tests/golden/rounding_ties.txt, by hand)."""
+    n = 0
+    for parts in _golden_lines("rounding_ties.txt"):
+        if parts[0] == "exact_k":
+            assert so.exact_k(int(parts[1]), float(parts[2])) == int(parts[3]), parts
+        else:
+            assert parts[0] == "keep_threshold"
+            assert so.keep_threshold(float(parts[1])) == int(parts[2]), parts
+        n += 1
+    assert n == 12
+    # the single-precision product is what separates 5 * 0.7 from a double-precision evaluation
+    assert int(np.floor(np.float64(np.float32(0.7)) * 5 + 0.5)) == 3 and so.exact_k(5, 0.7) == 4
+    # the mask built from it keeps exactly that many
+    assert np.all(so.prf_exact_k_mask(1, 0, 0, 9, 8, 0.3125).sum(axis=1) == 3)
+
+
+def test_prf_hash_and_masks_match_stored_vectors():
+    """Regression pins written by tests/golden/make_prf_vectors.py (which imports only the oracle)."""
+    lines = _golden_lines("prf_vectors.txt")
+    hashes = [(int(p[1], 16), int(p[2], 16)) for p in lines if p[0] == "lowbias32"]
+    assert len(hashes) == 16
+    got = so.lowbias32(np.array([a for a, _ in hashes], np.uint32))
+    assert [int(x) for x in got] == [b for _, b in hashes]
+    args = dict(seed=0x5EED, layer=3, step=17, tokens=4, features=16)
+    want = np.array([[int(c) for c in p[1]] for p in lines if p[0] == "keep_mask"], float)
+    assert want.shape == (4, 16) and np.array_equal(so.prf_keep_mask(keep=0.5, **args), want)
+    want = np.array([[int(c) for c in p[1]] for p in lines if p[0] == "exact_k_mask"], float)
+    assert want.shape == (4, 16) and np.array_equal(so.prf_exact_k_mask(keep=0.25, **args), want)
+    assert np.all(want.sum(axis=1) == 4)
+
+
+# ----------------------------------------------------------------- dual-EMA step on G_proj
+def test_ademamix_one_element_hand_calc():
+    g = read_golden("ademamix_one_element.txt")
+    W, m1, m2, v = so.ademamix_step(np.array([2.0]), np.array([0.5]), np.array([0.2]), np.array([0.04]),
+                                    np.array([-1.0]), 3, 0.01, 0.9, 0.999, 0.99, 5.0, 1e-8, 0.1)
+    assert abs(m1[0] - g["m1"][0]) < 1e-15 and abs(m2[0] - g["m2"][0]) < 1e-15 and abs(v[0] - g["v"][0]) < 1e-15
+    assert abs(W[0] - g["W"][0]) < 1e-14
+
+
+def test_ademamix_reduces_to_adamw():
+    rng = np.random.default_rng(11)
+    W, m, v, g = (rng.standard_normal((5, 7)) for _ in range(4))
+    v = np.abs(v)
+    m2 = rng.standard_normal((5, 7))
+    # mix_alpha = 0: the slow EMA is carried but unused, everything else is AdamW
+    Wa, ma, va = so.adamw_step(W, m, v, g, 7, 1e-2, 0.9, 0.999, 1e-8, 0.05)
+    Wx, m1x, m2x, vx = so.ademamix_step(W, m, m2, v, g, 7, 1e-2, 0.9, 0.999, 0.9999, 0.0, 1e-8, 0.05)
+    assert np.array_equal(Wa, Wx) and np.array_equal(ma, m1x) and np.array_equal(va, vx)
+    assert np.allclose(m2x, 0.9999 * m2 + (1.0 - 0.9999) * g, rtol=1e-14, atol=0)
+    # beta3 = beta1 from a zero state: m2 == m1 at every step, so the parameter change is AdamW's times
+    # (1 + mix_alpha (1 - beta1^t)), without decay
+    Wm, Wd = W.copy(), W.copy()
+    m1 = m2 = mm = np.zeros_like(W); v1 = v2 = np.zeros_like(W)
+    for t in range(1, 6):
+        gt = rng.standard_normal(W.shape)
+        W_new, m1, m2, v1 = so.ademamix_step(Wm, m1, m2, v1, gt, t, 1e-2, 0.9, 0.999, 0.9, 3.0, 1e-8, 0.0)
+        Wd_new, mm, v2 = so.adamw_step(Wm, mm, v2, gt, t, 1e-2, 0.9, 0.999, 1e-8, 0.0)
+        assert np.allclose(m1, m2, rtol=0, atol=1e-16)
+        assert rel(W_new - Wm, (Wd_new - Wm) * (1.0 + 3.0 * (1.0 - 0.9 ** t))) < 1e-12
+        Wm = W_new
+
+
+def test_ademamix_slow_ema_fixed_point_and_memory():
+    g = np.array([[0.7, -1.3]])
+    m1 = m2 = v = np.zeros_like(g); W = np.zeros_like(g)
+    for t in range(1, 4001):
+        W, m1, m2, v = so.ademamix_step(W, m1, m2, v, g, t, 1e-3, 0.9, 0.999, 0.99, 5.0, 1e-8, 0.0)
+        if t == 10:      # closed form of an EMA of a constant from zero: g (1 - beta^t)
+            assert np.allclose(m2, g * (1 - 0.99 ** 10), rtol=1e-12) and np.allclose(m1, g * (1 - 0.9 ** 10), rtol=1e-12)
+    assert np.allclose(m2, g, rtol=1e-12) and np.allclose(v, g * g * (1 - 0.999 ** 4000), rtol=1e-12)
+    # at the fixed point one step moves theta by lr (1 + mix_alpha) sign(g) (up to eps and the bias correction of v)
+    W2, *_ = so.ademamix_step(W, m1, m2, v, g, 4001, 1e-3, 0.9, 0.999, 0.99, 5.0, 0.0, 0.0)
+    assert np.allclose(W2 - W, -1e-3 * 6.0 * np.sign(g), rtol=1e-6)
+
+
+def test_correct_and_step_ademamix_composes_correction_and_dual_ema():
+    rng = np.random.default_rng(5)
+    m, n, r = 12, 9, 3
+    st = so.new_state(m, n)
+    hp = so.Hyper(tau_p=0.5, max_grad_norm=0.3, beta3=0.99, mix_alpha=2.0, lr=1e-2)
+    so.anchor_update(st, rng.standard_normal((m, n)), hp, r, mode="exact")
+    G = rng.standard_normal((m, n)); W = rng.standard_normal((m, n))
+    z = np.zeros((m, n))
+    Wn, a, b, vn, gp = so.correct_and_step_ademamix([st], [G], [W], [z], [z], [z], 1, hp)
+    # the gradient fed to the optimizer is exactly what the AdamW form of the step feeds (same correction and clip)
+    _, _, _, gp_adam = so.correct_and_step([st], [G], [W], [z], [z], 1, hp)
+    assert np.array_equal(gp[0], gp_adam[0]) and abs(np.linalg.norm(gp[0]) - 0.3) < 1e-12
+    W_ref, a_ref, b_ref, v_ref = so.ademamix_step(W, z, z, z, gp[0], 1, hp.lr, hp.beta1, hp.beta2, hp.beta3, hp.mix_alpha,
+                                                  hp.eps, hp.weight_decay)
+    assert np.array_equal(Wn[0], W_ref) and np.array_equal(b[0], b_ref)

@@ -5,7 +5,8 @@ framework's caching allocator already owns HBM, or the path must not synchronise
 keeps its intermediates in a fixed array inside the library. This test calls it through the C ABI twice in a
 row - a large matrix first, a smaller one second, so the second call runs on top of the first call's leftovers -
 and checks both results against the projection the plan-based entry points compute, within the tolerance the
-other projection tests use for X (5e-4 relative Frobenius: the plan path forms X on tf32 tensor cores).
+other projection tests use for X (5e-4 relative Frobenius: the plan path forms X on tf32 tensor cores), and against
+the fp64 oracle's X = U^T G V on the same device arrays at 1e-5 (this entry point works in plain fp32 FMA).
 
 Collected last on purpose (file name): a run that stops at the first failure has then run everything else.
 """
@@ -14,10 +15,12 @@ import ctypes as C
 import numpy as np
 import pytest
 
+from oracle import spectral_oracle as so
 from parity_util import Case, GpuRun, make_inputs, rel
 
 pytestmark = pytest.mark.gpu
 TOL = 5e-4
+TOL_ORACLE = 1e-5
 
 
 @pytest.fixture(scope="module")
@@ -54,6 +57,9 @@ def test_two_calls_in_a_row_match_the_plan_path(torch):
     torch.cuda.synchronize()
     assert rel(Xb.double().cpu().numpy(), b[3]) < TOL
     assert rel(Xs.double().cpu().numpy(), s[3]) < TOL
+    for X, (G, U, V, _) in ((Xb, b), (Xs, s)):
+        want = so.project(U.double().cpu().numpy(), G.double().cpu().numpy(), V.double().cpu().numpy())
+        assert rel(X.double().cpu().numpy(), want) <= TOL_ORACLE
     # and once more in the opposite order, results unchanged
     Xs2 = sc.project_static(s[0], s[1], s[2])
     Xb2 = sc.project_static(b[0], b[1], b[2])
