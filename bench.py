@@ -40,6 +40,9 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b")
+    ap.add_argument("--optimizer", default="adamw", choices=["adamw", "ademamix"],
+                    help="ademamix: the dual-EMA optimizer on G_proj (one more fp32 state array, 36 B/element); use "
+                         "--workload llama8b_24layers, the full 8B set does not fit in 180 GB with it")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--short", action="store_true", help="with --wgrad: time exactly --steps passes (profiler runs)")
@@ -204,7 +207,8 @@ def run_e2e(args, torch, plan, buf, shapes, n_elems, gsize, world, device):
             for d, h in zip(buf["Ga"], ha):
                 d.copy_(h, non_blocking=True)
             plan.anchor_update(buf["Ga"], base + i)
-        plan.correct_and_step_host(hg, buf["G"], buf["W"], buf["M1"], buf["M2"], 100 + base + i, params_bf16=buf["Wb"])
+        plan.correct_and_step_host(hg, buf["G"], buf["W"], buf["M1"], buf["M2"], 100 + base + i, params_bf16=buf["Wb"],
+                                   exp_avg_slow=buf.get("MS"))
 
     one(0); one(1)
     torch.cuda.synchronize()
@@ -244,15 +248,21 @@ def run_ours(args):
     cfg, shapes, buf = build_workload(args.workload, device, torch)
     n_elems = sum(m * n for m, n in shapes)
     gsize = 2 if cfg["dtype"] == "bf16" else 4
+    mix = args.optimizer == "ademamix"
     hp = sc.Hparams.default(grad_dtype=sc.SC_DTYPE_BF16 if cfg["dtype"] == "bf16" else sc.SC_DTYPE_FP32,
-                            power_iters=1, warm_start=1, warm_power_iters=0, tau_p=1e-3)
+                            power_iters=1, warm_start=1, warm_power_iters=0, tau_p=1e-3,
+                            optimizer=sc.SC_OPT_ADEMAMIX if mix else sc.SC_OPT_ADAMW)
     plan = sc.Plan(shapes, cfg["r"], cfg["keep"], hp, device=device)
     lib = sc.load_library()
+    buf["MS"] = [torch.zeros_like(w) for w in buf["W"]] if mix else None      # slow EMA of the dual-EMA optimizer
+    bytes_steady = BYTES_PER_ELEM_STEADY + (8.0 if mix else 0.0)               # + read and write of the slow EMA
+    bytes_update = BYTES_PER_ELEM_UPDATE + (8.0 if mix else 0.0)
 
     def one_step(i):
         if i % REFRESH_EVERY == 0:
             plan.anchor_update(buf["Ga"], i)
-        plan.correct_and_step(buf["G"], buf["W"], buf["M1"], buf["M2"], 100 + i, params_bf16=buf["Wb"])
+        plan.correct_and_step(buf["G"], buf["W"], buf["M1"], buf["M2"], 100 + i, params_bf16=buf["Wb"],
+                              exp_avg_slow=buf["MS"])
 
     def sync_all():
         torch.cuda.synchronize()
@@ -294,15 +304,15 @@ def run_ours(args):
     update_ms = prof["update"]["ms"] / nprof
 
     peaks = measured_peaks()
-    upd_gbs = n_elems * BYTES_PER_ELEM_UPDATE / (update_ms * 1e-3) / 1e9
+    upd_gbs = n_elems * bytes_update / (update_ms * 1e-3) / 1e9
     upd_launches = max(prof["update"]["spans"] / nprof, 1)          # one launch per shape class and step
     roofline = {"bound": "hbm", "kernel": "fused_update_stream_kernel", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"],
-                "traffic": TRAFFIC_PER_ELEM_UPDATE * n_elems / upd_launches, "peak_source": peaks["source"],
-                "algorithmic_bytes_per_element": BYTES_PER_ELEM_UPDATE,
-                "algorithmic_bytes_per_launch": BYTES_PER_ELEM_UPDATE * n_elems / upd_launches,
+                "traffic": None if mix else TRAFFIC_PER_ELEM_UPDATE * n_elems / upd_launches,
+                "peak_source": peaks["source"], "algorithmic_bytes_per_element": bytes_update,
+                "algorithmic_bytes_per_launch": bytes_update * n_elems / upd_launches,
                 "launches_per_step": upd_launches, "launch_ms": update_ms / upd_launches}
-    step_roofline_ms = max(n_elems * BYTES_PER_ELEM_STEADY / (peaks["hbm_gbs"] * 1e9),
+    step_roofline_ms = max(n_elems * bytes_steady / (peaks["hbm_gbs"] * 1e9),
                            n_elems * 4.0 * cfg["r"] / (peaks["bf16_tflops"] * 1e12)) * 1e3
 
     line = {
@@ -311,7 +321,7 @@ def run_ours(args):
         "dtype": "bf16" if cfg["dtype"] == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": args.workload, "matrices": len(shapes), "elements": n_elems, "rank": cfg["r"],
                    "keep": cfg["keep"], "tokens": cfg["tokens"], "anchor_refresh_every": REFRESH_EVERY,
-                   "power_iters": 1, "range_finder": "cold start q=1 on the first arrival, warm start (previous V) q=0 afterwards",
+                   "optimizer": args.optimizer, "power_iters": 1, "range_finder": "cold start q=1 on the first arrival, warm start (previous V) q=0 afterwards",
                    "parallelism": "replicas x%d" % world,
                    "l2": "inputs (>100 GB resident) far larger than L2; no flush needed"},
         "gpu_launches": int(launches),

@@ -71,6 +71,12 @@ typedef enum sc_dtype { SC_DTYPE_BF16 = 0, SC_DTYPE_FP32 = 1 } sc_dtype;
  * shapes they support (cols % 8 == 0), plain fp32 CUDA-core kernels otherwise (fp32 gradients, odd shapes). */
 typedef enum sc_engine { SC_ENGINE_AUTO = 0, SC_ENGINE_SIMT = 1 } sc_engine;
 
+/* Which optimizer consumes G_proj. ADAMW: Algorithm 1 line 13. ADEMAMIX: the dual-EMA composition of the appendix
+ * "On the Compatibility with Dual-EMA Optimizers": a fast EMA m1 (beta1, bias-corrected) and a slow EMA m2 (beta3, not
+ * bias-corrected) of G_proj, W <- W (1 - lr wd) - lr (m1_hat + mix_alpha m2) / (sqrt(v_hat) + eps); one more fp32 state
+ * array per matrix (sc_opt_state.exp_avg_slow). */
+typedef enum sc_optimizer { SC_OPT_ADAMW = 0, SC_OPT_ADEMAMIX = 1 } sc_optimizer;
+
 typedef struct sc_shape {
   int64_t rows; /* m, out features */
   int64_t cols; /* n, in features  */
@@ -98,8 +104,10 @@ typedef struct sc_hparams {
                               The anchor momentum drifts slowly, so successive arrivals act as accumulated subspace
                               iterations at two sweeps per arrival. 0: always start from the sketch. */
   int32_t warm_power_iters; /* q used on a warm start, 0..16 */
-  int32_t reserved;
+  int32_t optimizer;       /* sc_optimizer */
   uint64_t seed;           /* key of the counter-based Rademacher sketch */
+  float beta3;             /* SC_OPT_ADEMAMIX: decay of the slow EMA, in [0, 1) */
+  float mix_alpha;         /* SC_OPT_ADEMAMIX: weight of the slow EMA in the update, >= 0 */
 } sc_hparams;
 
 /* AdamW state handed to sc_correct_and_step. Arrays of n_mats device pointers, held in host memory. */
@@ -107,6 +115,7 @@ typedef struct sc_opt_state {
   void* const* exp_avg;     /* m: fp32 rows x cols, updated in place */
   void* const* exp_avg_sq;  /* v: fp32 rows x cols, updated in place */
   void* const* params_bf16; /* optional bf16 copy of the updated weights (written only); NULL or NULL entries = none */
+  void* const* exp_avg_slow; /* SC_OPT_ADEMAMIX only: slow EMA m2, fp32 rows x cols, updated in place; NULL for AdamW */
 } sc_opt_state;
 
 /* Per-matrix statistics of the last sc_correct_and_step (by-products of the projection). */
@@ -118,7 +127,8 @@ typedef struct sc_mat_stats {
 } sc_mat_stats;
 
 /* Fill *hp with defaults: alpha 0.3, tau_p 1e-3, beta_anc 0.9, lr 2e-5, betas (0.9, 0.999), eps 1e-8,
- * weight_decay 0, no clipping, grads prescaled, bf16 gradients, l = rank, q = 1, cold starts only, engine AUTO, no stats, seed 0.
+ * weight_decay 0, no clipping, grads prescaled, bf16 gradients, l = rank, q = 1, cold starts only, engine AUTO, no stats, seed 0,
+ * optimizer AdamW, beta3 0.9999, mix_alpha 5 (the values the dual-EMA appendix quotes).
  * (alpha, tau_p, lr, betas: the paper's defaults; the others are not given there.) */
 SC_API sc_status sc_hparams_default(sc_hparams* hp);
 
@@ -160,7 +170,8 @@ SC_API sc_status sc_anchor_update_factored(sc_plan* plan, const void* const* P_f
 /* sc_correct_and_step - one fast-circuit optimizer step over all matrices (Algorithm 1 lines 10-13).
  *   masked_grads   host array of n_mats device pointers (grad_dtype, rows x cols), read only
  *   params         host array of n_mats device pointers, fp32 master weights, updated in place
- *   state          AdamW moments (updated in place) and the optional bf16 weight copy
+ *   state          optimizer moments (updated in place) and the optional bf16 weight copy; with SC_OPT_ADEMAMIX
+ *                  state->exp_avg_slow is required (SC_ERR_INVALID_ARG when it is NULL)
  *   step           optimizer step count t >= 1 (AdamW bias correction; staleness report)
  * Returns SC_WARN_NO_ANCHOR (still a completed step) when no anchor has arrived yet. */
 SC_API sc_status sc_correct_and_step(sc_plan* plan, const void* const* masked_grads, void* const* params,

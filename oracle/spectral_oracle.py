@@ -26,7 +26,10 @@ one-sided Jacobi SVD, rank-1 / diagonal closed forms, Lemma 1 and Lemma 2,
 idempotence at tau_p = 0, the alpha / rank / keep limit cases, torch AdamW in
 fp64, the closed-form global norm, MIRROR == EXACT for rank(M) <= r; the dual-EMA
 step by a one-element hand calculation, its mix_alpha = 0 and beta3 = beta1 special
-cases (both reduce to adamw_step) and the fixed point of the slow EMA.
+cases (both reduce to adamw_step) and the fixed point of the slow EMA; the low-rank
+compressor by exact recovery of rank <= rho inputs, orthogonality of the error to
+the transmitted range, linearity over workers, the telescoping identity of error
+feedback and convergence to the truncated SVD (Eckart-Young) under repetition.
 Parity unpinned: end-to-end MIRROR vs EXACT on inputs with no spectral gap at r
 (the cut is ill-posed there; it is reported, not gated).
 """
@@ -475,3 +478,39 @@ def exact_k(features: int, keep: float) -> int:
     """K = round(keep * H) (halves round up; the product is formed in fp32 as the C ABI does), at least 1, at most H."""
     x = np.float32(keep) * np.float32(features)
     return int(min(features, max(1, int(np.floor(np.float64(x) + 0.5)))))
+
+
+# --------------------------------------------------------------------------
+# Low-rank gradient compressor with error feedback (DP-compression appendix, "Low-rank factorization (F3)":
+# rank-1..4 factors from one subspace-iteration step per gradient, a linear map so that it commutes with the
+# sum over workers, error feedback for what the factors miss).  Plain definition, one matrix:
+#     M = G + E                       gradient plus the error memory
+#     P = M Q_prev                    (sum over workers here)
+#     P_hat = orthonormalise(P)       Gram-Schmidt, column by column
+#     Q = M^T P_hat                   (sum over workers here)
+#     G_hat = P_hat Q^T ;  E <- M - G_hat
+# Q is carried to the next step as the start of its subspace iteration.
+# --------------------------------------------------------------------------
+def gram_schmidt(P, drop_tol: float = 1e-6) -> np.ndarray:
+    """Columns of P orthonormalised in order (modified Gram-Schmidt, fp64).  A column whose remainder is below
+    drop_tol times its original norm lies in the span of the earlier ones and is dropped (left as zeros)."""
+    P = np.array(P, F64)
+    out = np.zeros_like(P)
+    for k in range(P.shape[1]):
+        v = P[:, k].copy()
+        n0 = np.linalg.norm(v)
+        for j in range(k):
+            v -= (out[:, j] @ v) * out[:, j]
+        nv = np.linalg.norm(v)
+        if n0 > 0.0 and nv > drop_tol * n0:
+            out[:, k] = v / nv
+    return out
+
+
+def lowrank_compress(G, E, Q_prev):
+    """One compression step.  Returns (P_hat m x rho, Q n x rho, E_new m x n); the transmitted approximation is
+    P_hat Q^T.  E may be None (no error feedback: the error is returned but nothing was added to G)."""
+    M = np.asarray(G, F64) + (0.0 if E is None else np.asarray(E, F64))
+    P_hat = gram_schmidt(M @ np.asarray(Q_prev, F64))
+    Q = M.T @ P_hat
+    return P_hat, Q, M - P_hat @ Q.T

@@ -16,6 +16,7 @@ SC_OK = 0
 SC_WARN_NO_ANCHOR = 1
 SC_DTYPE_BF16, SC_DTYPE_FP32 = 0, 1
 SC_ENGINE_AUTO, SC_ENGINE_SIMT = 0, 1
+SC_OPT_ADAMW, SC_OPT_ADEMAMIX = 0, 1
 
 
 class SCError(RuntimeError):
@@ -35,7 +36,7 @@ class Hparams(C.Structure):
                 ("max_grad_norm", C.c_float), ("grads_prescaled", C.c_int32), ("grad_dtype", C.c_int32),
                 ("sketch_width", C.c_int32), ("power_iters", C.c_int32), ("engine", C.c_int32),
                 ("collect_stats", C.c_int32), ("warm_start", C.c_int32), ("warm_power_iters", C.c_int32),
-                ("reserved", C.c_int32), ("seed", C.c_uint64)]
+                ("optimizer", C.c_int32), ("seed", C.c_uint64), ("beta3", C.c_float), ("mix_alpha", C.c_float)]
 
     @classmethod
     def default(cls, **kw) -> "Hparams":
@@ -50,7 +51,7 @@ class Hparams(C.Structure):
 
 class OptState(C.Structure):
     _fields_ = [("exp_avg", C.POINTER(C.c_void_p)), ("exp_avg_sq", C.POINTER(C.c_void_p)),
-                ("params_bf16", C.POINTER(C.c_void_p))]
+                ("params_bf16", C.POINTER(C.c_void_p)), ("exp_avg_slow", C.POINTER(C.c_void_p))]
 
 
 class Profile(C.Structure):
@@ -302,16 +303,19 @@ class Plan:
                                                          _ptr_array(Q_factors, self.n_mats, True), int(rho),
                                                          int(step_tag)), "sc_anchor_update_factored")
 
-    def correct_and_step(self, masked_grads, params, exp_avg, exp_avg_sq, step: int, params_bf16=None) -> int:
+    def correct_and_step(self, masked_grads, params, exp_avg, exp_avg_sq, step: int, params_bf16=None,
+                         exp_avg_slow=None) -> int:
+        """exp_avg_slow: the slow EMA of the dual-EMA optimizer (required when hp.optimizer is SC_OPT_ADEMAMIX)."""
         n = self.n_mats
         st = OptState(_ptr_array(exp_avg, n, False), _ptr_array(exp_avg_sq, n, False),
-                      _ptr_array(params_bf16, n, True) if params_bf16 is not None else None)
+                      _ptr_array(params_bf16, n, True) if params_bf16 is not None else None,
+                      _ptr_array(exp_avg_slow, n, False) if exp_avg_slow is not None else None)
         return _check(self.lib.sc_correct_and_step(self.handle, _ptr_array(masked_grads, n, False),
                                                    _ptr_array(params, n, False), C.byref(st), int(step)),
                       "sc_correct_and_step", allow=(SC_OK, SC_WARN_NO_ANCHOR))
 
     def correct_and_step_host(self, host_grads, grad_staging, params, exp_avg, exp_avg_sq, step: int, params_bf16=None,
-                              want_stats: bool = True):
+                              want_stats: bool = True, exp_avg_slow=None):
         """Gradients in host tensors (pin them for overlap); returns (status, stats or None, clip)."""
         n = self.n_mats
         harr = (C.c_void_p * n)()
@@ -320,7 +324,8 @@ class Plan:
                 raise ValueError("host gradient %d must be a contiguous CPU tensor" % i)
             harr[i] = t.data_ptr()
         st = OptState(_ptr_array(exp_avg, n, False), _ptr_array(exp_avg_sq, n, False),
-                      _ptr_array(params_bf16, n, True) if params_bf16 is not None else None)
+                      _ptr_array(params_bf16, n, True) if params_bf16 is not None else None,
+                      _ptr_array(exp_avg_slow, n, False) if exp_avg_slow is not None else None)
         stats = (MatStats * n)() if want_stats else None
         clip = C.c_float(1.0)
         rc = _check(self.lib.sc_correct_and_step_host(self.handle, harr, _ptr_array(grad_staging, n, False),

@@ -74,6 +74,7 @@ struct MatDev {
   float* m1;          // AdamW first moment
   float* m2;          // AdamW second moment
   bf16* Wb;           // optional bf16 weight copy
+  float* ms;          // slow EMA of the dual-EMA optimizer (null for AdamW)
   float* gproj_dbg;   // optional G_proj output
   int m, n;
   int inst;           // index of this matrix inside its shape class (selects its tensor maps)
@@ -103,6 +104,10 @@ struct StepScalars {       // scalars of one step, passed by value to kernels
   float inv_sqrt_bc2;      // 1 / sqrt(1 - beta2^t)
   float eps;
   float decay;             // 1 - lr * weight_decay
+  // dual-EMA optimizer only (mix != 0): W <- W decay - (step_size m1 + lr_mix m_slow) / den
+  float beta3, one_m_beta3;
+  float lr_mix;            // lr * mix_alpha (the slow EMA is not bias-corrected)
+  int mix;
 };
 
 }  // namespace sc
@@ -200,7 +205,7 @@ size_t tc_tmaps_bytes(int count);
 sc_status tc_init();   // resolves the driver entry point for tensor-map encoding
 sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_call_part);
 sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count);   // T = G V
-sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc);
+sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int count, const StepScalars& sc);   // AdamW or dual EMA (sc.mix)
 sc_status tc_launch_wait_probe(sc_plan* p, int max_polls);
 sc_status tc_encode_anchor(sc_plan* p, ShapeClass& c, const std::vector<int>& ids);
 sc_status tc_launch_ema_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, int b_field_off);

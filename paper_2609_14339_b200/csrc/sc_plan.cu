@@ -55,6 +55,10 @@ bool valid_hparams(const sc_hparams* hp) {
   if (!(hp->beta_anc >= 0.f && hp->beta_anc < 1.f)) return false;
   if (!(hp->beta1 >= 0.f && hp->beta1 < 1.f) || !(hp->beta2 >= 0.f && hp->beta2 < 1.f)) return false;
   if (!(hp->eps >= 0.f) || !isfinite(hp->lr) || !(hp->weight_decay >= 0.f)) return false;
+  if (hp->optimizer != SC_OPT_ADAMW && hp->optimizer != SC_OPT_ADEMAMIX) return false;
+  if (hp->optimizer == SC_OPT_ADEMAMIX &&
+      (!(hp->beta3 >= 0.f && hp->beta3 < 1.f) || !(hp->mix_alpha >= 0.f) || !isfinite(hp->mix_alpha)))
+    return false;
   return true;
 }
 
@@ -331,6 +335,7 @@ sc_status sc_hparams_default(sc_hparams* hp) {
   hp->max_grad_norm = 0.f; hp->grads_prescaled = 1; hp->grad_dtype = SC_DTYPE_BF16;
   hp->sketch_width = 0; hp->power_iters = 1; hp->engine = SC_ENGINE_AUTO; hp->collect_stats = 0; hp->seed = 0;
   hp->warm_start = 0; hp->warm_power_iters = 0;
+  hp->optimizer = SC_OPT_ADAMW; hp->beta3 = 0.9999f; hp->mix_alpha = 5.f;
   return SC_OK;
 }
 
@@ -586,6 +591,9 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
   if (state->params_bf16 &&
       (st = check_ptr_array(reinterpret_cast<const void* const*>(state->params_bf16), p->n_mats, true)) != SC_OK)
     return st;
+  const bool mix = p->hp.optimizer == SC_OPT_ADEMAMIX;
+  if (mix && (st = check_ptr_array(reinterpret_cast<const void* const*>(state->exp_avg_slow), p->n_mats, false)) != SC_OK)
+    return st;
   cudaStream_t s = p->stream;
   const sc_hparams& hp = p->hp;
   const int rp = p->rp;
@@ -599,8 +607,9 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
     md.m1 = static_cast<float*>(state->exp_avg[i]);
     md.m2 = static_cast<float*>(state->exp_avg_sq[i]);
     md.Wb = state->params_bf16 ? static_cast<bf16*>(state->params_bf16[i]) : nullptr;
+    md.ms = mix ? static_cast<float*>(state->exp_avg_slow[i]) : nullptr;
     g_changed = g_changed || before.G != md.G || before.W != md.W || before.m1 != md.m1 || before.m2 != md.m2 ||
-                before.Wb != md.Wb;
+                before.Wb != md.Wb || before.ms != md.ms;
     md.gproj_dbg = static_cast<float*>(p->dbg_out[i]);
   }
   if ((st = upload_table(p)) != SC_OK) return st;
@@ -617,6 +626,9 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
   sc.inv_sqrt_bc2 = (float)(1.0 / sqrt(bc2));
   sc.eps = hp.eps;
   sc.decay = 1.f - hp.lr * hp.weight_decay;
+  sc.mix = mix ? 1 : 0;
+  sc.beta3 = hp.beta3; sc.one_m_beta3 = 1.f - hp.beta3;
+  sc.lr_mix = hp.lr * hp.mix_alpha;
   const bool clip_on = hp.max_grad_norm > 0.f;
   const bool want_norm = clip_on || hp.collect_stats;
 

@@ -124,7 +124,14 @@ __global__ void __launch_bounds__(256) gemm_kernel(GemmArgs a, EpiAdamW epi) {
         const float mo = fmaf(s.beta1, md.m1[o], s.one_m_beta1 * g);
         const float vo = fmaf(s.beta2, md.m2[o], s.one_m_beta2 * g * g);
         const float den = fmaf(sqrtf(vo), s.inv_sqrt_bc2, s.eps);
-        const float w = fmaf(-s.step_size, mo / den, md.W[o] * s.decay);
+        float w;
+        if (s.mix) {     // dual EMA: the slow average of G_proj joins the numerator, not bias-corrected
+          const float mslow = fmaf(s.beta3, md.ms[o], s.one_m_beta3 * g);
+          md.ms[o] = mslow;
+          w = md.W[o] * s.decay - fmaf(s.lr_mix, mslow, s.step_size * mo) / den;
+        } else {
+          w = fmaf(-s.step_size, mo / den, md.W[o] * s.decay);
+        }
         md.m1[o] = mo;
         md.m2[o] = vo;
         md.W[o] = w;

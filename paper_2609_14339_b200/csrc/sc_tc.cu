@@ -16,12 +16,13 @@
 
 namespace sc {
 
-constexpr int kMapsPerMat = 26;
-constexpr int kPerCallMaps = 6;   // the first six are rebuilt whenever the caller's buffers move
+constexpr int kMapsPerMat = 27;
+constexpr int kPerCallMaps = 7;   // the first seven are rebuilt whenever the caller's buffers move
 enum { MAP_G = 0,    // masked gradient, bf16, box 64 x 128 (MMA A operand of the projection)
        MAP_G32,      // masked gradient, bf16, box 32 x 128, 64-byte swizzle (streaming tile of the fused update)
        MAP_W, MAP_M1, MAP_M2,   // fp32 weights and AdamW moments, box 32 x 128, 128-byte swizzle (load and store)
        MAP_WB,       // bf16 weight copy, box 32 x 128, 64-byte swizzle (store only)
+       MAP_MS,       // slow EMA of the dual-EMA optimizer, fp32, same box as MAP_M1 (a copy of MAP_M1 when unused)
        MAP_VTHI, MAP_VTLO, MAP_UHI, MAP_ULO, MAP_CTHI, MAP_CTLO,
        MAP_CT64HI, MAP_CT64LO,   // C^T with a 64 x 64 box (N = 64 tiles of the streaming update)
        MAP_M_K,      // anchor momentum as a K-major A operand: box 32 floats x 128 rows
@@ -473,6 +474,24 @@ __device__ __forceinline__ void adamw4(const StepScalars& s, float clip, const f
   }
 }
 
+// The same four elements under the dual-EMA optimizer: the slow average ms of G_proj (decay beta3, no bias correction)
+// joins the bias-corrected fast average in the numerator.
+__device__ __forceinline__ void ademamix4(const StepScalars& s, float clip, const float g_raw[4], const float4& r,
+                                          float4& w, float4& m1, float4& m2, float4& ms, float4& gp) {
+  const float rr[4] = {r.x, r.y, r.z, r.w};
+  float* W = &w.x; float* M1 = &m1.x; float* M2 = &m2.x; float* MS = &ms.x; float* GP = &gp.x;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float g = clip * fmaf(s.alpha_s, g_raw[j], rr[j]);
+    const float mo = fmaf(s.beta1, M1[j], s.one_m_beta1 * g);
+    const float so = fmaf(s.beta3, MS[j], s.one_m_beta3 * g);
+    const float vo = fmaf(s.beta2, M2[j], s.one_m_beta2 * g * g);
+    const float den = fmaf(sqrt_nobranch(vo), s.inv_sqrt_bc2, s.eps);
+    W[j] = W[j] * s.decay - div_nobranch(fmaf(s.lr_mix, so, s.step_size * mo), den);
+    M1[j] = mo; M2[j] = vo; MS[j] = so; GP[j] = g;
+  }
+}
+
 // =====================================================================================================
 // Fused correction + AdamW, streaming form: no thread touches global memory for the state.
 //   Persistent blocks (one per SM) draw work items (matrix, 128-row panel, one 64-column tile) from a counter.
@@ -482,16 +501,26 @@ __device__ __forceinline__ void adamw4(const StepScalars& s, float clip, const f
 //   warps 2-9  consumers, one thread per (row, half unit): R from TMEM, W/m/v/G from swizzled shared memory,
 //            blend + AdamW, results written back in place; one elected thread sends the unit out with TMA stores
 //            and hands the stage back once those stores have read it.
+// MIX = true is the dual-EMA optimizer: a fourth fp32 array (the slow average) travels with every unit, so a stage
+// is 72 KB and only two fit beside the operands. With two stages a stage has to go back to the producer as soon as
+// its stores have read it, so a warp of its own (warp 10) issues the stores and waits for them, instead of a
+// consumer thread that would stall its warp.
 // =====================================================================================================
 constexpr int kUnitW = 32;                                   // columns per streaming unit
 constexpr int kTileN = 64;                                   // columns per MMA tile (2 units)
 constexpr int kUnitF32 = 128 * kUnitW * 4;                   // 16 KB: one fp32 array of a unit
 constexpr int kUnitBf16 = 128 * kUnitW * 2;                  // 8 KB
-constexpr int kStreamStageBytes = 3 * kUnitF32 + kUnitBf16;  // 56 KB
-constexpr int kStreamStages = 3;
+constexpr int kStreamStages = 3;                             // most stages any variant uses (sizes the barrier arrays)
 constexpr int kOpndU = 2 * kTileBytes;                       // U hi + lo, 128 rows x 64 bf16 each
 constexpr int kOpndC = 2 * (kTileN * 128);                   // C^T hi + lo, 64 rows x 64 bf16 each
-constexpr int kStreamSmem = kStreamStages * kStreamStageBytes + kOpndU + kOpndC;
+template <bool MIX>
+struct StreamCfg {
+  static constexpr int kF32 = MIX ? 4 : 3;                              // fp32 arrays per unit: W, m, v (, slow m)
+  static constexpr int kStages = MIX ? 2 : 3;
+  static constexpr int kStageBytes = kF32 * kUnitF32 + kUnitBf16;      // 56 KB / 72 KB
+  static constexpr int kSmem = kStages * kStageBytes + kOpndU + kOpndC;
+  static constexpr int kThreads = MIX ? 352 : 320;
+};
 
 // Work items are handed out by an atomic counter: blocks do not run at the same speed (the slowest of a static split
 // finished 7% after the median), so each block's producer draws the next item when it needs one and passes the index
@@ -504,6 +533,7 @@ struct StreamBars {
   uint64_t opnd_full, opnd_empty;
   uint64_t acc_full[2], acc_empty[2];
   uint64_t item_ready[kItemSlots];
+  uint64_t store_ready[kStreamStages];   // MIX only: the consumers have finished a unit, the store warp may send it
   int item_slot[kItemSlots];
   uint32_t tmem_slot;
   int abort_flag;
@@ -524,20 +554,25 @@ __device__ __forceinline__ void decode_item(const StreamGeom& g, int item, int& 
   ct1 = min(g.col_tiles, ct0 + g.tiles_per_chunk);
 }
 
-__global__ void __launch_bounds__(320, 1)
+template <bool MIX>
+__global__ void __launch_bounds__(StreamCfg<MIX>::kThreads, 1)
 fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx,
                            const CUtensorMap* __restrict__ maps, StreamGeom g, StepScalars sc,
                            const float* __restrict__ clip_ptr, unsigned* status, unsigned* work_counter) {
+  constexpr int kStages = StreamCfg<MIX>::kStages, kStreamStageBytes = StreamCfg<MIX>::kStageBytes;
+  constexpr int kStreamSmem = StreamCfg<MIX>::kSmem, kF32 = StreamCfg<MIX>::kF32;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* opnd = smem + kStreamStages * kStreamStageBytes;
+  uint8_t* opnd = smem + kStages * kStreamStageBytes;
   StreamBars* bars = reinterpret_cast<StreamBars*>(smem + kStreamSmem);
   volatile int* abort_flag = &bars->abort_flag;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nch = (g.rp + 63) >> 6;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStreamStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+    for (int s = 0; s < kStreamStages; ++s) {
+      mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); mbar_init(&bars->store_ready[s], 1);
+    }
     mbar_init(&bars->opnd_full, 1);
     mbar_init(&bars->opnd_empty, 1);
     for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 8); }
@@ -577,6 +612,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
           tensormap_acquire(mp + MAP_CT64HI); tensormap_acquire(mp + MAP_CT64LO);
           tensormap_acquire(mp + MAP_W); tensormap_acquire(mp + MAP_M1); tensormap_acquire(mp + MAP_M2);
           tensormap_acquire(mp + MAP_G32);
+          if (MIX) tensormap_acquire(mp + MAP_MS);
           last_inst = inst;
           last_panel = -1;
         }
@@ -597,15 +633,16 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
           last_panel = rt;
           const int units = (g.n - ct * kTileN > kUnitW) ? 2 : 1;
           for (int u = 0; u < units; ++u, ++unit_it) {
-            const int s = unit_it % kStreamStages;
-            if (!mbar_wait(&bars->empty[s], ((unit_it / kStreamStages) & 1) ^ 1, abort_flag)) { dead = true; break; }
+            const int s = unit_it % kStages;
+            if (!mbar_wait(&bars->empty[s], ((unit_it / kStages) & 1) ^ 1, abort_flag)) { dead = true; break; }
             uint8_t* st = smem + (size_t)s * kStreamStageBytes;
             const int x = ct * kTileN + u * kUnitW;
             mbar_expect_tx(&bars->full[s], kStreamStageBytes);
             tma_load_2d(st, mp + MAP_W, &bars->full[s], x, row0);
             tma_load_2d(st + kUnitF32, mp + MAP_M1, &bars->full[s], x, row0);
             tma_load_2d(st + 2 * kUnitF32, mp + MAP_M2, &bars->full[s], x, row0);
-            tma_load_2d(st + 3 * kUnitF32, mp + MAP_G32, &bars->full[s], x, row0);
+            if (MIX) tma_load_2d(st + 3 * kUnitF32, mp + MAP_MS, &bars->full[s], x, row0);
+            tma_load_2d(st + kF32 * kUnitF32, mp + MAP_G32, &bars->full[s], x, row0);
           }
         }
       }
@@ -614,8 +651,8 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
         *abort_flag = 1;
         // let the copies already in flight land before this block's shared memory goes away (bounded waits)
         volatile int never = 0;
-        for (uint32_t u = unit_it > kStreamStages ? unit_it - kStreamStages : 0; u < unit_it; ++u)
-          mbar_wait(&bars->full[u % kStreamStages], (u / kStreamStages) & 1, &never);
+        for (uint32_t u = unit_it > (uint32_t)kStages ? unit_it - kStages : 0; u < unit_it; ++u)
+          mbar_wait(&bars->full[u % kStages], (u / kStages) & 1, &never);
         if (op_it > 0) mbar_wait(&bars->opnd_full, (op_it - 1) & 1, &never);
       }
     }
@@ -658,7 +695,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
       if (dead) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
     }
     __syncwarp();
-  } else {
+  } else if (warp >= 2 && warp < 10) {
     // -------------------------------------------------------------------- consumers
     const int q = warp & 3, h = (warp - 2) >> 2;
     const int r = q * 32 + lane;                 // row inside the 128-row panel
@@ -675,7 +712,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
       decode_item(g, item, inst, rt, ct0, ct1);
       const MatDev& md = tab[idx[inst]];
       const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
-      if (leader && inst != last_inst) {
+      if (!MIX && leader && inst != last_inst) {
         tensormap_acquire(mp + MAP_W); tensormap_acquire(mp + MAP_M1); tensormap_acquire(mp + MAP_M2);
         tensormap_acquire(mp + MAP_WB);
       }
@@ -689,8 +726,8 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
         tc_fence_after();
         const int units = (g.n - ct * kTileN > kUnitW) ? 2 : 1;
         for (int u = 0; u < units; ++u, ++unit_it) {
-          const int s = unit_it % kStreamStages;
-          if (!mbar_wait(&bars->full[s], (unit_it / kStreamStages) & 1, abort_flag)) { dead = true; break; }
+          const int s = unit_it % kStages;
+          if (!mbar_wait(&bars->full[s], (unit_it / kStages) & 1, abort_flag)) { dead = true; break; }
           uint8_t* st = smem + (size_t)s * kStreamStageBytes;
           float rv[16];
           tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + ab * kTileN + u * kUnitW + h * 16, rv);
@@ -698,11 +735,12 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
           float4* Ws = reinterpret_cast<float4*>(st);
           float4* M1s = reinterpret_cast<float4*>(st + kUnitF32);
           float4* M2s = reinterpret_cast<float4*>(st + 2 * kUnitF32);
-          uint4* Gs = reinterpret_cast<uint4*>(st + 3 * kUnitF32);
+          float4* MSs = reinterpret_cast<float4*>(st + 3 * kUnitF32);   // MIX only
+          uint4* Gs = reinterpret_cast<uint4*>(st + kF32 * kUnitF32);
           // all of this thread's 16 elements are read first, so that the 16 AdamW chains are independent work for
           // the scheduler; results go back in place afterwards
           int fidx[4], gidx[2];
-          float4 w[4], m1[4], m2[4], gp[4];
+          float4 w[4], m1[4], m2[4], ms[4], gp[4];
           uint4 graw[2];
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
@@ -713,6 +751,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
           for (int i = 0; i < 4; ++i) {
             fidx[i] = r * 8 + ((4 * h + i) ^ (r & 7));
             w[i] = Ws[fidx[i]]; m1[i] = M1s[fidx[i]]; m2[i] = M2s[fidx[i]];
+            if (MIX) ms[i] = MSs[fidx[i]];
           }
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -722,12 +761,14 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
             const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162*>(&hi);
             const float g4[4] = {__low2float(g01), __high2float(g01), __low2float(g23), __high2float(g23)};
             const float4 rr = make_float4(rv[4 * i], rv[4 * i + 1], rv[4 * i + 2], rv[4 * i + 3]);
-            adamw4(sc, clip, g4, rr, w[i], m1[i], m2[i], gp[i]);
+            if (MIX) ademamix4(sc, clip, g4, rr, w[i], m1[i], m2[i], ms[i], gp[i]);
+            else adamw4(sc, clip, g4, rr, w[i], m1[i], m2[i], gp[i]);
           }
           float gout[16];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             Ws[fidx[i]] = w[i]; M1s[fidx[i]] = m1[i]; M2s[fidx[i]] = m2[i];
+            if (MIX) MSs[fidx[i]] = ms[i];
             gout[4 * i] = gp[i].x; gout[4 * i + 1] = gp[i].y; gout[4 * i + 2] = gp[i].z; gout[4 * i + 3] = gp[i].w;
           }
 #pragma unroll
@@ -747,7 +788,9 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
           }
           fence_proxy_async();
           consumer_barrier();
-          if (leader) {
+          if (MIX) {
+            if (leader) mbar_arrive(&bars->store_ready[s]);       // the store warp sends the unit and frees the stage
+          } else if (leader) {
             tma_store_2d(mp + MAP_W, st, x, row0);
             tma_store_2d(mp + MAP_M1, st + kUnitF32, x, row0);
             tma_store_2d(mp + MAP_M2, st + 2 * kUnitF32, x, row0);
@@ -755,7 +798,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
             tma_store_commit();
             // hand the previous unit's stage back once its stores have finished reading shared memory
             tma_store_wait_read<1>();
-            if (unit_it > 0) mbar_arrive(&bars->empty[(unit_it - 1) % kStreamStages]);
+            if (unit_it > 0) mbar_arrive(&bars->empty[(unit_it - 1) % kStages]);
           }
         }
         if (dead) break;
@@ -765,7 +808,50 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
       }
     }
     if (dead && lane == 0) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
-    if (leader) tma_store_wait_all();
+    if (!MIX && leader) tma_store_wait_all();
+  } else if (MIX) {
+    // -------------------------------------------------------------------- store warp (dual-EMA variant only)
+    if (lane == 0) {
+      uint32_t unit_it = 0;
+      int last_inst = -1;
+      bool dead = false;
+      for (uint32_t item_it = 0; !dead; ++item_it) {
+        if (!mbar_wait(&bars->item_ready[item_it % kItemSlots], (item_it / kItemSlots) & 1, abort_flag)) { dead = true; break; }
+        const int item = *reinterpret_cast<volatile int*>(&bars->item_slot[item_it % kItemSlots]);
+        if (item < 0) break;
+        int inst, rt, ct0, ct1;
+        decode_item(g, item, inst, rt, ct0, ct1);
+        const MatDev& md = tab[idx[inst]];
+        const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
+        if (inst != last_inst) {
+          tensormap_acquire(mp + MAP_W); tensormap_acquire(mp + MAP_M1); tensormap_acquire(mp + MAP_M2);
+          tensormap_acquire(mp + MAP_MS); tensormap_acquire(mp + MAP_WB);
+          last_inst = inst;
+        }
+        const int row0 = rt * 128;
+        const bool has_wb = md.Wb != nullptr;
+        for (int ct = ct0; ct < ct1 && !dead; ++ct) {
+          const int units = (g.n - ct * kTileN > kUnitW) ? 2 : 1;
+          for (int u = 0; u < units; ++u, ++unit_it) {
+            const int s = unit_it % kStages;
+            if (!mbar_wait(&bars->store_ready[s], (unit_it / kStages) & 1, abort_flag)) { dead = true; break; }
+            uint8_t* st = smem + (size_t)s * kStreamStageBytes;
+            const int x = ct * kTileN + u * kUnitW;
+            tma_store_2d(mp + MAP_W, st, x, row0);
+            tma_store_2d(mp + MAP_M1, st + kUnitF32, x, row0);
+            tma_store_2d(mp + MAP_M2, st + 2 * kUnitF32, x, row0);
+            tma_store_2d(mp + MAP_MS, st + 3 * kUnitF32, x, row0);
+            if (has_wb) tma_store_2d(mp + MAP_WB, st + kF32 * kUnitF32, x, row0);
+            tma_store_commit();
+            tma_store_wait_read<0>();          // the stage is free as soon as the stores have read it
+            mbar_arrive(&bars->empty[s]);
+          }
+        }
+      }
+      if (dead) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
+      tma_store_wait_all();
+    }
+    __syncwarp();
   }
   tc_fence_before();
   __syncthreads();
@@ -808,8 +894,10 @@ sc_status tc_init() {
   }
   // per device: the opt-in shared-memory sizes (cheap, so simply repeated for every plan)
   if (cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
-      cudaFuncSetAttribute(fused_update_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           kStreamSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(fused_update_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           StreamCfg<false>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(fused_update_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           StreamCfg<true>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
       cudaFuncSetAttribute(ema_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
@@ -861,6 +949,7 @@ sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_
       ok = ok && encode2d(mp + MAP_M2, f32, 4, md.m2, c.n, c.m, c.n, 32, 128, CU_TENSOR_MAP_SWIZZLE_128B);
       ok = ok && encode2d(mp + MAP_WB, b16, 2, md.Wb ? (const void*)md.Wb : md.G, c.n, c.m, c.n, 32, 128,
                           CU_TENSOR_MAP_SWIZZLE_64B);
+      ok = ok && encode2d(mp + MAP_MS, f32, 4, md.ms ? md.ms : md.m1, c.n, c.m, c.n, 32, 128, CU_TENSOR_MAP_SWIZZLE_128B);
       if (!ok) return SC_ERR_CUDA;
     }
     if (static_part) {
@@ -1064,10 +1153,17 @@ sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int coun
   g.csplit = (g.col_tiles + g.tiles_per_chunk - 1) / g.tiles_per_chunk;
   g.n_items = count * g.row_tiles * g.csplit;
   const int grid = g.n_items < n_sm ? g.n_items : n_sm;
-  const size_t smem = kStreamSmem + sizeof(StreamBars) + 1024;
   if (cudaMemsetAsync(p->work_dev, 0, sizeof(unsigned), p->stream) != cudaSuccess) return SC_ERR_CUDA;
-  fused_update_stream_kernel<<<grid, 320, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps),
-                                                             g, sc, p->clip_dev, p->status_dev, p->work_dev);
+  const CUtensorMap* maps = static_cast<const CUtensorMap*>(c.tmaps);
+  if (sc.mix) {
+    const size_t smem = StreamCfg<true>::kSmem + sizeof(StreamBars) + 1024;
+    fused_update_stream_kernel<true><<<grid, StreamCfg<true>::kThreads, smem, p->stream>>>(
+        p->dev_tab, idx, maps, g, sc, p->clip_dev, p->status_dev, p->work_dev);
+  } else {
+    const size_t smem = StreamCfg<false>::kSmem + sizeof(StreamBars) + 1024;
+    fused_update_stream_kernel<false><<<grid, StreamCfg<false>::kThreads, smem, p->stream>>>(
+        p->dev_tab, idx, maps, g, sc, p->clip_dev, p->status_dev, p->work_dev);
+  }
   ++g_kernel_launches;
   return cuda_ok(cudaGetLastError());
 }

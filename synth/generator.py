@@ -166,6 +166,8 @@ CONFIGS = {
     "llama8b": dict(layers=32, shapes=llama_layer_shapes(4096, 14336, 1024), tokens=4096, keep=0.1, k=32, r=64, dtype="bf16"),
     "ffn_sweep": dict(layers=1, shapes=[(14336, 4096)], tokens=4096, keep=0.1, k=32, r=64, dtype="bf16"),
     "llama70b_slice": dict(layers=8, shapes=llama_layer_shapes(8192, 28672, 1024), tokens=8192, keep=0.05, k=64, r=128, dtype="bf16"),
+    # 24 of the 32 8B-shaped layers: the largest slice whose state still fits in 180 GB with a fourth fp32 array per weight
+    "llama8b_24layers": dict(layers=24, shapes=llama_layer_shapes(4096, 14336, 1024), tokens=4096, keep=0.1, k=32, r=64, dtype="bf16"),
     # two 8B-shaped layers: small enough (6 GB resident) for multi-pass profiler captures of the short kernels
     "llama8b_2layers": dict(layers=2, shapes=llama_layer_shapes(4096, 14336, 1024), tokens=4096, keep=0.1, k=32, r=64, dtype="bf16"),
 }

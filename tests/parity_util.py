@@ -41,6 +41,9 @@ class Case:
     n_anchor: int = 1              # anchor arrivals before the step
     warm: bool = False             # warm-started range finder from the second arrival on
     q_warm: int = 0
+    optimizer: int = 0             # 0 AdamW, 1 dual EMA (AdEMAMix) on G_proj
+    beta3: float = 0.99
+    mix_alpha: float = 5.0
     extra: dict = field(default_factory=dict)
 
 
@@ -52,12 +55,14 @@ def specs(case: Case):
 def make_inputs(case: Case):
     """Stored arrays (exact bits both sides see) for anchors, masked gradient and optimizer state."""
     sp = specs(case)
-    out = dict(specs=sp, anchors=[], G=[], W=[], m=[], v=[])
+    out = dict(specs=sp, anchors=[], G=[], W=[], m=[], v=[], ms=[])
     for s in sp:
         out["anchors"].append([gen.round_to(gen.anchor_gradient(s, a), case.dtype) for a in range(case.n_anchor)])
         out["G"].append(gen.round_to(gen.masked_gradient(s, case.n_anchor + 1, rescale=case.prescaled), case.dtype))
         W, m, v = gen.optimizer_state(s, warmed=case.warmed)
         out["W"].append(W); out["m"].append(m); out["v"].append(v)
+        # slow EMA of the dual-EMA optimizer: a seeded array of its own (a shifted, rescaled copy of the fast moment)
+        out["ms"].append(np.ascontiguousarray(np.roll(m, 1, axis=1) * np.float32(0.5)))
     return out
 
 
@@ -67,7 +72,8 @@ def oracle_hyper(case: Case) -> so.Hyper:
     f = lambda x: float(np.float32(x))
     return so.Hyper(alpha=f(case.alpha), tau_p=f(case.tau_p), beta_anc=f(case.beta_anc), lr=f(case.lr), eps=f(case.eps),
                     weight_decay=f(case.weight_decay), max_grad_norm=f(case.max_grad_norm),
-                    beta1=f(0.9), beta2=f(0.999), grads_prescaled=case.prescaled, keep=f(case.keep))
+                    beta1=f(0.9), beta2=f(0.999), grads_prescaled=case.prescaled, keep=f(case.keep),
+                    beta3=f(case.beta3), mix_alpha=f(case.mix_alpha))
 
 
 def to_dev(arr, dtype: str, torch, device):
@@ -84,6 +90,7 @@ def make_plan(case: Case, torch, device="cuda:0"):
                             grad_dtype=sc.SC_DTYPE_BF16 if case.dtype == "bf16" else sc.SC_DTYPE_FP32,
                             sketch_width=case.l, power_iters=case.q, engine=case.engine, collect_stats=1,
                             warm_start=int(case.warm), warm_power_iters=case.q_warm,
+                            optimizer=case.optimizer, beta3=case.beta3, mix_alpha=case.mix_alpha,
                             seed=case.seed)
     return sc.Plan(case.shapes, case.rank, case.keep, hp, device=device)
 
@@ -111,17 +118,19 @@ class GpuRun:
         W = [torch.from_numpy(inputs["W"][i].copy()).to(device) for i in range(n)]
         m = [torch.from_numpy(inputs["m"][i].copy()).to(device) for i in range(n)]
         v = [torch.from_numpy(inputs["v"][i].copy()).to(device) for i in range(n)]
+        ms = [torch.from_numpy(inputs["ms"][i].copy()).to(device) for i in range(n)] if case.optimizer == 1 else None
         Wb = [torch.zeros(s, dtype=torch.bfloat16, device=device) for s in case.shapes]
         gp = [torch.zeros(s, dtype=torch.float32, device=device) for s in case.shapes]
         self.plan.set_debug_gproj_out(gp)
         t = case.t0 if case.warmed else 1
-        self.step_status = self.plan.correct_and_step(G, W, m, v, t, params_bf16=Wb)
+        self.step_status = self.plan.correct_and_step(G, W, m, v, t, params_bf16=Wb, exp_avg_slow=ms)
         torch.cuda.synchronize()
         self.dev_status = self.plan.get_device_status()
         self.stats, self.clip = self.plan.get_stats()
         self.W = [x.double().cpu().numpy() for x in W]
         self.m = [x.double().cpu().numpy() for x in m]
         self.v = [x.double().cpu().numpy() for x in v]
+        self.ms = [x.double().cpu().numpy() for x in ms] if ms is not None else None
         self.Wb = [x.float().double().cpu().numpy() for x in Wb]
         self.gproj = [x.double().cpu().numpy() for x in gp]
         self.uses_tc = self.plan.uses_tensor_cores()
@@ -153,9 +162,13 @@ class OracleRun:
         G = [gen.stored_to_f64(inputs["G"][i], case.dtype) for i in range(n)]
         t = case.t0 if case.warmed else 1
         self.W0 = [np.asarray(w, np.float64) for w in inputs["W"]]
-        self.W, self.m, self.v, self.gproj = so.correct_and_step(
-            self.states, G, self.W0, [np.asarray(x, np.float64) for x in inputs["m"]],
-            [np.asarray(x, np.float64) for x in inputs["v"]], t, hp)
+        f64 = lambda key: [np.asarray(x, np.float64) for x in inputs[key]]
+        if case.optimizer == 1:
+            self.W, self.m, self.ms, self.v, self.gproj = so.correct_and_step_ademamix(
+                self.states, G, self.W0, f64("m"), f64("ms"), f64("v"), t, hp)
+        else:
+            self.ms = None
+            self.W, self.m, self.v, self.gproj = so.correct_and_step(self.states, G, self.W0, f64("m"), f64("v"), t, hp)
         self.G = G
         self.hp = hp
 
@@ -167,6 +180,8 @@ def compare_step(g: GpuRun, o: OracleRun, mask_small_g=False):
         errs["gproj"] = max(errs["gproj"], rel(g.gproj[i], o.gproj[i]))
         errs["m"] = max(errs["m"], rel(g.m[i], o.m[i]))
         errs["v"] = max(errs["v"], rel(g.v[i], o.v[i]))
+        if o.ms is not None:
+            errs["ms"] = max(errs.get("ms", 0.0), rel(g.ms[i], o.ms[i]))
         dWg = g.W[i] - o.W0[i]
         dWo = o.W[i] - o.W0[i]
         if mask_small_g:

@@ -511,3 +511,61 @@ def test_correct_and_step_ademamix_composes_correction_and_dual_ema():
     W_ref, a_ref, b_ref, v_ref = so.ademamix_step(W, z, z, z, gp[0], 1, hp.lr, hp.beta1, hp.beta2, hp.beta3, hp.mix_alpha,
                                                   hp.eps, hp.weight_decay)
     assert np.array_equal(Wn[0], W_ref) and np.array_equal(b[0], b_ref)
+
+
+# ----------------------------------------------------------------- low-rank compressor with error feedback
+def test_gram_schmidt_against_library_qr_and_on_dependent_columns():
+    rng = np.random.default_rng(21)
+    P = rng.standard_normal((40, 4))
+    Qn, Rn = np.linalg.qr(P)
+    assert rel(so.gram_schmidt(P), Qn * np.sign(np.diag(Rn))) < 1e-12        # QR with a positive diagonal is unique
+    P[:, 2] = 2.0 * P[:, 0] - P[:, 1]                                         # third column in the span of the first two
+    Ph = so.gram_schmidt(P)
+    assert np.all(Ph[:, 2] == 0) and abs(np.linalg.norm(Ph[:, 3]) - 1) < 1e-12
+    G = Ph.T @ Ph
+    assert np.allclose(G, np.diag([1, 1, 0, 1]), atol=1e-12)
+
+
+def test_lowrank_compress_is_exact_on_low_rank_input_and_orthogonal_otherwise():
+    rng = np.random.default_rng(22)
+    m, n, rho = 30, 24, 3
+    M = rng.standard_normal((m, rho)) @ rng.standard_normal((rho, n))         # rank 3
+    Q0 = rng.standard_normal((n, rho))
+    Ph, Q, E = so.lowrank_compress(M, None, Q0)
+    assert rel(Ph @ Q.T, M) < 1e-12 and np.linalg.norm(E) < 1e-12 * np.linalg.norm(M)
+    G = rng.standard_normal((m, n)); E0 = 0.1 * rng.standard_normal((m, n))
+    Ph, Q, E = so.lowrank_compress(G, E0, Q0)
+    assert np.allclose(Ph.T @ Ph, np.eye(rho), atol=1e-12)
+    assert rel(Ph @ Q.T, Ph @ (Ph.T @ (G + E0))) < 1e-12                      # orthogonal projection of M onto range(P_hat)
+    assert np.linalg.norm(Ph.T @ E) < 1e-12 * np.linalg.norm(E)               # what is left is orthogonal to what was sent
+    assert abs(np.linalg.norm(G + E0) ** 2 - np.linalg.norm(Ph @ Q.T) ** 2 - np.linalg.norm(E) ** 2) < 1e-9
+
+
+def test_lowrank_compress_commutes_with_the_sum_over_workers():
+    rng = np.random.default_rng(23)
+    m, n, rho = 20, 16, 2
+    Gs = [rng.standard_normal((m, n)) for _ in range(3)]
+    Q0 = rng.standard_normal((n, rho))
+    Ph, Q, _ = so.lowrank_compress(sum(Gs), None, Q0)
+    P_sum = sum(G @ Q0 for G in Gs)                                            # each worker's P, summed
+    Ph2 = so.gram_schmidt(P_sum)
+    Q_sum = sum(G.T @ Ph2 for G in Gs)                                         # each worker's Q, summed
+    assert rel(Ph2, Ph) < 1e-12 and rel(Q_sum, Q) < 1e-12
+
+
+def test_lowrank_error_feedback_telescopes_and_repetition_reaches_the_truncated_svd():
+    rng = np.random.default_rng(24)
+    m, n, rho = 25, 18, 2
+    E = np.zeros((m, n)); Q = rng.standard_normal((n, rho))
+    sent, given = np.zeros((m, n)), np.zeros((m, n))
+    for t in range(6):
+        G = rng.standard_normal((m, n))
+        Ph, Q, E = so.lowrank_compress(G, E, Q)
+        sent += Ph @ Q.T; given += G
+    assert rel(sent + E, given) < 1e-12                                        # nothing is lost, only delayed
+    M = rng.standard_normal((m, n)) * np.logspace(0, -2, n)[None, :]
+    Q = rng.standard_normal((n, rho))
+    for _ in range(200):                                                       # same matrix again and again, no feedback
+        Ph, Q, Err = so.lowrank_compress(M, None, Q)
+    s = np.linalg.svd(M, compute_uv=False)
+    assert abs(np.linalg.norm(Err) - np.sqrt(np.sum(s[rho:] ** 2))) < 1e-8 * np.linalg.norm(M)
