@@ -48,6 +48,8 @@ def parse_args():
     ap.add_argument("--short", action="store_true", help="with --wgrad: time exactly --steps passes (profiler runs)")
     ap.add_argument("--wgrad", action="store_true",
                     help="time the masked weight gradients of one 8B-shaped layer (mask pass + tensor-core GEMM)")
+    ap.add_argument("--lowrank", action="store_true",
+                    help="time the rank-4 gradient compressor with error feedback on the seven matrices of one 8B-shaped layer")
     ap.add_argument("--sweep", action="store_true",
                     help="config 4: one 14336x4096 matrix, rank x keep grid; prints one JSON line with a 'cells' list")
     return ap.parse_args()
@@ -488,8 +490,67 @@ def run_wgrad(args):
         "clocks": clocks}), flush=True)
 
 
+def run_lowrank(args):
+    """The low-rank compressor with error feedback (DP-compression appendix, F3) on the seven gradient matrices of one
+    8B-shaped layer, rank 4: three passes over each matrix, 22 algorithmic bytes per element (G 2, E read 4 + M written
+    4, M read 4, M read 4 + E written 4). HBM-bound; the roofline is the measured copy bandwidth."""
+    import torch
+    import paper_2609_14339_b200 as sc
+    from paper_2609_14339_b200 import build as _build
+    from synth import generator as gen
+    _build.build()
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    peaks = measured_peaks()
+    rho = 4
+    shapes = gen.CONFIGS["llama8b"]["shapes"]
+    g = torch.Generator(device=device); g.manual_seed(11)
+    G = [(torch.randn((m, n), generator=g, device=device)).to(torch.bfloat16) for m, n in shapes]
+    E = [torch.zeros((m, n), device=device) for m, n in shapes]
+    Q = [sc.lowrank_init_q(n, rho, seed=i) for i, (m, n) in enumerate(shapes)]
+    P = [torch.empty((m, rho), device=device) for m, n in shapes]
+    ws = [None] * len(shapes)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)      # larger than L2
+
+    def layer_pass():
+        for i in range(len(shapes)):
+            _, _, ws[i] = sc.lowrank_compress(G[i], Q[i], E=E[i], P=P[i], workspace=ws[i])
+
+    for _ in range(max(args.warmup, 3)):
+        layer_pass()
+    lib = sc.load_library()
+    launches0 = lib.sc_kernel_launch_count()
+    sampler = ClockSampler(0)
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    times = []
+    steps = max(args.steps, 50)
+    for _ in range(steps):
+        flush.zero_()
+        e[0].record(); layer_pass(); e[1].record(); torch.cuda.synchronize()
+        times.append(e[0].elapsed_time(e[1]))
+    launches = lib.sc_kernel_launch_count() - launches0
+    clocks = sampler.stop()
+    ms = statistics.median(times)
+    elems = sum(m * n for m, n in shapes)
+    gbs = elems * 22.0 / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "low-rank gradient compressor with error feedback, one 8B-shaped layer (7 matrices), rank 4: gradient GB/s",
+        "value": elems * 2 / (ms * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": 1, "steps": steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": {"workload": "lowrank_llama8b_layer", "rho": rho, "elements": elems,
+                                        "l2": "256 MB buffer rewritten between timed iterations"},
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "kernel": "lowrank_mq_kernel + lowrank_mtp_kernel + lowrank_residual_kernel",
+                     "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                     "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes_per_element": 22.0},
+        "clocks": clocks}), flush=True)
+
+
 def main():
     args = parse_args()
+    if args.lowrank:
+        run_lowrank(args)
+        return
     if args.wgrad:
         run_wgrad(args)
         return

@@ -222,6 +222,36 @@ SC_API sc_status sc_apply_prf_mask_exact_k(const void* X_dev, void* out_dev, int
                                            float keep, uint64_t seed, uint32_t layer, uint64_t step, int rescale,
                                            void* stream);
 
+/* sc_lowrank_compress - low-rank compression of one gradient matrix with error feedback (DP-compression appendix,
+ * "Low-rank factorization (F3)": rank-1..4 factors from one subspace-iteration step per gradient; the map is linear, so
+ * it commutes with the sum over data-parallel workers; error feedback keeps what the factors miss for the next step):
+ *     M = G + E      P = M Q_prev      P_hat = orth(P)      Q = M^T P_hat      E <- M - P_hat Q^T
+ * The transmitted approximation is P_hat Q^T; (P_hat, Q) is exactly the factored form sc_anchor_update_factored takes.
+ * Stand-alone (no plan), asynchronous on `stream`.
+ *   G_dev      device: rows x cols, grad_dtype (sc_dtype), row-major, read only
+ *   E_dev      device: rows x cols fp32 error memory, updated in place (start it at zero), or NULL for no error feedback.
+ *              Between phase A and phase C it holds M.
+ *   P_dev      device: rows x rho fp32 row-major. Out of phase A: P = M Q_prev; out of phase B: P_hat (orthonormal
+ *              columns; a column that depends on the earlier ones to single precision - remainder below 1e-3 of its
+ *              norm - is dropped, i.e. zero).
+ *   Q_dev      device: cols x rho fp32 row-major. In: Q_prev (sc_lowrank_init_q for the first step, afterwards the Q of
+ *              the previous step); out of phase B: Q = M^T P_hat.
+ *   rho        1..8
+ *   phases     bit mask: 1 = A (M, P), 2 = B (orthonormalise P, Q), 4 = C (E). 7 runs everything (one worker). With
+ *              several workers: call with 1, sum P over workers, call with 2, sum Q over workers, call with 4.
+ *   workspace  device: caller-owned scratch of sc_lowrank_workspace_bytes(rows, cols, rho) bytes, 256-byte aligned
+ * Pointers 16-byte aligned; cols % 4 == 0 (SC_ERR_SHAPE otherwise). All arithmetic is fp32 on the CUDA cores (at most
+ * 16 flops per byte: HBM-bound), every reduction two-stage in a fixed order.
+ * Errors: INVALID_ARG, DTYPE, SHAPE, TOO_LARGE, ALIGNMENT, WORKSPACE, CUDA. */
+SC_API size_t sc_lowrank_workspace_bytes(int64_t rows, int64_t cols, int rho);
+SC_API sc_status sc_lowrank_compress(const void* G_dev, int grad_dtype, void* E_dev, void* P_dev, void* Q_dev,
+                                     int64_t rows, int64_t cols, int rho, int phases, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+
+/* Fill Q (cols x rho fp32) with the counter-based +-1 sketch keyed on `seed`: the start of the first compression step
+ * (the same start on every worker, nothing transmitted). */
+SC_API sc_status sc_lowrank_init_q(void* Q_dev, int64_t cols, int rho, uint64_t seed, void* stream);
+
 /* ---- inspection / test hooks ------------------------------------------------------------------------- */
 
 /* Copy matrix `mat`'s cached basis into caller device buffers (any may be NULL):

@@ -491,9 +491,10 @@ def exact_k(features: int, keep: float) -> int:
 #     G_hat = P_hat Q^T ;  E <- M - G_hat
 # Q is carried to the next step as the start of its subspace iteration.
 # --------------------------------------------------------------------------
-def gram_schmidt(P, drop_tol: float = 1e-6) -> np.ndarray:
+def gram_schmidt(P, drop_tol: float = 1e-3) -> np.ndarray:
     """Columns of P orthonormalised in order (modified Gram-Schmidt, fp64).  A column whose remainder is below
-    drop_tol times its original norm lies in the span of the earlier ones and is dropped (left as zeros)."""
+    drop_tol times its original norm lies in the span of the earlier ones and is dropped (left as zeros); the
+    default is the level at which a single-precision implementation can still tell the remainder from rounding."""
     P = np.array(P, F64)
     out = np.zeros_like(P)
     for k in range(P.shape[1]):

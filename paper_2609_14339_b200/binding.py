@@ -84,6 +84,10 @@ EXPORTS = {
                                         C.c_uint64, C.c_uint32, C.c_uint64, _VP, _VP]),
     "sc_apply_prf_mask_exact_k": (C.c_int, [_VP, _VP, C.c_int64, C.c_int64, C.c_float, C.c_uint64, C.c_uint32, C.c_uint64,
                                             C.c_int, _VP]),
+    "sc_lowrank_workspace_bytes": (C.c_size_t, [C.c_int64, C.c_int64, C.c_int]),
+    "sc_lowrank_compress": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP, C.c_int64, C.c_int64, C.c_int, C.c_int, _VP, C.c_size_t,
+                                      _VP]),
+    "sc_lowrank_init_q": (C.c_int, [_VP, C.c_int64, C.c_int, C.c_uint64, _VP]),
     "sc_export_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
     "sc_import_basis": (C.c_int, [_VP, C.c_int, _VP, _VP, _VP]),
     "sc_export_projection": (C.c_int, [_VP, C.c_int, _VP, _VP]),
@@ -184,6 +188,46 @@ def project_static(G, U, V, X_out=None, stream=None):
         _check(lib.sc_project_static(G.data_ptr(), dt, U.data_ptr(), V.data_ptr(), rows, cols, r, X_out.data_ptr(),
                                      st.cuda_stream), "sc_project_static")
     return X_out
+
+
+def lowrank_init_q(cols: int, rho: int, seed: int, device="cuda:0", stream=None):
+    """The +-1 start basis of the first compression step (cols x rho fp32)."""
+    import torch
+    lib = load_library()
+    Q = torch.empty((cols, rho), dtype=torch.float32, device=device)
+    st = stream if stream is not None else torch.cuda.current_stream(Q.device)
+    with torch.cuda.device(Q.device):
+        _check(lib.sc_lowrank_init_q(Q.data_ptr(), cols, rho, int(seed), st.cuda_stream), "sc_lowrank_init_q")
+    return Q
+
+
+def lowrank_compress(G, Q, E=None, P=None, phases: int = 7, workspace=None, stream=None):
+    """One low-rank compression step with error feedback through sc_lowrank_compress.
+
+    G: rows x cols bf16/fp32; Q: cols x rho fp32 (in: previous Q, out: new Q); E: rows x cols fp32 error memory
+    (updated in place) or None; P: rows x rho fp32 (allocated when None). Returns (P, Q, workspace)."""
+    import torch
+    lib = load_library()
+    rows, cols = G.shape
+    rho = Q.shape[1]
+    assert Q.shape == (cols, rho) and Q.dtype == torch.float32 and Q.is_contiguous() and G.is_contiguous()
+    if P is None:
+        P = torch.empty((rows, rho), dtype=torch.float32, device=G.device)
+    assert P.shape == (rows, rho) and P.dtype == torch.float32 and P.is_contiguous()
+    if E is not None:
+        assert E.shape == (rows, cols) and E.dtype == torch.float32 and E.is_contiguous()
+    need = lib.sc_lowrank_workspace_bytes(rows, cols, rho)
+    if need == 0:
+        raise SCError(-1, "sc_lowrank_workspace_bytes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=G.device)
+    dt = SC_DTYPE_BF16 if G.dtype == torch.bfloat16 else SC_DTYPE_FP32
+    st = stream if stream is not None else torch.cuda.current_stream(G.device)
+    with torch.cuda.device(G.device):
+        _check(lib.sc_lowrank_compress(G.data_ptr(), dt, E.data_ptr() if E is not None else None, P.data_ptr(),
+                                       Q.data_ptr(), rows, cols, rho, int(phases), workspace.data_ptr(),
+                                       workspace.numel(), st.cuda_stream), "sc_lowrank_compress")
+    return P, Q, workspace
 
 
 def masked_weight_grad(dY, X, keep: float, seed: int, layer: int, step: int, out_dtype=None, Xm=None, out=None,

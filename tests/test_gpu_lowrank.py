@@ -1,0 +1,157 @@
+"""Low-rank gradient compressor with error feedback (DP-compression appendix, "Low-rank factorization (F3)") on the
+GPU against the fp64 oracle: the orthonormal factor P_hat (unique: triangular factor with a positive diagonal), the
+second factor Q, and the error memory E, element by element.  All arithmetic on the GPU is fp32 (bf16 only as the
+storage type of G), so 1e-5 is asserted for fp32 gradients and for bf16 gradients alike (the stated bar for bf16
+operands is 2e-3)."""
+import numpy as np
+import pytest
+
+from oracle import spectral_oracle as so
+from parity_util import rel
+from synth import generator as gen
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch
+    return torch
+
+
+def _grad(m, n, dtype, seed, planted=3):
+    spec = gen.GradSpec(m=m, n=n, tokens=96, keep=0.5, planted_rank=planted, snr=1.0, seed=seed)
+    return gen.round_to(gen.masked_gradient(spec, 1), dtype)
+
+
+def _dev(torch, arr, dtype):
+    from parity_util import to_dev
+    return to_dev(arr, dtype, torch, "cuda:0")
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("m,n,rho", [(200, 136, 1), (330, 520, 4), (64, 2052, 2), (129, 1028, 8)])
+def test_three_steps_with_error_feedback_match_the_oracle(torch, dtype, m, n, rho):
+    import paper_2609_14339_b200 as sc
+    Q = sc.lowrank_init_q(n, rho, seed=9)
+    assert np.array_equal(Q.cpu().numpy(), so.rademacher_sketch(9, 0, n, rho))
+    Qo = Q.double().cpu().numpy()
+    E = torch.zeros((m, n), dtype=torch.float32, device="cuda:0")
+    Eo = np.zeros((m, n))
+    ws = None
+    for step in range(3):
+        Gs = _grad(m, n, dtype, seed=10 + step)
+        P, Q, ws = sc.lowrank_compress(_dev(torch, Gs, dtype), Q, E=E, workspace=ws)
+        Po, Qo, Eo = so.lowrank_compress(gen.stored_to_f64(Gs, dtype), Eo, Qo)
+        torch.cuda.synchronize()
+        Pg = P.double().cpu().numpy()
+        assert np.abs(Pg.T @ Pg - np.eye(rho)).max() < 1e-5
+        e = dict(P=rel(Pg, Po), Q=rel(Q.double().cpu().numpy(), Qo), E=rel(E.double().cpu().numpy(), Eo))
+        assert max(e.values()) < TOL, (step, e)
+
+
+def test_phases_called_one_by_one_and_two_workers(torch):
+    import paper_2609_14339_b200 as sc
+    m, n, rho = 264, 392, 3
+    G1, G2 = _grad(m, n, "bf16", 31), _grad(m, n, "bf16", 32)
+    Q0 = sc.lowrank_init_q(n, rho, seed=4)
+    # one call with all phases ...
+    Ea = torch.zeros((m, n), dtype=torch.float32, device="cuda:0")
+    Pa, Qa, _ = sc.lowrank_compress(_dev(torch, G1, "bf16"), Q0.clone(), E=Ea)
+    # ... equals three calls, bit for bit
+    Eb = torch.zeros_like(Ea); Qb = Q0.clone()
+    Pb, _, ws = sc.lowrank_compress(_dev(torch, G1, "bf16"), Qb, E=Eb, phases=1)
+    sc.lowrank_compress(_dev(torch, G1, "bf16"), Qb, E=Eb, P=Pb, phases=2, workspace=ws)
+    sc.lowrank_compress(_dev(torch, G1, "bf16"), Qb, E=Eb, P=Pb, phases=4, workspace=ws)
+    torch.cuda.synchronize()
+    assert torch.equal(Pa, Pb) and torch.equal(Qa, Qb) and torch.equal(Ea, Eb)
+    # two workers: P and Q are summed between the phases; the result is the compression of the summed gradient
+    dev = [_dev(torch, G, "bf16") for G in (G1, G2)]
+    Qw = [Q0.clone(), Q0.clone()]
+    Pw = [sc.lowrank_compress(dev[w], Qw[w], phases=1)[0] for w in range(2)]
+    Psum = Pw[0] + Pw[1]
+    Ph = [Psum.clone(), Psum.clone()]
+    for w in range(2):
+        sc.lowrank_compress(dev[w], Qw[w], P=Ph[w], phases=2)
+    Qsum = Qw[0] + Qw[1]
+    torch.cuda.synchronize()
+    Po, Qo, _ = so.lowrank_compress(gen.stored_to_f64(G1, "bf16") + gen.stored_to_f64(G2, "bf16"), None,
+                                    Q0.double().cpu().numpy())
+    assert rel(Ph[0].double().cpu().numpy(), Po) < TOL and rel(Qsum.double().cpu().numpy(), Qo) < TOL
+
+
+def test_degenerate_inputs(torch):
+    import paper_2609_14339_b200 as sc
+    m, n, rho = 72, 136, 2
+    # zero gradient, zero memory: every column is dropped, nothing non-finite
+    Q = sc.lowrank_init_q(n, rho, seed=1)
+    E = torch.zeros((m, n), dtype=torch.float32, device="cuda:0")
+    P, Q, _ = sc.lowrank_compress(torch.zeros((m, n), dtype=torch.float32, device="cuda:0"), Q, E=E)
+    torch.cuda.synchronize()
+    assert float(P.abs().max()) == 0 and float(Q.abs().max()) == 0 and float(E.abs().max()) == 0
+    # a rank-1 gradient with rho = 2: the second direction is dropped, the first reproduces the gradient exactly
+    rng = np.random.default_rng(3)
+    G = np.outer(rng.integers(-3, 4, m), rng.integers(-3, 4, n)).astype(np.float32)
+    Q = sc.lowrank_init_q(n, rho, seed=2)
+    E = torch.zeros((m, n), dtype=torch.float32, device="cuda:0")
+    P, Q, _ = sc.lowrank_compress(torch.from_numpy(G).cuda(), Q, E=E)
+    torch.cuda.synchronize()
+    Po, Qo, Eo = so.lowrank_compress(G, np.zeros((m, n)), so.rademacher_sketch(2, 0, n, rho))
+    assert np.all(Po[:, 1] == 0) and float(P[:, 1].abs().max()) == 0
+    assert rel(P.double().cpu().numpy(), Po) < TOL and rel(Q.double().cpu().numpy(), Qo) < TOL
+    assert float(E.abs().max()) < 1e-4 * np.abs(G).max()
+
+
+def test_factors_feed_the_factored_anchor_update(torch):
+    """The anchor gradient pushed as rank-rho factors: compress, then sc_anchor_update_factored(P_hat, Q)."""
+    import paper_2609_14339_b200 as sc
+    m, n, rho = 256, 384, 4
+    Ga = _grad(m, n, "bf16", 41, planted=4)
+    Q = sc.lowrank_init_q(n, rho, seed=6)
+    for _ in range(2):                                     # two subspace-iteration steps on the same matrix
+        P, Q, _ = sc.lowrank_compress(_dev(torch, Ga, "bf16"), Q)
+    plan = sc.Plan([(m, n)], 4, 0.5, sc.Hparams.default(beta_anc=0.5))
+    plan.anchor_update_factored([P], [Q], 0)
+    torch.cuda.synchronize()
+    Qo = so.rademacher_sketch(6, 0, n, rho)
+    for _ in range(2):
+        Po, Qo, _ = so.lowrank_compress(gen.stored_to_f64(Ga, "bf16"), None, Qo)
+    want = so.anchor_ema(np.zeros((m, n)), Po @ Qo.T, float(np.float32(0.5)))
+    assert rel(plan.export_anchor_momentum(0).double().cpu().numpy(), want) < 1e-5
+
+
+def test_full_size_ffn_matrix(torch):
+    """One 14336 x 4096 bf16 gradient, rank 4, with a non-zero error memory: the launch configuration of bench.py --lowrank."""
+    import paper_2609_14339_b200 as sc
+    m, n, rho = 14336, 4096, 4
+    dev = torch.device("cuda", 0)
+    spec = gen.GradSpec(m=m, n=n, tokens=4096, keep=0.1, planted_rank=32, snr=1.0, seed=0)
+    G = gen.torch_gradients(spec, 1, dev, torch.bfloat16)
+    gg = torch.Generator(device=dev); gg.manual_seed(5)
+    E = torch.randn((m, n), generator=gg, device=dev) * 50.0
+    Q = sc.lowrank_init_q(n, rho, seed=3)
+    Go, Eo, Qo = G.double().cpu().numpy(), E.double().cpu().numpy(), Q.double().cpu().numpy()
+    P, Q, _ = sc.lowrank_compress(G, Q, E=E)
+    torch.cuda.synchronize()
+    Po, Qo, Eo = so.lowrank_compress(Go, Eo, Qo)
+    e = dict(P=rel(P.double().cpu().numpy(), Po), Q=rel(Q.double().cpu().numpy(), Qo), E=rel(E.double().cpu().numpy(), Eo))
+    print("low-rank full-size errors", e)
+    assert max(e.values()) < TOL, e
+
+
+def test_rejects_bad_arguments(torch):
+    import paper_2609_14339_b200 as sc
+    lib = sc.load_library()
+    x = torch.zeros(4096, device="cuda:0")
+    p = x.data_ptr()
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda:0")
+    w = ws.data_ptr()
+    assert lib.sc_lowrank_workspace_bytes(128, 128, 9) == 0
+    assert lib.sc_lowrank_compress(p, 1, None, p, p, 32, 32, 9, 7, w, ws.numel(), None) == -1      # rho > 8
+    assert lib.sc_lowrank_compress(p, 1, None, p, p, 32, 30, 2, 7, w, ws.numel(), None) == -2      # cols % 4
+    assert lib.sc_lowrank_compress(p, 3, None, p, p, 32, 32, 2, 7, w, ws.numel(), None) == -3
+    assert lib.sc_lowrank_compress(p + 4, 1, None, p, p, 32, 32, 2, 7, w, ws.numel(), None) == -4
+    assert lib.sc_lowrank_compress(p, 1, None, p, p, 32, 32, 2, 7, w, 16, None) == -5
+    assert lib.sc_lowrank_compress(p, 1, None, p, p, 32, 32, 2, 0, w, ws.numel(), None) == -1
+    torch.cuda.synchronize()
