@@ -108,6 +108,16 @@ typedef struct sc_hparams {
   uint64_t seed;           /* key of the counter-based Rademacher sketch */
   float beta3;             /* SC_OPT_ADEMAMIX: decay of the slow EMA, in [0, 1) */
   float mix_alpha;         /* SC_OPT_ADEMAMIX: weight of the slow EMA in the update, >= 0 */
+  int32_t full_spectrum;   /* 1: the main-text form of Section 3.2 - no rank cut, the soft weights d_i = s_i / (s_i + tau_p)
+                              apply to all min(rows, cols) singular directions: G_filt = P_U G P_V with
+                              P_U = U diag(d) U^T, P_V = V diag(d) V^T. Create the plan with rank = 0. On anchor arrival
+                              the two soft projectors are built by matrix products only (Newton-Schulz square root of the
+                              Gram matrix, then Newton-Schulz inverse), in fp64; every step is two dense tensor-core
+                              contractions per matrix plus one elementwise AdamW pass. Needs tau_p > 0, bf16 gradients,
+                              AdamW, no clipping, rows and cols multiples of 8 in [256, 8192]. */
+  int32_t fs_sqrt_iters;   /* full_spectrum: iterations of the square-root stage, 1..200 (default 30) */
+  int32_t fs_inv_iters;    /* full_spectrum: iterations of the inverse stage, 1..200 (default 14) */
+  int32_t reserved;
 } sc_hparams;
 
 /* AdamW state handed to sc_correct_and_step. Arrays of n_mats device pointers, held in host memory. */

@@ -29,7 +29,9 @@ step by a one-element hand calculation, its mix_alpha = 0 and beta3 = beta1 spec
 cases (both reduce to adamw_step) and the fixed point of the slow EMA; the low-rank
 compressor by exact recovery of rank <= rho inputs, orthogonality of the error to
 the transmitted range, linearity over workers, the telescoping identity of error
-feedback and convergence to the truncated SVD (Eckart-Young) under repetition.
+feedback and convergence to the truncated SVD (Eckart-Young) under repetition;
+the full-spectrum filter by its equality with the rank-min(m,n) basis form, closed
+forms on diagonal input, and the product-only iteration by convergence to it.
 Parity unpinned: end-to-end MIRROR vs EXACT on inputs with no spectral gap at r
 (the cut is ill-posed there; it is reported, not gated).
 """
@@ -478,6 +480,78 @@ def exact_k(features: int, keep: float) -> int:
     """K = round(keep * H) (halves round up; the product is formed in fp32 as the C ABI does), at least 1, at most H."""
     x = np.float32(keep) * np.float32(features)
     return int(min(features, max(1, int(np.floor(np.float64(x) + 0.5)))))
+
+
+# --------------------------------------------------------------------------
+# Full-spectrum soft filter: the main-text form of Section 3.2 ("Filtering d_i = s_i / (s_i + tau_p)"), where the
+# soft weights apply to ALL singular directions of the anchor momentum and there is no rank cut.  With
+# M = U S V^T (thin, all min(m, n) directions):
+#     P_U = U diag(d) U^T = A (A + tau I)^-1,  A = (M M^T)^(1/2)        (m x m)
+#     P_V = V diag(d) V^T = B (B + tau I)^-1,  B = (M^T M)^(1/2)        (n x n)
+#     G_filt = P_U G P_V
+# which is filtered_gradient() with r = min(m, n), written without an explicit basis.
+# --------------------------------------------------------------------------
+def full_spectrum_projectors(M, tau_p: float):
+    """(P_U, P_V) by the plain definition: full thin SVD, Eq. 2 on every singular value."""
+    U, s, V = svd_exact(M)
+    d = filter_weights(s, tau_p)
+    return (U * d) @ U.T, (V * d) @ V.T
+
+
+def full_spectrum_filtered(M, G, tau_p: float):
+    """G_filt = P_U G P_V."""
+    PU, PV = full_spectrum_projectors(M, tau_p)
+    return PU @ np.asarray(G, F64) @ PV
+
+
+def soft_projector_iterative(A, tau_p: float, n_sqrt: int, n_inv: int):
+    """f(A) = A^(1/2) (A^(1/2) + tau I)^-1 for a symmetric positive semi-definite A (a Gram matrix of the anchor
+    momentum) by products only - the iteration the GPU path runs, restated in fp64 step by step:
+
+      square root (coupled Newton-Schulz):  Y_0 = A / c, Z_0 = I, c = ||A||_F (an upper bound of the largest eigenvalue)
+                                            T = (3 I - Z Y) / 2 ;  Y <- Y T ;  Z <- T Z          (n_sqrt times)
+                                            S = sqrt(c) Y   ->  A^(1/2)
+      inverse (Newton-Schulz):              B = S + tau I, X_0 = I / (||S||_F + tau)
+                                            X <- X (2 I - B X)                                   (n_inv times)
+      result                                I - tau X       ->  S (S + tau I)^-1
+
+    An eigenvalue lam of A moves as p <- p (3 - p)^2 / 4 from p_0 = lam / c, y = sqrt(lam p / c): directions far
+    below the threshold converge last and are UNDER-estimated until then (y < sqrt(lam / c)), which only pushes their
+    filter weight further towards 0.  On the null space of A the companion iterate Z grows by 3/2 per
+    iteration and drags rounding noise with it, so n_sqrt is a few dozen, not hundreds (fp64: the result is
+    good to 1e-9 at 40 iterations on a singular Gram matrix and breaks down past about 70).  tau_p must be
+    positive (for tau_p = 0 the operator is a projector and B is singular)."""
+    A = np.asarray(A, F64)
+    k = A.shape[0]
+    I = np.eye(k)
+    c = np.linalg.norm(A)
+    if c == 0.0:
+        return np.zeros_like(A)
+    Y, Z = A / c, I.copy()
+    for _ in range(int(n_sqrt)):
+        T = 1.5 * I - 0.5 * (Z @ Y)
+        Y, Z = Y @ T, T @ Z
+    S = np.sqrt(c) * Y
+    B = S + tau_p * I
+    X = I / (np.linalg.norm(S) + tau_p)
+    for _ in range(int(n_inv)):
+        X = X @ (2.0 * I - B @ X)
+    return I - tau_p * X
+
+
+def full_spectrum_filtered_iterative(M, G, tau_p: float, n_sqrt: int, n_inv: int):
+    """G_filt with both soft projectors from soft_projector_iterative (mirror of the GPU path)."""
+    M = np.asarray(M, F64)
+    PU = soft_projector_iterative(M @ M.T, tau_p, n_sqrt, n_inv)
+    PV = soft_projector_iterative(M.T @ M, tau_p, n_sqrt, n_inv)
+    return PU @ np.asarray(G, F64) @ PV
+
+
+def correct_full_spectrum(M_anc, G_mask, hp: Hyper):
+    """G_proj (Eq. 3) with the full-spectrum filter, before clipping."""
+    scale = 1.0 if hp.grads_prescaled else 1.0 / hp.keep
+    g = scale * np.asarray(G_mask, F64)
+    return blend(g, full_spectrum_filtered(M_anc, g, hp.tau_p), hp.alpha)
 
 
 # --------------------------------------------------------------------------

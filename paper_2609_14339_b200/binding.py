@@ -36,7 +36,9 @@ class Hparams(C.Structure):
                 ("max_grad_norm", C.c_float), ("grads_prescaled", C.c_int32), ("grad_dtype", C.c_int32),
                 ("sketch_width", C.c_int32), ("power_iters", C.c_int32), ("engine", C.c_int32),
                 ("collect_stats", C.c_int32), ("warm_start", C.c_int32), ("warm_power_iters", C.c_int32),
-                ("optimizer", C.c_int32), ("seed", C.c_uint64), ("beta3", C.c_float), ("mix_alpha", C.c_float)]
+                ("optimizer", C.c_int32), ("seed", C.c_uint64), ("beta3", C.c_float), ("mix_alpha", C.c_float),
+                ("full_spectrum", C.c_int32), ("fs_sqrt_iters", C.c_int32), ("fs_inv_iters", C.c_int32),
+                ("reserved", C.c_int32)]
 
     @classmethod
     def default(cls, **kw) -> "Hparams":

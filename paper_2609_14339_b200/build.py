@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libspectral_correction.so")
-SOURCES = ["sc_plan.cu", "sc_simt.cu", "sc_tc.cu", "sc_noalloc.cu", "sc_mask.cu", "sc_wgrad.cu", "sc_lowrank.cu"]
+SOURCES = ["sc_plan.cu", "sc_simt.cu", "sc_tc.cu", "sc_noalloc.cu", "sc_mask.cu", "sc_wgrad.cu", "sc_lowrank.cu", "sc_fullspec.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-fvisibility=hidden", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -110,6 +110,21 @@ struct StepScalars {       // scalars of one step, passed by value to kernels
   int mix;
 };
 
+// Full-spectrum variant (no rank cut): per-matrix soft projectors and the scratch one matrix needs at a time.
+struct FsMat {
+  bf16 *PUhi, *PUlo;   // m x m, P_U = U diag(d) U^T as a bf16 hi/lo pair
+  bf16 *PVhi, *PVlo;   // n x n
+};
+struct FsState {
+  std::vector<FsMat> mats;
+  double* work[5] = {};     // k x k fp64 each, k = the largest dimension of any matrix
+  double* part = nullptr;   // partial sums of the norms
+  double* scal = nullptr;   // [0] ||Gram||_F, [1] ||Y||_F
+  bf16* T1hi = nullptr;     // (G^T P_U) as hi/lo, n x m
+  bf16* T1lo = nullptr;
+  float* F = nullptr;       // (1 - alpha) scale * P_U G P_V, m x n
+};
+
 }  // namespace sc
 
 struct sc_plan {
@@ -141,6 +156,8 @@ struct sc_plan {
   std::vector<void*> dbg_out;
   bool table_dirty = true;
   bool tensor_any = false;
+  bool full = false;                  // full-spectrum soft filter (no rank cut)
+  sc::FsState fs;
   int n_sm = 0;                       // SM count of the plan's device
   // host-gradient path: copies run on their own stream, one event per shape class
   cudaStream_t copy_stream = nullptr;
@@ -212,5 +229,14 @@ sc_status tc_launch_ema_pass(sc_plan* p, ShapeClass& c, const int* idx, int coun
 sc_status tc_launch_gram(sc_plan* p, ShapeClass& c, const int* idx, int count, int panel_field_off, int rows, int slices);
 sc_status tc_launch_xpart(sc_plan* p, ShapeClass& c, const int* idx, int count, int slices);
 sc_status tc_launch_pass(sc_plan* p, ShapeClass& c, const int* idx, int count, bool transposed, int b_field_off);
+
+// ---- full-spectrum soft filter (sc_fullspec.cu) and the general A^T B tensor-core GEMM (sc_wgrad.cu) ------------
+size_t fs_layout(sc_plan* p, char* base);       // base == nullptr: only measures
+sc_status fs_refresh(sc_plan* p, int mat);
+sc_status fs_step_filter(sc_plan* p, int mat, float filt_scale);
+sc_status fs_step_update(sc_plan* p, int mat, const StepScalars& sc);
+sc_status launch_tn_gemm(const void* const* A_segs, const void* const* B_segs, int nseg, int64_t K, int64_t M, int64_t N,
+                         void* out, void* out_lo, int out_mode, float scale, float diag, unsigned* status,
+                         cudaStream_t s);
 
 }  // namespace sc

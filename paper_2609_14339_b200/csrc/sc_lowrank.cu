@@ -6,7 +6,7 @@
 // With rho <= 8 there are at most 16 flops per byte of the matrix, so every pass is bound by HBM and runs on the CUDA cores
 // with 128-bit accesses: no tensor cores here. Three passes over the matrix:
 //   phase A  reads G (and E), writes M into E, forms P                      lowrank_mq_kernel        (2 + 4 + 4 B/element)
-//   phase B  orthonormalises P (Cholesky QR twice on rho x rho Gram matrices), reads M, forms Q       (4 B/element)
+//   phase B  orthonormalises P (Cholesky QR twice, one block), reads M, forms Q   lowrank_mtp_kernel  (4 B/element)
 //   phase C  reads M, writes E = M - P_hat Q^T                               lowrank_residual_kernel  (4 + 4 B/element)
 // All sums over rows or columns are two-stage in a fixed order (no float atomics), so results are reproducible.
 #include "sc_internal.cuh"
@@ -20,12 +20,11 @@ constexpr int kChunkA = 1024;            // columns of Q staged in shared memory
 constexpr int kColsPerBlock = 1024;      // phases B and C: 256 threads x 4 columns
 constexpr int kSlabRows = 128;           // rows of P_hat staged in shared memory at a time (phases B and C)
 constexpr int kMaxSlabs = 4096;
-constexpr int kGramRows = 2048;          // rows per block of the Gram-matrix partials of P
 
 inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 struct Layout {          // carve-up of the caller's workspace
-  size_t gram_part, gram_blocks, rinv, qpart, q_slabs, total;
+  size_t qpart, q_slabs, total;
 };
 
 int slabs_for(int64_t rows, int64_t cols) {
@@ -40,9 +39,6 @@ int slabs_for(int64_t rows, int64_t cols) {
 Layout layout_for(int64_t rows, int64_t cols, int rho) {
   Layout L{};
   size_t off = 0;
-  L.gram_blocks = (size_t)((rows + kGramRows - 1) / kGramRows);
-  L.gram_part = off; off = align256(off + L.gram_blocks * rho * rho * sizeof(float));
-  L.rinv = off;      off = align256(off + (size_t)rho * rho * sizeof(float));
   L.q_slabs = (size_t)slabs_for(rows, cols);
   L.qpart = off;     off = align256(off + L.q_slabs * (size_t)cols * rho * sizeof(float));
   L.total = off;
@@ -90,6 +86,7 @@ lowrank_mq_kernel(const void* __restrict__ G, float* __restrict__ E, const float
     }
     __syncthreads();
     if (!live) continue;
+#pragma unroll 4
     for (int j = lane * 4; j < cw; j += 128) {                      // cols % 4 == 0, so a group of four is all in or out
       const size_t off = (size_t)row * cols + c0 + j;
       float4 mv = load_g4<G_BF16>(G, off);
@@ -114,98 +111,88 @@ lowrank_mq_kernel(const void* __restrict__ G, float* __restrict__ E, const float
   }
 }
 
-// Sum of the Gram partials (fixed order), Cholesky factor Gram = R^T R and its inverse, one warp. A column whose
-// pivot has cancelled to less than 1e-6 of its own squared norm (remainder below 1e-3 of the column's norm) lies in the
-// span of the earlier columns to single precision: it is dropped (its column of R^-1 is zero).
-__global__ void lowrank_chol_kernel(const float* __restrict__ gram_part, int nblocks, int rho, float* __restrict__ rinv) {
-  __shared__ float Gm[kMaxRho][kMaxRho], R[kMaxRho][kMaxRho], Ri[kMaxRho][kMaxRho];
-  const int t = threadIdx.x;
-  if (t < rho * rho) {
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-    int b = 0;
-    for (; b + 3 < nblocks; b += 4) {
-      s0 += gram_part[(size_t)b * rho * rho + t];       s1 += gram_part[(size_t)(b + 1) * rho * rho + t];
-      s2 += gram_part[(size_t)(b + 2) * rho * rho + t]; s3 += gram_part[(size_t)(b + 3) * rho * rho + t];
-    }
-    for (; b < nblocks; ++b) s0 += gram_part[(size_t)b * rho * rho + t];
-    Gm[t / rho][t % rho] = (s0 + s1) + (s2 + s3);
-  }
-  __syncthreads();
-  if (t == 0) {
-    for (int j = 0; j < rho; ++j) {
-      for (int i = 0; i < rho; ++i) { R[j][i] = 0.f; Ri[j][i] = 0.f; }
-    }
-    for (int j = 0; j < rho; ++j) {
-      float s = Gm[j][j];
-      for (int k = 0; k < j; ++k) s -= R[k][j] * R[k][j];
-      const bool ok = Gm[j][j] > 0.f && s > 1e-6f * Gm[j][j];
-      const float rjj = ok ? sqrtf(s) : 0.f, inv = ok ? 1.f / rjj : 0.f;
-      R[j][j] = rjj;
-      for (int i = j + 1; i < rho; ++i) {
-        float v = Gm[j][i];
-        for (int k = 0; k < j; ++k) v -= R[k][j] * R[k][i];
-        R[j][i] = v * inv;
-      }
-      Ri[j][j] = inv;
-    }
-    // inverse of the upper-triangular factor, column by column (dropped columns stay zero)
-    for (int c = 0; c < rho; ++c) {
-      if (Ri[c][c] == 0.f) continue;
-      for (int i = c - 1; i >= 0; --i) {
-        float s = 0.f;
-        for (int k = i + 1; k <= c; ++k) s += R[i][k] * Ri[k][c];
-        Ri[i][c] = -s * Ri[i][i];
-      }
-    }
-    for (int i = 0; i < rho; ++i)
-      for (int c = 0; c < rho; ++c) rinv[i * rho + c] = Ri[i][c];
-  }
-}
+// P_hat = orth(P) in one block: Cholesky QR twice. Each round: Gram matrix of the rows x rho panel (per-thread partial
+// sums over a fixed row assignment, then a fixed-order tree over the block), Cholesky factor Gram = R^T R and R^-1 by
+// one thread, P <- P R^-1. A column whose pivot has cancelled to less than 1e-6 of its own squared norm (remainder
+// below 1e-3 of the column's norm) lies in the span of the earlier columns to single precision: it is dropped (its
+// column of R^-1 is zero). The panel is a few hundred KB at most and stays in L2 between the rounds.
+constexpr int kOrthThreads = 1024;
 
-// P <- P R^-1 (rows x rho, in place) and the Gram partials of the result for the next round. rinv == nullptr stands
-// for the identity (only the Gram partials are wanted: P came from outside, e.g. summed over workers).
-__global__ void __launch_bounds__(256) lowrank_apply_kernel(float* __restrict__ P, const float* __restrict__ rinv,
-                                                            float* __restrict__ gram_part, int rows, int rho,
-                                                            int rows_per_block) {
-  __shared__ float Ri[kMaxRho * kMaxRho];
-  __shared__ float part[8][kMaxRho * kMaxRho];
-  if (threadIdx.x < rho * rho)
-    Ri[threadIdx.x] = rinv ? rinv[threadIdx.x] : ((threadIdx.x / rho == threadIdx.x % rho) ? 1.f : 0.f);
-  __syncthreads();
-  const int r_lo = blockIdx.x * rows_per_block, r_hi = min(rows, r_lo + rows_per_block);
-  float g[kMaxRho * kMaxRho];
+__global__ void __launch_bounds__(kOrthThreads) lowrank_orth_kernel(float* __restrict__ P, int rows, int rho) {
+  __shared__ float part[kOrthThreads / 32][kMaxRho * kMaxRho];
+  __shared__ float Gm[kMaxRho][kMaxRho], R[kMaxRho][kMaxRho], Ri[kMaxRho][kMaxRho];
+  const int t = threadIdx.x, warp = t >> 5, lane = t & 31;
+  for (int round = 0; round < 2; ++round) {
+    float g[kMaxRho * kMaxRho];
 #pragma unroll
-  for (int e = 0; e < kMaxRho * kMaxRho; ++e) g[e] = 0.f;
-  for (int i = r_lo + threadIdx.x; i < r_hi; i += blockDim.x) {
-    float p[kMaxRho], o[kMaxRho];
+    for (int e = 0; e < kMaxRho * kMaxRho; ++e) g[e] = 0.f;
+    for (int i = t; i < rows; i += kOrthThreads) {
+      float p[kMaxRho];
 #pragma unroll
-    for (int k = 0; k < kMaxRho; ++k) p[k] = k < rho ? P[(size_t)i * rho + k] : 0.f;
+      for (int k = 0; k < kMaxRho; ++k) p[k] = k < rho ? P[(size_t)i * rho + k] : 0.f;
 #pragma unroll
-    for (int c = 0; c < kMaxRho; ++c) {
-      float s = 0.f;
+      for (int a = 0; a < kMaxRho; ++a)
 #pragma unroll
-      for (int k = 0; k < kMaxRho; ++k)
-        if (k <= c && c < rho) s = fmaf(p[k], Ri[k * rho + c], s);
-      o[c] = s;
-      if (c < rho) P[(size_t)i * rho + c] = s;
+        for (int b = a; b < kMaxRho; ++b) g[a * kMaxRho + b] = fmaf(p[a], p[b], g[a * kMaxRho + b]);
     }
 #pragma unroll
     for (int a = 0; a < kMaxRho; ++a)
 #pragma unroll
-      for (int b = 0; b < kMaxRho; ++b) g[a * kMaxRho + b] = fmaf(o[a], o[b], g[a * kMaxRho + b]);
-  }
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+      for (int b = a; b < kMaxRho; ++b) {
+        const float s = warp_sum(g[a * kMaxRho + b]);
+        if (lane == 0) part[warp][a * kMaxRho + b] = s;
+      }
+    __syncthreads();
+    if (t < kMaxRho * kMaxRho) {
+      const int a = t / kMaxRho, b = t % kMaxRho;
+      if (a <= b) {
+        float s = 0.f;
+        for (int w = 0; w < kOrthThreads / 32; ++w) s += part[w][t];
+        Gm[a][b] = s; Gm[b][a] = s;
+      }
+    }
+    __syncthreads();
+    if (t == 0) {
+      for (int j = 0; j < rho; ++j)
+        for (int i = 0; i < rho; ++i) { R[j][i] = 0.f; Ri[j][i] = 0.f; }
+      for (int j = 0; j < rho; ++j) {
+        float s = Gm[j][j];
+        for (int k = 0; k < j; ++k) s -= R[k][j] * R[k][j];
+        const bool ok = Gm[j][j] > 0.f && s > 1e-6f * Gm[j][j];
+        const float rjj = ok ? sqrtf(s) : 0.f, inv = ok ? 1.f / rjj : 0.f;
+        R[j][j] = rjj;
+        for (int i = j + 1; i < rho; ++i) {
+          float v = Gm[j][i];
+          for (int k = 0; k < j; ++k) v -= R[k][j] * R[k][i];
+          R[j][i] = v * inv;
+        }
+        Ri[j][j] = inv;
+      }
+      // inverse of the upper-triangular factor, column by column (dropped columns stay zero)
+      for (int c = 0; c < rho; ++c) {
+        if (Ri[c][c] == 0.f) continue;
+        for (int i = c - 1; i >= 0; --i) {
+          float s = 0.f;
+          for (int k = i + 1; k <= c; ++k) s += R[i][k] * Ri[k][c];
+          Ri[i][c] = -s * Ri[i][i];
+        }
+      }
+    }
+    __syncthreads();
+    for (int i = t; i < rows; i += kOrthThreads) {
+      float p[kMaxRho];
 #pragma unroll
-  for (int e = 0; e < kMaxRho * kMaxRho; ++e) {
-    const float s = warp_sum(g[e]);
-    if (lane == 0) part[warp][e] = s;
-  }
-  __syncthreads();
-  if (threadIdx.x < rho * rho) {
-    const int a = threadIdx.x / rho, b = threadIdx.x % rho;
-    float s = 0.f;
-    for (int w = 0; w < 8; ++w) s += part[w][a * kMaxRho + b];
-    gram_part[(size_t)blockIdx.x * rho * rho + threadIdx.x] = s;
+      for (int k = 0; k < kMaxRho; ++k) p[k] = k < rho ? P[(size_t)i * rho + k] : 0.f;
+#pragma unroll
+      for (int c = 0; c < kMaxRho; ++c) {
+        float s = 0.f;
+#pragma unroll
+        for (int k = 0; k < kMaxRho; ++k)
+          if (k <= c && c < rho) s = fmaf(p[k], Ri[k][c], s);
+        if (c < rho) P[(size_t)i * rho + c] = s;
+      }
+    }
+    __syncthreads();     // the same thread re-reads its own rows next round; the barrier orders the shared arrays
   }
 }
 
@@ -347,8 +334,6 @@ extern "C" sc_status sc_lowrank_compress(const void* G_dev, int grad_dtype, void
   const Layout L = layout_for(rows, cols, rho);
   if (workspace_bytes < L.total) return SC_ERR_WORKSPACE;
   char* ws = static_cast<char*>(workspace);
-  float* gram_part = reinterpret_cast<float*>(ws + L.gram_part);
-  float* rinv = reinterpret_cast<float*>(ws + L.rinv);
   float* qpart = reinterpret_cast<float*>(ws + L.qpart);
   float* E = static_cast<float*>(E_dev);
   float* P = static_cast<float*>(P_dev);
@@ -365,15 +350,8 @@ extern "C" sc_status sc_lowrank_compress(const void* G_dev, int grad_dtype, void
     ++launches;
   }
   if (phases & 2) {        // B: P_hat = orth(P) by Cholesky QR, twice; Q = M^T P_hat
-    // P may have come from outside (summed over workers), so its Gram matrix is always formed here, the same way
-    const int nblocks = (int)L.gram_blocks;
-    lowrank_apply_kernel<<<nblocks, 256, 0, s>>>(P, nullptr, gram_part, m, rho, kGramRows);
+    lowrank_orth_kernel<<<1, kOrthThreads, 0, s>>>(P, m, rho);
     ++launches;
-    for (int round = 0; round < 2; ++round) {
-      lowrank_chol_kernel<<<1, 64, 0, s>>>(gram_part, nblocks, rho, rinv);
-      lowrank_apply_kernel<<<nblocks, 256, 0, s>>>(P, rinv, gram_part, m, rho, kGramRows);
-      launches += 2;
-    }
     const void* Msrc = E ? static_cast<const void*>(E) : G_dev;
     const bool m_bf16 = E ? false : g_bf16;
     DISPATCH_RHO(rho, launch_mtp<R>(Msrc, m_bf16, P, qpart, m, n, slabs, rps, s));

@@ -59,7 +59,23 @@ bool valid_hparams(const sc_hparams* hp) {
   if (hp->optimizer == SC_OPT_ADEMAMIX &&
       (!(hp->beta3 >= 0.f && hp->beta3 < 1.f) || !(hp->mix_alpha >= 0.f) || !isfinite(hp->mix_alpha)))
     return false;
+  if (hp->full_spectrum != 0 && hp->full_spectrum != 1) return false;
+  if (hp->full_spectrum) {
+    if (!(hp->tau_p > 0.f) || hp->grad_dtype != SC_DTYPE_BF16 || hp->optimizer != SC_OPT_ADAMW || hp->max_grad_norm > 0.f)
+      return false;
+    if (hp->fs_sqrt_iters < 1 || hp->fs_sqrt_iters > 200 || hp->fs_inv_iters < 1 || hp->fs_inv_iters > 200) return false;
+  }
   return true;
+}
+
+// The full-spectrum variant has no rank and runs its contractions on 256 x 256 tensor-core tiles.
+sc_status check_full_spectrum(const sc_shape* shapes, int n_mats, int rank) {
+  if (rank != 0) return SC_ERR_INVALID_ARG;
+  for (int i = 0; i < n_mats; ++i) {
+    if (shapes[i].rows < 256 || shapes[i].cols < 256 || (shapes[i].rows % 8) || (shapes[i].cols % 8)) return SC_ERR_SHAPE;
+    if (shapes[i].rows > 8192 || shapes[i].cols > 8192) return SC_ERR_TOO_LARGE;
+  }
+  return SC_OK;
 }
 
 struct ClassKey {
@@ -336,16 +352,18 @@ sc_status sc_hparams_default(sc_hparams* hp) {
   hp->sketch_width = 0; hp->power_iters = 1; hp->engine = SC_ENGINE_AUTO; hp->collect_stats = 0; hp->seed = 0;
   hp->warm_start = 0; hp->warm_power_iters = 0;
   hp->optimizer = SC_OPT_ADAMW; hp->beta3 = 0.9999f; hp->mix_alpha = 5.f;
+  hp->full_spectrum = 0; hp->fs_sqrt_iters = 30; hp->fs_inv_iters = 14;
   return SC_OK;
 }
 
 size_t sc_plan_workspace_bytes(const sc_shape* shapes, int n_mats, int rank, const sc_hparams* hp) {
   Dims d;
   if (!valid_hparams(hp) || check_shapes(shapes, n_mats, rank) != SC_OK || !derive_dims(rank, hp, &d)) return 0;
+  if (hp->full_spectrum && check_full_spectrum(shapes, n_mats, rank) != SC_OK) return 0;
   sc_plan tmp;
   fill_plan_basics(&tmp, shapes, n_mats, rank, hp, d);
   tmp.ws = nullptr;
-  return layout(&tmp, false);
+  return layout(&tmp, false) + (hp->full_spectrum ? fs_layout(&tmp, nullptr) : 0);
 }
 
 sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int rank, float keep_ratio,
@@ -360,6 +378,7 @@ sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int 
   if (st != SC_OK) return st;
   Dims d;
   if (!derive_dims(rank, hp, &d)) return SC_ERR_INVALID_ARG;
+  if (hp->full_spectrum && (st = check_full_spectrum(shapes, n_mats, rank)) != SC_OK) return st;
   if (!workspace) return SC_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(workspace) & (kAlign - 1)) return SC_ERR_ALIGNMENT;
 
@@ -376,7 +395,9 @@ sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int 
   p->n_sm = n_sm;
   p->stream = reinterpret_cast<cudaStream_t>(stream);
   p->ws = nullptr;
-  const size_t need = layout(p, false);
+  p->full = hp->full_spectrum != 0;
+  const size_t need_base = layout(p, false);
+  const size_t need = need_base + (p->full ? fs_layout(p, nullptr) : 0);
   if (workspace_bytes < need) { delete p; return SC_ERR_WORKSPACE; }
   p->ws = static_cast<char*>(workspace);
   p->ws_bytes = need;
@@ -384,6 +405,7 @@ sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int 
   p->has_basis.assign(n_mats, 0);
   p->dbg_out.assign(n_mats, nullptr);
   layout(p, true);
+  if (p->full) fs_layout(p, p->ws + need_base);
   for (auto& c : p->classes)
     for (int id : c.mats) { p->host_tab[id].omega_t = c.omega_t; p->host_tab[id].omega = c.omega; }
 
@@ -504,6 +526,12 @@ static sc_status anchor_impl(sc_plan* p, const void* const* anchor_grads, const 
           launch_gemm(ga, a.cnt, s);
         }
       }
+  }
+  if (p->full) {      // no basis: the two soft projectors of every arrived matrix, by matrix products only
+    ProfScope ps(p, PROF_SMALL);
+    for (int w = 0; w < 2; ++w)
+      for (int id : flat[w])
+        if ((st = fs_refresh(p, id)) != SC_OK) return st;
   }
   for (int w = 0; w < 2 && p->rank > 0; ++w) {
     if (flat[w].empty()) continue;
@@ -646,6 +674,19 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
       }
       if (cudaEventRecord(p->copy_done[k], p->copy_stream) != cudaSuccess) return SC_ERR_CUDA;
     }
+  }
+  if (p->full) {
+    if (host_grads)
+      for (size_t k = 0; k < p->classes.size(); ++k)
+        if (cudaStreamWaitEvent(s, p->copy_done[k], 0) != cudaSuccess) return SC_ERR_CUDA;
+    bool any = false;
+    for (int i = 0; i < p->n_mats; ++i) {
+      { ProfScope ps(p, PROF_PROJECT); if ((st = fs_step_filter(p, i, (1.f - hp.alpha) * scale)) != SC_OK) return st; }
+      { ProfScope ps(p, PROF_UPDATE);  if ((st = fs_step_update(p, i, sc)) != SC_OK) return st; }
+      any = any || p->has_basis[i];
+    }
+    if (cudaGetLastError() != cudaSuccess) return SC_ERR_CUDA;
+    return any ? SC_OK : SC_WARN_NO_ANCHOR;
   }
   auto project = [&](ShapeClass& c) -> sc_status {
     const int cnt = (int)c.mats.size(), m = (int)c.m, n = (int)c.n;
@@ -948,6 +989,9 @@ sc_status sc_state_import(sc_plan* p, const void* host_buf, size_t bytes) {
   // the copies above read caller memory: finish them before returning
   if (cudaStreamSynchronize(p->stream) != cudaSuccess) return SC_ERR_CUDA;
   for (int i = 0; i < p->n_mats; ++i) p->has_basis[i] = flags[i];
+  if (p->full)       // the soft projectors are not part of the blob: rebuild them from the imported momentum
+    for (int i = 0; i < p->n_mats; ++i)
+      if (p->has_basis[i] && (st = fs_refresh(p, i)) != SC_OK) return st;
   p->last_tag = h.last_tag;
   return cuda_ok(cudaGetLastError());
 }
@@ -981,7 +1025,7 @@ sc_status sc_get_profile(sc_plan* p, sc_profile* out) {
 
 int64_t sc_kernel_launch_count(void) { return (int64_t)g_kernel_launches.load(); }
 
-int sc_plan_uses_tensor_cores(const sc_plan* p) { return p && p->tensor_any ? 1 : 0; }
+int sc_plan_uses_tensor_cores(const sc_plan* p) { return p && (p->tensor_any || p->full) ? 1 : 0; }
 
 const char* sc_status_string(sc_status s) {
   switch (s) {

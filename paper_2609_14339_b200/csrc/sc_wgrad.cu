@@ -255,10 +255,26 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16_mn_pair(int N) {   // M = 25
          ((uint32_t)(256 >> 4) << 24);
 }
 
+// The kernel is also the library's general "A^T B" GEMM (sc::launch_tn_gemm): up to three operand pairs are contracted
+// one after the other into the same accumulator (a split-precision product: hi*hi + lo*hi + hi*lo), the epilogue can
+// add a multiple of the identity and can write the result as fp32, as bf16, or as a bf16 hi/lo pair.
+struct TnMaps {
+  CUtensorMap a[3], b[3];
+};
+struct TnEpilogue {
+  void* out;        // out_mode 0: bf16, 1: fp32, 2: bf16 hi part of a hi/lo pair
+  void* out_lo;     // out_mode 2: the lo part
+  int out_mode;
+  float scale;      // result = scale * sum + diag * I
+  float diag;
+};
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1)
-wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_constant__ CUtensorMap map_x,
-                  void* __restrict__ G, int out_f32, int tokens, int rows, int cols, float scale, int n_fastest,
-                  unsigned* status) {
+wgrad_pair_kernel(const __grid_constant__ TnMaps maps, int nseg, TnEpilogue epi, int tokens, int rows, int cols,
+                  int n_fastest, unsigned* status) {
+  void* __restrict__ G = epi.out;
+  const int out_f32 = epi.out_mode == 1;
+  const float scale = epi.scale;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   W2Bars* bars = reinterpret_cast<W2Bars*>(smem + kW2Stages * kW2StageBytes);
@@ -295,16 +311,17 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_const
       bool dead = false;
       for (int tile = pair; tile < tiles && !dead; tile += n_pairs) {
         const int tm = n_fastest ? tile / tiles_n : tile % tiles_m, tn = n_fastest ? tile % tiles_n : tile / tiles_m;
-        for (int kc = 0; kc < kchunks; ++kc, ++it) {
+        for (int kk = 0; kk < kchunks * nseg; ++kk, ++it) {
+          const int seg = kk / kchunks, kc = kk - seg * kchunks;
           const int s = it % kW2Stages;
           if (!mbar_wait(&bars->empty[s], ((it / kW2Stages) & 1) ^ 1, abort_flag)) { dead = true; break; }
           uint8_t* st = smem + (size_t)s * kW2StageBytes;
           if (rank == 0) mbar_expect_tx(&bars->full[s], 2 * kW2StageBytes);      // both blocks' bytes
           const uint32_t leader_bar = map_to_rank(smem_u32(&bars->full[s]), 0);
           for (int b = 0; b < 2; ++b)
-            tma_load_2d_pair(st + b * kWgBox, &map_dy, leader_bar, tm * 256 + (int)rank * 128 + b * 64, kc * kWgBK);
+            tma_load_2d_pair(st + b * kWgBox, &maps.a[seg], leader_bar, tm * 256 + (int)rank * 128 + b * 64, kc * kWgBK);
           for (int b = 0; b < 2; ++b)
-            tma_load_2d_pair(st + kW2ABytes + b * kWgBox, &map_x, leader_bar, tn * 256 + (int)rank * 128 + b * 64,
+            tma_load_2d_pair(st + kW2ABytes + b * kWgBox, &maps.b[seg], leader_bar, tn * 256 + (int)rank * 128 + b * 64,
                              kc * kWgBK);
         }
       }
@@ -334,7 +351,7 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_const
         if (!mbar_wait(&bars->acc_empty[ab], ((t >> 1) & 1) ^ 1, abort_flag)) { dead = true; break; }
         tc_fence_after();
         const uint32_t d = tmem_base + ab * 256;
-        for (int kc = 0; kc < kchunks; ++kc, ++it) {
+        for (int kc = 0; kc < kchunks * nseg; ++kc, ++it) {
           const int s = it % kW2Stages;
           if (!mbar_wait(&bars->full[s], (it / kW2Stages) & 1, abort_flag)) { dead = true; break; }
           tc_fence_after();
@@ -377,7 +394,27 @@ wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_dy, const __grid_const
         if (row < rows && col < cols) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) v[j] *= scale;
-          if (out_f32) {
+          if (epi.diag != 0.f && row >= col && row < col + 16) v[row - col] += epi.diag;
+          if (epi.out_mode == 2) {        // bf16 hi/lo pair: hi = rn(v), lo = rn(v - hi)
+            bf16* oh = static_cast<bf16*>(G) + (size_t)row * cols + col;
+            bf16* ol = static_cast<bf16*>(epi.out_lo) + (size_t)row * cols + col;
+#pragma unroll
+            for (int j = 0; j < 16; j += 8) {
+              if (col + j < cols) {
+                uint32_t hw[4], lw[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const float x0 = v[j + 2 * e], x1 = v[j + 2 * e + 1];
+                  const __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
+                  const __nv_bfloat162 l2 = __floats2bfloat162_rn(x0 - __low2float(h2), x1 - __high2float(h2));
+                  hw[e] = *reinterpret_cast<const uint32_t*>(&h2);
+                  lw[e] = *reinterpret_cast<const uint32_t*>(&l2);
+                }
+                *reinterpret_cast<uint4*>(oh + j) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+                *reinterpret_cast<uint4*>(ol + j) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+              }
+            }
+          } else if (out_f32) {
             float* o = static_cast<float*>(G) + (size_t)row * cols + col;
 #pragma unroll
             for (int j = 0; j < 16; j += 8) {
@@ -447,6 +484,34 @@ bool encode_mn(CUtensorMap* out, const void* base, int64_t tokens, int64_t width
 }
 
 }  // namespace
+
+// C[M x N] = scale * sum_seg A_seg^T B_seg + diag * I on the tensor cores (pairs of SMs, 256 x 256 tiles).
+// A_seg: K x M bf16 row-major, B_seg: K x N bf16 row-major (the contraction index is the slow one in memory).
+// out_mode 0: bf16 C; 1: fp32 C; 2: C as a bf16 hi/lo pair (out, out_lo). M, N >= 256, multiples of 8; any K.
+sc_status launch_tn_gemm(const void* const* A_segs, const void* const* B_segs, int nseg, int64_t K, int64_t M, int64_t N,
+                         void* out, void* out_lo, int out_mode, float scale, float diag, unsigned* status,
+                         cudaStream_t s) {
+  if (nseg < 1 || nseg > 3 || M < 256 || N < 256 || (M % 8) || (N % 8) || K < 1) return SC_ERR_SHAPE;
+  TnMaps maps;
+  for (int i = 0; i < 3; ++i) {
+    const int j = i < nseg ? i : 0;
+    if (!encode_mn(&maps.a[i], A_segs[j], K, M) || !encode_mn(&maps.b[i], B_segs[j], K, N)) return SC_ERR_CUDA;
+  }
+  int dev = 0, n_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 2)
+    return SC_ERR_CUDA;
+  const size_t smem2 = (size_t)kW2Stages * kW2StageBytes + sizeof(W2Bars) + 1024;
+  if (cudaFuncSetAttribute(wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
+    return SC_ERR_CUDA;
+  const long long tiles2 = ((M + 255) / 256) * ((N + 255) / 256);
+  const int n_pairs = tiles2 < n_sm / 2 ? (int)tiles2 : n_sm / 2;
+  const TnEpilogue epi{out, out_lo, out_mode, scale, diag};
+  wgrad_pair_kernel<<<2 * n_pairs, 192, smem2, s>>>(maps, nseg, epi, (int)K, (int)M, (int)N, M >= N ? 1 : 0, status);
+  ++g_kernel_launches;
+  return cudaGetLastError() == cudaSuccess ? SC_OK : SC_ERR_CUDA;
+}
+
 }  // namespace sc
 
 using namespace sc;
@@ -491,9 +556,11 @@ extern "C" sc_status sc_masked_weight_grad(const void* dY_dev, const void* X_dev
     if (cudaFuncSetAttribute(wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
       return SC_ERR_CUDA;
     const int n_pairs = tiles2 < n_sm / 2 ? (int)tiles2 : n_sm / 2;
-    wgrad_pair_kernel<<<2 * n_pairs, 192, smem2, s>>>(map_dy, map_x, G_dev, out_dtype == SC_DTYPE_FP32, (int)tokens,
-                                                      (int)rows, (int)cols, scale, rows >= cols ? 1 : 0,
-                                                      static_cast<unsigned*>(status_dev));
+    TnMaps maps;
+    maps.a[0] = map_dy; maps.b[0] = map_x;
+    const TnEpilogue epi{G_dev, nullptr, out_dtype == SC_DTYPE_FP32 ? 1 : 0, scale, 0.f};
+    wgrad_pair_kernel<<<2 * n_pairs, 192, smem2, s>>>(maps, 1, epi, (int)tokens, (int)rows, (int)cols,
+                                                      rows >= cols ? 1 : 0, static_cast<unsigned*>(status_dev));
   } else {
     const long long tiles = ((rows + kWgBM - 1) / kWgBM) * ((cols + kWgBN - 1) / kWgBN);
     const int grid = tiles < n_sm ? (int)tiles : n_sm;

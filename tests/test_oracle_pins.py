@@ -569,3 +569,43 @@ def test_lowrank_error_feedback_telescopes_and_repetition_reaches_the_truncated_
         Ph, Q, Err = so.lowrank_compress(M, None, Q)
     s = np.linalg.svd(M, compute_uv=False)
     assert abs(np.linalg.norm(Err) - np.sqrt(np.sum(s[rho:] ** 2))) < 1e-8 * np.linalg.norm(M)
+
+
+# ----------------------------------------------------------------- full-spectrum soft filter (no rank cut)
+def test_full_spectrum_filter_is_the_rank_min_mn_basis_form():
+    rng = np.random.default_rng(31)
+    for m, n in ((9, 14), (14, 9), (11, 11)):
+        M = rng.standard_normal((m, n)); G = rng.standard_normal((m, n)); tau = 0.7
+        U, s, V = so.svd_exact(M)
+        want = so.filtered_gradient(U, so.filter_weights(s, tau), G, V)            # r = min(m, n)
+        assert rel(so.full_spectrum_filtered(M, G, tau), want) < 1e-12
+        PU, PV = so.full_spectrum_projectors(M, tau)
+        assert np.allclose(PU, PU.T, atol=1e-13) and np.allclose(PV, PV.T, atol=1e-13)
+        ev = np.linalg.eigvalsh(PU)
+        assert ev.min() > -1e-12 and ev.max() < 1.0                                 # 0 <= d < 1
+        assert rel(PU @ M, M @ PV) < 1e-12                                          # both equal U diag(d s) V^T
+        assert rel(PU @ M, (U * (s * so.filter_weights(s, tau))) @ V.T) < 1e-12
+        hp = so.Hyper(alpha=0.3, tau_p=tau)
+        assert rel(so.correct_full_spectrum(M, G, hp), 0.3 * G + 0.7 * want) < 1e-12
+    # diagonal momentum: P_U = P_V = diag(s / (s + tau)), elementwise closed form
+    sv = np.array([3.0, 1.0, 0.25, 0.0])
+    G = rng.standard_normal((4, 4))
+    d = sv / (sv + 0.5)
+    assert rel(so.full_spectrum_filtered(np.diag(sv), G, 0.5), d[:, None] * G * d[None, :]) < 1e-13
+
+
+def test_product_only_iteration_converges_to_the_soft_projector():
+    rng = np.random.default_rng(32)
+    m, n, tau = 24, 40, 1.5
+    M = rng.standard_normal((m, n)) @ np.diag(np.logspace(0, -1.5, n))
+    PU, PV = so.full_spectrum_projectors(M, tau)
+    errs = [rel(so.soft_projector_iterative(M @ M.T, tau, q, 30), PU) for q in (2, 4, 8, 16)]
+    assert all(b < a for a, b in zip(errs, errs[1:])) and errs[-1] < 1e-12, errs
+    errs = [rel(so.soft_projector_iterative(M.T @ M, tau, 20, q), PV) for q in (2, 4, 8, 16)]       # n > m: singular Gram
+    assert all(b < a for a, b in zip(errs, errs[1:])) and errs[-1] < 1e-9, errs
+    G = rng.standard_normal((m, n))
+    assert rel(so.full_spectrum_filtered_iterative(M, G, tau, 20, 16), so.full_spectrum_filtered(M, G, tau)) < 1e-9
+    # a direction that has not converged yet is under-weighted, never over-weighted
+    few = so.soft_projector_iterative(M @ M.T, tau, 6, 30)
+    assert np.all(np.linalg.eigvalsh(few) <= np.linalg.eigvalsh(PU) + 1e-9)
+    assert np.array_equal(so.soft_projector_iterative(np.zeros((5, 5)), tau, 10, 10), np.zeros((5, 5)))
