@@ -150,6 +150,41 @@ def test_llama8b_two_layers_warm_refresh_as_benchmarked(torch):
     print("llama8b warm worst errors", worst)
 
 
+def test_planted_subspace_against_the_exact_oracle_at_the_benchmarked_settings(torch):
+    """The well-posed part of the rule against the EXACT oracle (full fp64 SVD), at the range-finder settings bench.py
+    times (l = r, cold q = 1, warm starts with q = 0), on the attention shapes of the 8B set after three arrivals of
+    independent anchor batches: the planted rank-32 subspace (a wide spectral gap below it) and the filtered gradient
+    restricted to it must meet the stated 2e-3. The other half of the rank-64 basis lies in a gapless noise bulk where
+    the rank cut itself is ill-posed; that part is reported by bench.py, not gated."""
+    import paper_2609_14339_b200 as sc
+    import bench
+    saved = gen.CONFIGS["llama8b"]
+    gen.CONFIGS["llama8b"] = dict(saved, layers=1)
+    try:
+        device = torch.device("cuda", 0)
+        cfg, shapes, buf = bench.build_workload("llama8b", device, torch)
+    finally:
+        gen.CONFIGS["llama8b"] = saved
+    hp = sc.Hparams.default(power_iters=1, warm_start=1, warm_power_iters=0, tau_p=1e-3)
+    plan = sc.Plan(shapes, cfg["r"], cfg["keep"], hp, device=device)
+    plan.anchor_update(buf["Ga"], 0)
+    for a in (1, 2):
+        anc = []
+        for i, (m, n) in enumerate(shapes):
+            spec = gen.GradSpec(m=m, n=n, tokens=cfg["tokens"], keep=cfg["keep"], planted_rank=cfg["k"], snr=1.0, seed=0,
+                                layer=0, mat_id=i)
+            anc.append(gen.torch_gradients(spec, a, device, torch.bfloat16, anchor=True))
+        plan.anchor_update(anc, a)
+        torch.cuda.synchronize()
+    assert plan.get_device_status() == 0
+    for mat in (0, 1):                                     # 4096 x 4096 and 1024 x 4096
+        rep = bench.exact_parity_report(plan, cfg, shapes, buf, mat, 0.3, 1e-3)
+        print("exact-side report", rep)
+        assert rep["relative_gap_at_k"] > 0.1                      # the planted subspace is well separated
+        assert rep["top_k_projector_distance_U"] < TOL and rep["top_k_projector_distance_V"] < TOL, rep
+        assert rep["gfilt_top_k_rel_vs_exact"] < TOL, rep
+
+
 @pytest.mark.parametrize("rank,keep", [(8, 0.05), (16, 0.1), (32, 0.1), (128, 0.1), (256, 0.5)])
 def test_ffn_sweep_corner_cells(torch, rank, keep):
     """Config 4: one 14336x4096 matrix; every rank class of the sweep (the smallest and largest at the extreme keep
