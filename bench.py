@@ -43,13 +43,18 @@ def parse_args():
     ap.add_argument("--optimizer", default="adamw", choices=["adamw", "ademamix"],
                     help="ademamix: the dual-EMA optimizer on G_proj (one more fp32 state array, 36 B/element); use "
                          "--workload llama8b_24layers, the full 8B set does not fit in 180 GB with it")
+    ap.add_argument("--ranks", default="8,16,32,64,128,256", help="with --sweep: comma-separated ranks")
+    ap.add_argument("--keeps", default="0.05,0.1,0.25,0.5", help="with --sweep: comma-separated keep ratios")
     ap.add_argument("--sketch-width", type=int, default=0, help="l of the range finder (0 = rank)")
     ap.add_argument("--power-iters", type=int, default=1, help="q of a cold start")
-    ap.add_argument("--warm-power-iters", type=int, default=0, help="q of a warm start")
+    ap.add_argument("--warm-power-iters", type=int, default=1,
+                    help="q of a warm start (1: the planted subspace meets 2e-3 against the exact SVD from the first warm "
+                         "arrival on; 0 halves the refresh but leaves the left basis one application behind)")
     ap.add_argument("--no-exact-parity", action="store_true", help="skip the report against the exact oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--short", action="store_true", help="with --wgrad: time exactly --steps passes (profiler runs)")
+    ap.add_argument("--short", action="store_true",
+                    help="with --wgrad, --lowrank, --full-spectrum: time exactly --steps passes (profiler runs)")
     ap.add_argument("--wgrad", action="store_true",
                     help="time the masked weight gradients of one 8B-shaped layer (mask pass + tensor-core GEMM)")
     ap.add_argument("--lowrank", action="store_true",
@@ -239,6 +244,28 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def exact_side_probe(args, cfg, shapes, device, torch, sc):
+    """Distance to the paper's exact rule at the range-finder settings of this run: one matrix of the smallest shape in
+    a plan of its own, three arrivals of INDEPENDENT anchor batches (the timed loop re-sends one batch, which would
+    flatter a warm-started iteration), then the cached basis against the full fp64 SVD of the same momentum."""
+    from synth import generator as gen
+    mat = min(range(len(shapes)), key=lambda i: shapes[i][0] * shapes[i][1])
+    m, n = shapes[mat]
+    per_layer = len(cfg["shapes"])
+    spec = gen.GradSpec(m=m, n=n, tokens=cfg["tokens"], keep=cfg["keep"], planted_rank=cfg["k"], snr=1.0, seed=0,
+                        layer=mat // per_layer, mat_id=mat % per_layer)
+    hp = sc.Hparams.default(power_iters=args.power_iters, warm_start=1, warm_power_iters=args.warm_power_iters,
+                            sketch_width=args.sketch_width, tau_p=1e-3)
+    small = sc.Plan([(m, n)], cfg["r"], cfg["keep"], hp, device=device)
+    for a in range(3):
+        small.anchor_update([gen.torch_gradients(spec, a, device, torch.bfloat16, anchor=True)], a)
+    G = gen.torch_gradients(spec, 1, device, torch.bfloat16)
+    rep = exact_parity_report(small, cfg, [(m, n)], dict(G=[G]), 0, 0.3, 1e-3)
+    rep["anchor_arrivals_before"] = 3
+    small.close()
+    return rep
+
+
 # ------------------------------------------------------------------------------------------ our arm
 def build_workload(name, device, torch):
     """Parameter set, optimizer state and seeded synthetic gradients resident on the device."""
@@ -416,10 +443,7 @@ def run_ours(args):
         "tensor_cores": plan.uses_tensor_cores(),
     }
     if rank == 0 and world == 1 and not args.no_exact_parity and cfg["r"] > 0:
-        # one sampled matrix (the smallest shape) after the timed arrivals: distance to the paper's exact rule
-        mat = min(range(len(shapes)), key=lambda i: shapes[i][0] * shapes[i][1])
-        line["parity_vs_exact"] = exact_parity_report(plan, cfg, shapes, buf, mat, 0.3, 1e-3)
-        line["parity_vs_exact"]["anchor_arrivals_before"] = (args.warmup + args.steps + REFRESH_EVERY - 1) // REFRESH_EVERY
+        line["parity_vs_exact"] = exact_side_probe(args, cfg, shapes, device, torch, sc)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sec, cores, desc = oracle_per_shape_run(cfg, cfg["layers"])
         line["cpu_baseline"] = {"value": n_elems * gsize / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
@@ -454,8 +478,8 @@ def run_sweep(args):
     M2 = torch.rand((m, n), generator=g, device=device) * 4000.0 + 100.0
     Wb = torch.empty((m, n), device=device, dtype=torch.bfloat16)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)      # larger than L2
-    for keep in (0.05, 0.1, 0.25, 0.5):
-        for r in (8, 16, 32, 64, 128, 256):
+    for keep in [float(x) for x in args.keeps.split(",")]:
+        for r in [int(x) for x in args.ranks.split(",")]:
             spec = gen.GradSpec(m=m, n=n, tokens=T, keep=keep, planted_rank=max(r // 2, 1), snr=1.0, seed=0)
             G = gen.torch_gradients(spec, 1, device, torch.bfloat16)
             Ga = gen.torch_gradients(spec, 0, device, torch.bfloat16, anchor=True)
@@ -465,6 +489,7 @@ def run_sweep(args):
                 plan.correct_and_step([G], [W], [M1], [M2], 100 + i, params_bf16=[Wb])
             steady, refresh = [], []
             ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            plan.set_profiling(True)
             for i in range(args.steps):
                 flush.zero_()                                              # evict the state from L2 between iterations
                 ev[0].record()
@@ -477,6 +502,9 @@ def run_sweep(args):
                 ev[2].record()
                 torch.cuda.synchronize()
                 steady.append(ev[1].elapsed_time(ev[2]))
+            prof = plan.get_profile()
+            plan.set_profiling(False)
+            upd_ms = prof["update"]["ms"] / args.steps
             for i in range(args.steps):
                 flush.zero_()
                 torch.cuda.synchronize()
@@ -488,7 +516,9 @@ def run_sweep(args):
             ms = statistics.median(steady)
             roof = max(m * n * BYTES_PER_ELEM_STEADY / (peaks["hbm_gbs"] * 1e9), m * n * 4.0 * r / (peaks["bf16_tflops"] * 1e12)) * 1e3
             cells.append({"rank": r, "keep": keep, "steady_step_ms": ms, "roofline_ms": roof, "roofline_frac": roof / ms,
-                          "refresh_ms": statistics.median(refresh), "gradient_gbs": m * n * 2 / (ms * 1e-3) / 1e9})
+                          "refresh_ms": statistics.median(refresh), "gradient_gbs": m * n * 2 / (ms * 1e-3) / 1e9,
+                          "update_kernel_ms": upd_ms,
+                          "update_kernel_frac": m * n * BYTES_PER_ELEM_UPDATE / (peaks["hbm_gbs"] * 1e9) * 1e3 / upd_ms})
             plan.close()
             del plan, G, Ga
     print(json.dumps({"metric": "config 4 sweep: steady step ms and roofline fraction per (rank, keep) cell",
@@ -608,7 +638,7 @@ def run_lowrank(args):
     sampler = ClockSampler(0)
     e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
     times = []
-    steps = max(args.steps, 50)
+    steps = args.steps if args.short else max(args.steps, 50)
     for _ in range(steps):
         flush.zero_()
         e[0].record(); layer_pass(); e[1].record(); torch.cuda.synchronize()
@@ -672,7 +702,7 @@ def run_full_spectrum(args):
     launches0 = lib.sc_kernel_launch_count()
     sampler = ClockSampler(0)
     times = []
-    steps = max(args.steps, 20)
+    steps = args.steps if args.short else max(args.steps, 20)
     for i in range(steps):
         flush.zero_()
         ev[0].record(); plan.correct_and_step(G, W, M1, M2, 200 + i, params_bf16=Wb); ev[1].record(); torch.cuda.synchronize()

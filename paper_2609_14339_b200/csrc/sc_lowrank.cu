@@ -63,20 +63,22 @@ __device__ __forceinline__ float4 load_g4(const void* G, size_t off) {
   return *reinterpret_cast<const float4*>(static_cast<const float*>(G) + off);
 }
 
-// Phase A. One warp per row: M[i, :] = G[i, :] + E[i, :] (written back into E), P[i, :] = M[i, :] Q_prev.
+// Phase A. A warp owns ROWS rows at a time: M[i, :] = G[i, :] + E[i, :] (written back into E), P[i, :] = M[i, :] Q_prev.
 // Q_prev is staged chunk by chunk in shared memory, transposed (rho rows of kChunkA columns) so that a lane's four
-// consecutive columns are one conflict-free 128-bit read per factor.
-template <int RHO, bool G_BF16>
+// consecutive columns are one conflict-free 128-bit read per factor; with several rows per warp each such read serves
+// all of them and more loads of the matrix are in flight per lane.
+template <int RHO, bool G_BF16, int ROWS>
 __global__ void __launch_bounds__(32 * kRowsPerBlockA)
 lowrank_mq_kernel(const void* __restrict__ G, float* __restrict__ E, const float* __restrict__ Qprev,
                   float* __restrict__ P, int rows, int cols) {
   __shared__ __align__(16) float Qs[RHO][kChunkA];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row = blockIdx.x * kRowsPerBlockA + warp;
-  const bool live = row < rows;
-  float acc[RHO];
+  const int row0 = (blockIdx.x * kRowsPerBlockA + warp) * ROWS;
+  float acc[ROWS][RHO];
 #pragma unroll
-  for (int k = 0; k < RHO; ++k) acc[k] = 0.f;
+  for (int r = 0; r < ROWS; ++r)
+#pragma unroll
+    for (int k = 0; k < RHO; ++k) acc[r][k] = 0.f;
   for (int c0 = 0; c0 < cols; c0 += kChunkA) {
     const int cw = min(kChunkA, cols - c0);
     __syncthreads();
@@ -85,30 +87,41 @@ lowrank_mq_kernel(const void* __restrict__ G, float* __restrict__ E, const float
       Qs[k][j] = Qprev[(size_t)(c0 + j) * RHO + k];
     }
     __syncthreads();
-    if (!live) continue;
-#pragma unroll 4
+    if (row0 >= rows) continue;
+#pragma unroll 2
     for (int j = lane * 4; j < cw; j += 128) {                      // cols % 4 == 0, so a group of four is all in or out
-      const size_t off = (size_t)row * cols + c0 + j;
-      float4 mv = load_g4<G_BF16>(G, off);
-      if (E) {
-        const float4 e4 = *reinterpret_cast<const float4*>(E + off);
-        mv.x += e4.x; mv.y += e4.y; mv.z += e4.z; mv.w += e4.w;
-        *reinterpret_cast<float4*>(E + off) = mv;
+      float4 mv[ROWS];
+#pragma unroll
+      for (int r = 0; r < ROWS; ++r) {
+        mv[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row0 + r < rows) {
+          const size_t off = (size_t)(row0 + r) * cols + c0 + j;
+          mv[r] = load_g4<G_BF16>(G, off);
+          if (E) {
+            const float4 e4 = *reinterpret_cast<const float4*>(E + off);
+            mv[r].x += e4.x; mv[r].y += e4.y; mv[r].z += e4.z; mv[r].w += e4.w;
+            *reinterpret_cast<float4*>(E + off) = mv[r];
+          }
+        }
       }
 #pragma unroll
       for (int k = 0; k < RHO; ++k) {
         const float4 q = *reinterpret_cast<const float4*>(&Qs[k][j]);
-        acc[k] = fmaf(mv.x, q.x, acc[k]); acc[k] = fmaf(mv.y, q.y, acc[k]);
-        acc[k] = fmaf(mv.z, q.z, acc[k]); acc[k] = fmaf(mv.w, q.w, acc[k]);
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) {
+          acc[r][k] = fmaf(mv[r].x, q.x, acc[r][k]); acc[r][k] = fmaf(mv[r].y, q.y, acc[r][k]);
+          acc[r][k] = fmaf(mv[r].z, q.z, acc[r][k]); acc[r][k] = fmaf(mv[r].w, q.w, acc[r][k]);
+        }
       }
     }
   }
 #pragma unroll
-  for (int k = 0; k < RHO; ++k) acc[k] = warp_sum(acc[k]);
-  if (lane == 0 && live) {
+  for (int r = 0; r < ROWS; ++r)
 #pragma unroll
-    for (int k = 0; k < RHO; ++k) P[(size_t)row * RHO + k] = acc[k];
-  }
+    for (int k = 0; k < RHO; ++k) {
+      const float v = warp_sum(acc[r][k]);
+      if (lane == 0 && row0 + r < rows) P[(size_t)(row0 + r) * RHO + k] = v;
+    }
 }
 
 // P_hat = orth(P) in one block: Cholesky QR twice. Each round: Gram matrix of the rows x rho panel (per-thread partial
@@ -284,9 +297,16 @@ lowrank_residual_kernel(float* __restrict__ E, const float* __restrict__ Phat, c
 
 template <int RHO>
 void launch_phase_a(const void* G, bool g_bf16, float* E, const float* Q, float* P, int rows, int cols, cudaStream_t s) {
-  const int blocks = (rows + kRowsPerBlockA - 1) / kRowsPerBlockA;
-  if (g_bf16) lowrank_mq_kernel<RHO, true><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
-  else lowrank_mq_kernel<RHO, false><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
+  // four rows per warp when that still leaves every SM a few blocks, else one
+  if (rows >= 148 * 2 * kRowsPerBlockA * 4) {
+    const int blocks = (rows + kRowsPerBlockA * 4 - 1) / (kRowsPerBlockA * 4);
+    if (g_bf16) lowrank_mq_kernel<RHO, true, 4><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
+    else lowrank_mq_kernel<RHO, false, 4><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
+  } else {
+    const int blocks = (rows + kRowsPerBlockA - 1) / kRowsPerBlockA;
+    if (g_bf16) lowrank_mq_kernel<RHO, true, 1><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
+    else lowrank_mq_kernel<RHO, false, 1><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
+  }
 }
 template <int RHO>
 void launch_mtp(const void* M, bool m_bf16, const float* P, float* qpart, int rows, int cols, int slabs, int rps,

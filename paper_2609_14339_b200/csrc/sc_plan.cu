@@ -1,6 +1,7 @@
 // Host side of the spectral-correction library: the C ABI, argument checks, workspace layout and the
 // order in which the kernels of one anchor arrival / one optimizer step are queued.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -393,6 +394,9 @@ sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int 
   fill_plan_basics(p, shapes, n_mats, rank, hp, d);
   p->keep = keep_ratio;
   p->n_sm = n_sm;
+  p->no_tmem_u = getenv("SC_NO_TMEM_U") != nullptr;
+  p->ut_tiles = getenv("SC_UT_TILES") ? atoi(getenv("SC_UT_TILES")) : 0;
+  if (p->ut_tiles < 0 || p->ut_tiles > 64) p->ut_tiles = 0;
   p->stream = reinterpret_cast<cudaStream_t>(stream);
   p->ws = nullptr;
   p->full = hp->full_spectrum != 0;

@@ -162,6 +162,20 @@ __device__ __forceinline__ uint32_t umma_idesc_tf32(int N, int a_mn, int b_mn) {
          ((uint32_t)(N >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
+// A operand held in tensor memory: lane = row of the 128-row tile, one 32-bit column = two consecutive bf16 along K,
+// so a K step of 16 is 8 columns. tcgen05.cp moves exactly such a slab (128 rows x 256 bits) from a shared-memory
+// tile described like an MMA operand into tensor memory; issued by the MMA thread it is ordered with its MMAs.
+__device__ __forceinline__ void tmem_cp_128x256b(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.128x256b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+
 constexpr int kPassK = 32;                       // K per stage
 constexpr int kAtomBytes = kPassK * 128;         // one MN-major atom column: 32 K-rows x 128 bytes
 
@@ -501,6 +515,13 @@ __device__ __forceinline__ void ademamix4(const StepScalars& s, float clip, cons
 //   warps 2-9  consumers, one thread per (row, half unit): R from TMEM, W/m/v/G from swizzled shared memory,
 //            blend + AdamW, results written back in place; one elected thread sends the unit out with TMA stores
 //            and hands the stage back once those stores have read it.
+// UT = true (ranks above 64, i.e. more than one 64-wide K chunk): the U panel of a work item lives in TENSOR memory.
+// With U in shared memory every 128 x 64 tile re-fetched 32 KB of U per K chunk from L2, and at rank 128 / 256 that
+// traffic (12 / 24 B per element on top of the 28 streamed) made the kernel bound by what TMA can bring into the SM.
+// Here a work item is a run of four column tiles of one row panel: the producer sends the panel's U chunks once per
+// item through the 16 KB operand slots, the MMA thread copies them into tensor memory (tcgen05.cp, rk columns beside
+// the two accumulators) and every tile of the item takes its A operand from there; only the C^T chunks (16 KB each)
+// are fetched per tile.
 // MIX = true is the dual-EMA optimizer: a fourth fp32 array (the slow average) travels with every unit, so a stage
 // is 72 KB and only two fit beside the operands. With two stages a stage has to go back to the producer as soon as
 // its stores have read it, so a warp of its own (warp 10) issues the stores and waits for them, instead of a
@@ -519,8 +540,11 @@ struct StreamCfg {
   static constexpr int kStages = MIX ? 2 : 3;
   static constexpr int kStageBytes = kF32 * kUnitF32 + kUnitBf16;      // 56 KB / 72 KB
   static constexpr int kSmem = kStages * kStageBytes + kOpndU + kOpndC;
-  static constexpr int kThreads = MIX ? 352 : 320;
+  static constexpr int kStoreWarp = 10;                                 // MIX only
 };
+// warps: 0 producer, 1 MMA, 2-9 consumers, then one store warp (MIX)
+template <bool MIX, bool UT>
+constexpr int stream_threads() { return 320 + (MIX ? 32 : 0); }
 
 // Work items are handed out by an atomic counter: blocks do not run at the same speed (the slowest of a static split
 // finished 7% after the median), so each block's producer draws the next item when it needs one and passes the index
@@ -531,6 +555,7 @@ constexpr int kItemSlots = 8;
 struct StreamBars {
   uint64_t full[kStreamStages], empty[kStreamStages];
   uint64_t opnd_full, opnd_empty;
+  uint64_t op_full[3], op_empty[3];      // UT only: ring of three 16 KB operand slots
   uint64_t acc_full[2], acc_empty[2];
   uint64_t item_ready[kItemSlots];
   uint64_t store_ready[kStreamStages];   // MIX only: the consumers have finished a unit, the store warp may send it
@@ -554,8 +579,10 @@ __device__ __forceinline__ void decode_item(const StreamGeom& g, int item, int& 
   ct1 = min(g.col_tiles, ct0 + g.tiles_per_chunk);
 }
 
-template <bool MIX>
-__global__ void __launch_bounds__(StreamCfg<MIX>::kThreads, 1)
+constexpr int kOpSlot = 16 * 1024;      // UT: one operand slot = a 128 x 64 bf16 tile of U (hi or lo), or C^T hi + lo (2 x 8 KB)
+
+template <bool MIX, bool UT>
+__global__ void __launch_bounds__(stream_threads<MIX, UT>(), 1)
 fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx,
                            const CUtensorMap* __restrict__ maps, StreamGeom g, StepScalars sc,
                            const float* __restrict__ clip_ptr, unsigned* status, unsigned* work_counter) {
@@ -575,13 +602,16 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
     }
     mbar_init(&bars->opnd_full, 1);
     mbar_init(&bars->opnd_empty, 1);
+    for (int k = 0; k < 3; ++k) { mbar_init(&bars->op_full[k], 1); mbar_init(&bars->op_empty[k], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 8); }
     for (int k = 0; k < kItemSlots; ++k) mbar_init(&bars->item_ready[k], 1);
     bars->abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
   }
-  if (warp == 1) tmem_alloc(&bars->tmem_slot, 2 * kTileN);
+  // UT: the two accumulators plus rk columns for the U panel (hi: rk / 2 columns, lo: rk / 2), a power of two
+  const uint32_t tmem_cols = !UT ? 2 * kTileN : (2 * kTileN + nch * 64 <= 256 ? 256u : 512u);
+  if (warp == 1) tmem_alloc(&bars->tmem_slot, tmem_cols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -618,7 +648,26 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
         }
         const int row0 = rt * 128;
         for (int ct = ct0; ct < ct1 && !dead; ++ct) {
-          for (int kc = 0; kc < nch; ++kc, ++op_it) {
+          if (UT) {
+            // operand slots in the order the MMA thread consumes them: at the start of an item U hi and U lo of every
+            // K chunk, then for every tile its C^T chunks. (A thread of its own for these loads was measured and
+            // dropped: no gain on the 70B-shaped set, slower on a single matrix.)
+            const int n_u = ct == ct0 ? 2 * nch : 0;
+            for (int j = 0; j < n_u + nch && !dead; ++j, ++op_it) {
+              const int sl = op_it % 3;
+              if (!mbar_wait(&bars->op_empty[sl], ((op_it / 3) & 1) ^ 1, abort_flag)) { dead = true; break; }
+              uint8_t* dst = opnd + sl * kOpSlot;
+              mbar_expect_tx(&bars->op_full[sl], kOpSlot);
+              if (j < n_u) {
+                tma_load_2d(dst, mp + ((j & 1) ? MAP_ULO : MAP_UHI), &bars->op_full[sl], (j >> 1) * 64, row0);
+              } else {
+                const int kc = j - n_u;
+                tma_load_2d(dst, mp + MAP_CT64HI, &bars->op_full[sl], kc * 64, ct * kTileN);
+                tma_load_2d(dst + kTileN * 128, mp + MAP_CT64LO, &bars->op_full[sl], kc * 64, ct * kTileN);
+              }
+            }
+          }
+          for (int kc = 0; !UT && kc < nch; ++kc, ++op_it) {
             if (!mbar_wait(&bars->opnd_empty, (op_it & 1) ^ 1, abort_flag)) { dead = true; break; }
             const bool load_u = nch > 1 || last_panel != rt;
             mbar_expect_tx(&bars->opnd_full, kOpndC + (load_u ? kOpndU : 0));
@@ -653,7 +702,9 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
         volatile int never = 0;
         for (uint32_t u = unit_it > (uint32_t)kStages ? unit_it - kStages : 0; u < unit_it; ++u)
           mbar_wait(&bars->full[u % kStages], (u / kStages) & 1, &never);
-        if (op_it > 0) mbar_wait(&bars->opnd_full, (op_it - 1) & 1, &never);
+        if (!UT && op_it > 0) mbar_wait(&bars->opnd_full, (op_it - 1) & 1, &never);
+        if (UT)
+          for (uint32_t u = op_it > 3 ? op_it - 3 : 0; u < op_it; ++u) mbar_wait(&bars->op_full[u % 3], (u / 3) & 1, &never);
       }
     }
     __syncwarp();
@@ -675,7 +726,34 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
           if (!mbar_wait(&bars->acc_empty[ab], ((t >> 1) & 1) ^ 1, abort_flag)) { dead = true; break; }
           tc_fence_after();
           const uint32_t d = tmem_base + ab * kTileN;
-          for (int kc = 0; kc < nch; ++kc, ++op_it) {
+          if (UT) {
+            const uint32_t u_hi = tmem_base + 2 * kTileN, u_lo = u_hi + nch * 32;    // nch * 32 columns = rk / 2
+            const int n_u = ct == ct0 ? 2 * nch : 0;
+            for (int j = 0; j < n_u + nch && !dead; ++j, ++op_it) {
+              const int sl = op_it % 3;
+              if (!mbar_wait(&bars->op_full[sl], (op_it / 3) & 1, abort_flag)) { dead = true; break; }
+              tc_fence_after();
+              const uint32_t sa = uh + sl * kOpSlot;
+              if (j < n_u) {        // a U chunk: four K steps of 16 into tensor memory
+                const uint32_t dst = ((j & 1) ? u_lo : u_hi) + (j >> 1) * 32;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) tmem_cp_128x256b(dst + k * 8, umma_desc_k128(sa + k * 32));
+              } else {
+                const int kc = j - n_u;
+                const int ksteps = min(64, g.rp - kc * 64) >> 4;
+                const uint32_t sb = sa + kTileN * 128;
+                for (int k = 0; k < ksteps; ++k) {
+                  const uint32_t ah = u_hi + (kc * 4 + k) * 8, al = u_lo + (kc * 4 + k) * 8;
+                  const uint64_t bh = umma_desc_k128(sa + k * 32), bl = umma_desc_k128(sb + k * 32);
+                  umma_bf16_ts(d, ah, bh, idesc, (kc | k) != 0);
+                  umma_bf16_ts(d, ah, bl, idesc, 1);
+                  umma_bf16_ts(d, al, bh, idesc, 1);
+                }
+              }
+              umma_commit(&bars->op_empty[sl]);
+            }
+          }
+          for (int kc = 0; !UT && kc < nch; ++kc, ++op_it) {
             if (!mbar_wait(&bars->opnd_full, op_it & 1, abort_flag)) { dead = true; break; }
             tc_fence_after();
             const int ksteps = min(64, g.rp - kc * 64) >> 4;
@@ -809,7 +887,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
     }
     if (dead && lane == 0) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
     if (!MIX && leader) tma_store_wait_all();
-  } else if (MIX) {
+  } else if (MIX && warp == StreamCfg<MIX>::kStoreWarp) {
     // -------------------------------------------------------------------- store warp (dual-EMA variant only)
     if (lane == 0) {
       uint32_t unit_it = 0;
@@ -855,7 +933,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, 2 * kTileN);
+  if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
 }
 
 // A wait that nothing will ever satisfy, with a caller-chosen small poll limit: exercises the path by which a
@@ -894,9 +972,13 @@ sc_status tc_init() {
   }
   // per device: the opt-in shared-memory sizes (cheap, so simply repeated for every plan)
   if (cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
-      cudaFuncSetAttribute(fused_update_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      cudaFuncSetAttribute(fused_update_stream_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            StreamCfg<false>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
-      cudaFuncSetAttribute(fused_update_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      cudaFuncSetAttribute(fused_update_stream_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           StreamCfg<true>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(fused_update_stream_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           StreamCfg<false>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(fused_update_stream_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            StreamCfg<true>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
       cudaFuncSetAttribute(ema_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
@@ -1149,21 +1231,30 @@ sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int coun
   // then touch the same rows of DRAM, and the atomic hand-out has something to balance with. Measured on the 8B set,
   // update time per step for 1 / 2 / 4 / 8 tiles per item: 31.1 / 31.5 / 32.6 / 35.0 ms (the U panel that each item
   // reloads from L2 costs less than the locality lost with longer items).
-  g.tiles_per_chunk = 1;
+  // Ranks above 64 keep the U panel of an item in tensor memory: an item is then a run of four tiles that share it.
+  // Measured (update kernel against the HBM peak): the 70B-shaped set at rank 128 with runs of 1 (U re-fetched per tile)
+  // / 2 / 3 / 4 / 8 tiles: 0.85 / 0.91 / 0.90 / 0.89 / 0.84; one 14336 x 4096 matrix at rank 256 with runs of 1 / 2 / 3:
+  // 0.69 / 0.78 / 0.81. A single matrix at rank 128 is already at 0.93 with one tile per item (few items, all blocks on
+  // one matrix) and loses with longer items, so it keeps that.
+  const int ut_tiles = p->ut_tiles > 0 ? p->ut_tiles : (p->rp > 128 ? 3 : 2);
+  const long long items_ut = (long long)count * g.row_tiles * ((g.col_tiles + ut_tiles - 1) / ut_tiles);
+  const bool ut = p->rp > 64 && !p->no_tmem_u && (p->rp > 128 || items_ut >= 32ll * n_sm || p->ut_tiles > 0);
+  g.tiles_per_chunk = ut ? ut_tiles : 1;
   g.csplit = (g.col_tiles + g.tiles_per_chunk - 1) / g.tiles_per_chunk;
   g.n_items = count * g.row_tiles * g.csplit;
   const int grid = g.n_items < n_sm ? g.n_items : n_sm;
   if (cudaMemsetAsync(p->work_dev, 0, sizeof(unsigned), p->stream) != cudaSuccess) return SC_ERR_CUDA;
   const CUtensorMap* maps = static_cast<const CUtensorMap*>(c.tmaps);
-  if (sc.mix) {
-    const size_t smem = StreamCfg<true>::kSmem + sizeof(StreamBars) + 1024;
-    fused_update_stream_kernel<true><<<grid, StreamCfg<true>::kThreads, smem, p->stream>>>(
-        p->dev_tab, idx, maps, g, sc, p->clip_dev, p->status_dev, p->work_dev);
-  } else {
-    const size_t smem = StreamCfg<false>::kSmem + sizeof(StreamBars) + 1024;
-    fused_update_stream_kernel<false><<<grid, StreamCfg<false>::kThreads, smem, p->stream>>>(
-        p->dev_tab, idx, maps, g, sc, p->clip_dev, p->status_dev, p->work_dev);
-  }
+  const size_t smem_mix = StreamCfg<true>::kSmem + sizeof(StreamBars) + 1024;
+  const size_t smem_adam = StreamCfg<false>::kSmem + sizeof(StreamBars) + 1024;
+#define SC_LAUNCH_UPDATE(MIXV, UTV, SMEM)                                                                       \
+  fused_update_stream_kernel<MIXV, UTV><<<grid, stream_threads<MIXV, UTV>(), SMEM, p->stream>>>(                \
+      p->dev_tab, idx, maps, g, sc, p->clip_dev, p->status_dev, p->work_dev)
+  if (sc.mix && ut) SC_LAUNCH_UPDATE(true, true, smem_mix);
+  else if (sc.mix) SC_LAUNCH_UPDATE(true, false, smem_mix);
+  else if (ut) SC_LAUNCH_UPDATE(false, true, smem_adam);
+  else SC_LAUNCH_UPDATE(false, false, smem_adam);
+#undef SC_LAUNCH_UPDATE
   ++g_kernel_launches;
   return cuda_ok(cudaGetLastError());
 }
