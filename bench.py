@@ -365,9 +365,17 @@ def run_ours(args):
     bytes_steady = BYTES_PER_ELEM_STEADY + (8.0 if mix else 0.0)               # + read and write of the slow EMA
     bytes_update = BYTES_PER_ELEM_UPDATE + (8.0 if mix else 0.0)
 
-    def one_step(i):
+    refresh_events = []           # (start, end) CUDA events around the timed anchor arrivals, on the plan's stream
+
+    def one_step(i, timed=False):
         if i % REFRESH_EVERY == 0:
+            if timed:
+                ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                ev[0].record()
             plan.anchor_update(buf["Ga"], i)
+            if timed:
+                ev[1].record()
+                refresh_events.append(ev)
         plan.correct_and_step(buf["G"], buf["W"], buf["M1"], buf["M2"], 100 + i, params_bf16=buf["Wb"],
                               exp_avg_slow=buf["MS"])
 
@@ -391,7 +399,7 @@ def run_ours(args):
     sync_all()
     e0.record()
     for i in range(args.steps):
-        one_step(args.warmup + i)
+        one_step(args.warmup + i, timed=True)
     e1.record()
     sync_all()
     ms_total = e0.elapsed_time(e1)
@@ -407,7 +415,9 @@ def run_ours(args):
     nprof = args.steps
     n_refresh = sum(1 for i in range(args.steps) if (args.warmup + i) % REFRESH_EVERY == 0)
     steady_ms = (prof["projection"]["ms"] + prof["filter"]["ms"] + prof["update"]["ms"]) / nprof
-    refresh_ms = (prof["anchor_ema"]["ms"] + prof["basis_passes"]["ms"] + prof["basis_small"]["ms"]) / max(n_refresh, 1)
+    # wall time of an arrival on the plan's stream (the per-phase spans of different shape classes overlap: the basis
+    # builds of the classes run on streams of their own, so their sum is more than the wall time)
+    refresh_ms = (sum(a.elapsed_time(b) for a, b in refresh_events) / len(refresh_events)) if refresh_events else 0.0
     update_ms = prof["update"]["ms"] / nprof
 
     peaks = measured_peaks()

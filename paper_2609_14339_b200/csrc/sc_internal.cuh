@@ -161,6 +161,11 @@ struct sc_plan {
   int ut_tiles = 0;                   // test hook (environment SC_UT_TILES): tiles per item with U in tensor memory
   sc::FsState fs;
   int n_sm = 0;                       // SM count of the plan's device
+  // anchor refresh: the basis builds of different shape classes run on streams of their own (fork / join on `stream`)
+  bool overlap_classes = true;        // test hook (environment SC_NO_OVERLAP): queue everything on `stream` instead
+  std::vector<cudaStream_t> class_streams;
+  cudaEvent_t fork_ev = nullptr;
+  std::vector<cudaEvent_t> join_evs;
   // host-gradient path: copies run on their own stream, one event per shape class
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t copy_gate = nullptr;

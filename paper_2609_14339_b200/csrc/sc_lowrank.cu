@@ -131,6 +131,7 @@ lowrank_mq_kernel(const void* __restrict__ G, float* __restrict__ E, const float
 // column of R^-1 is zero). The panel is a few hundred KB at most and stays in L2 between the rounds.
 constexpr int kOrthThreads = 1024;
 
+template <int kMaxRho>      // instantiated per rho, so that every loop below has exactly rho trips
 __global__ void __launch_bounds__(kOrthThreads) lowrank_orth_kernel(float* __restrict__ P, int rows, int rho) {
   __shared__ float part[kOrthThreads / 32][kMaxRho * kMaxRho];
   __shared__ float Gm[kMaxRho][kMaxRho], R[kMaxRho][kMaxRho], Ri[kMaxRho][kMaxRho];
@@ -297,16 +298,11 @@ lowrank_residual_kernel(float* __restrict__ E, const float* __restrict__ Phat, c
 
 template <int RHO>
 void launch_phase_a(const void* G, bool g_bf16, float* E, const float* Q, float* P, int rows, int cols, cudaStream_t s) {
-  // four rows per warp when that still leaves every SM a few blocks, else one
-  if (rows >= 148 * 2 * kRowsPerBlockA * 4) {
-    const int blocks = (rows + kRowsPerBlockA * 4 - 1) / (kRowsPerBlockA * 4);
-    if (g_bf16) lowrank_mq_kernel<RHO, true, 4><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
-    else lowrank_mq_kernel<RHO, false, 4><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
-  } else {
-    const int blocks = (rows + kRowsPerBlockA - 1) / kRowsPerBlockA;
-    if (g_bf16) lowrank_mq_kernel<RHO, true, 1><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
-    else lowrank_mq_kernel<RHO, false, 1><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
-  }
+  // one row per warp: measured against four rows per warp (more loads in flight per lane, fewer streams) on
+  // 14336 x 4096: 0.18 ms against 0.25 ms
+  const int blocks = (rows + kRowsPerBlockA - 1) / kRowsPerBlockA;
+  if (g_bf16) lowrank_mq_kernel<RHO, true, 1><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
+  else lowrank_mq_kernel<RHO, false, 1><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
 }
 template <int RHO>
 void launch_mtp(const void* M, bool m_bf16, const float* P, float* qpart, int rows, int cols, int slabs, int rps,
@@ -370,7 +366,7 @@ extern "C" sc_status sc_lowrank_compress(const void* G_dev, int grad_dtype, void
     ++launches;
   }
   if (phases & 2) {        // B: P_hat = orth(P) by Cholesky QR, twice; Q = M^T P_hat
-    lowrank_orth_kernel<<<1, kOrthThreads, 0, s>>>(P, m, rho);
+    DISPATCH_RHO(rho, (lowrank_orth_kernel<R><<<1, kOrthThreads, 0, s>>>(P, m, rho)));
     ++launches;
     const void* Msrc = E ? static_cast<const void*>(E) : G_dev;
     const bool m_bf16 = E ? false : g_bf16;

@@ -424,6 +424,13 @@ sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int 
     ok = cudaEventCreateWithFlags(&p->staging_ev[i], cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&p->copy_gate, cudaEventDisableTiming) == cudaSuccess;
+  p->overlap_classes = getenv("SC_NO_OVERLAP") == nullptr;
+  p->class_streams.assign(p->classes.size(), nullptr);
+  p->join_evs.assign(p->classes.size(), nullptr);
+  ok = ok && cudaEventCreateWithFlags(&p->fork_ev, cudaEventDisableTiming) == cudaSuccess;
+  for (size_t k = 0; ok && k < p->classes.size(); ++k)
+    ok = cudaStreamCreateWithFlags(&p->class_streams[k], cudaStreamNonBlocking) == cudaSuccess &&
+         cudaEventCreateWithFlags(&p->join_evs[k], cudaEventDisableTiming) == cudaSuccess;
   p->copy_done.resize(p->classes.size(), nullptr);
   for (size_t k = 0; ok && k < p->classes.size(); ++k)
     ok = cudaEventCreateWithFlags(&p->copy_done[k], cudaEventDisableTiming) == cudaSuccess;
@@ -455,6 +462,11 @@ sc_status sc_plan_destroy(sc_plan* p) {
   for (cudaEvent_t e : p->copy_done)
     if (e) cudaEventDestroy(e);
   if (p->copy_gate) cudaEventDestroy(p->copy_gate);
+  if (p->fork_ev) cudaEventDestroy(p->fork_ev);
+  for (cudaEvent_t e : p->join_evs)
+    if (e) cudaEventDestroy(e);
+  for (cudaStream_t cs : p->class_streams)
+    if (cs) { cudaStreamSynchronize(cs); cudaStreamDestroy(cs); }
   if (p->copy_stream) { cudaStreamSynchronize(p->copy_stream); cudaStreamDestroy(p->copy_stream); }
   if (p->staging) cudaFreeHost(p->staging);
   delete p;
@@ -537,11 +549,9 @@ static sc_status anchor_impl(sc_plan* p, const void* const* anchor_grads, const 
       for (int id : flat[w])
         if ((st = fs_refresh(p, id)) != SC_OK) return st;
   }
-  for (int w = 0; w < 2 && p->rank > 0; ++w) {
-    if (flat[w].empty()) continue;
-    const std::vector<ActiveClass>& ac = act[w];
-    const int* glob = w ? p->idx_glob2 : p->idx_glob;
-    const int n_all = (int)flat[w].size();
+  // The basis build of one group of matrices (ac: their classes; glob / n_all: the flat list for the kernels that take
+  // all classes in one launch). Everything is queued on p->stream as it is at the time of the call.
+  auto run_chain = [&](const std::vector<ActiveClass>& ac, const int* glob, int n_all, int w) {
     const int q = w ? p->hp.warm_power_iters : p->q;
     // one sweep over the momentum: transposed ? Z <- M^T B : Y <- M B
     bool first_sweep = true;
@@ -553,9 +563,9 @@ static sc_status anchor_impl(sc_plan* p, const void* const* anchor_grads, const 
         if (a.c->tensor) { tc_launch_pass(p, *a.c, a.idx, a.cnt, transposed, offB); continue; }
         const int tB = offB == OFF(omega_t);
         if (!transposed)
-          launch_gemm(gemm(p, a.idx, OFF(Manc), offB, OFF(Y), m, lp, n, n, tB ? n : lp, lp, 0, tB), a.cnt, s);
+          launch_gemm(gemm(p, a.idx, OFF(Manc), offB, OFF(Y), m, lp, n, n, tB ? n : lp, lp, 0, tB), a.cnt, p->stream);
         else
-          launch_gemm(gemm(p, a.idx, OFF(Manc), offB, OFF(Z), n, lp, m, n, lp, lp, 1, 0), a.cnt, s);
+          launch_gemm(gemm(p, a.idx, OFF(Manc), offB, OFF(Z), n, lp, m, n, lp, lp, 1, 0), a.cnt, p->stream);
       }
       first_sweep = false;
     };
@@ -564,7 +574,7 @@ static sc_status anchor_impl(sc_plan* p, const void* const* anchor_grads, const 
       {
         ProfScope ps(p, PROF_SMALL);
         for (const auto& a : ac)
-          launch_warm_start(p->dev_tab, a.idx, a.cnt, (int)a.c->n, lp, p->l, rp, p->rank, p->hp.seed, s);
+          launch_warm_start(p->dev_tab, a.idx, a.cnt, (int)a.c->n, lp, p->l, rp, p->rank, p->hp.seed, p->stream);
       }
       pass(OFF(Z2), false);
     } else {
@@ -585,14 +595,36 @@ static sc_status anchor_impl(sc_plan* p, const void* const* anchor_grads, const 
     cholqr(p, ac, glob, n_all, OFF(Z), OFF(Z2), false, true, 2);
     {
       ProfScope ps(p, PROF_SMALL);
-      launch_jacobi(p->dev_tab, glob, n_all, lp, rp, p->rank, p->hp.tau_p, s);                        // + Eq. 2
+      launch_jacobi(p->dev_tab, glob, n_all, lp, rp, p->rank, p->hp.tau_p, p->stream);                 // + Eq. 2
       for (const auto& a : ac) {
         const int m = (int)a.c->m, n = (int)a.c->n;
-        launch_gemm(gemm(p, a.idx, OFF(Y), OFF(ub), OFF(U), m, rp, lp, lp, rp, rp, 0, 0), a.cnt, s);
-        launch_gemm(gemm(p, a.idx, OFF(Z), OFF(wb), OFF(V), n, rp, lp, lp, rp, rp, 0, 0), a.cnt, s);
+        launch_gemm(gemm(p, a.idx, OFF(Y), OFF(ub), OFF(U), m, rp, lp, lp, rp, rp, 0, 0), a.cnt, p->stream);
+        launch_gemm(gemm(p, a.idx, OFF(Z), OFF(wb), OFF(V), n, rp, lp, lp, rp, rp, 0, 0), a.cnt, p->stream);
         refresh_operands(p, *a.c, a.idx, a.cnt);
       }
     }
+  };
+  const size_t n_chains = act[0].size() + act[1].size();
+  if (p->rank > 0 && p->overlap_classes && n_chains > 1) {
+    // The chains of different shape classes are independent (every matrix has its own panels and factors), so each
+    // class runs on a stream of its own: the short, latency-bound factorisation kernels of one class then run beside
+    // the HBM-bound sweeps of another instead of leaving the chip idle between them.
+    cudaStream_t main_stream = p->stream;
+    if (cudaEventRecord(p->fork_ev, main_stream) != cudaSuccess) return SC_ERR_CUDA;
+    for (int w = 0; w < 2; ++w)
+      for (const auto& a : act[w]) {
+        const size_t ci = (size_t)(a.c - p->classes.data());
+        cudaStream_t cs = p->class_streams[ci];
+        if (cudaStreamWaitEvent(cs, p->fork_ev, 0) != cudaSuccess) return SC_ERR_CUDA;
+        p->stream = cs;
+        run_chain(std::vector<ActiveClass>{a}, a.idx, a.cnt, w);
+        p->stream = main_stream;
+        if (cudaEventRecord(p->join_evs[ci], cs) != cudaSuccess || cudaStreamWaitEvent(main_stream, p->join_evs[ci], 0) != cudaSuccess)
+          return SC_ERR_CUDA;
+      }
+  } else {
+    for (int w = 0; w < 2 && p->rank > 0; ++w)
+      if (!flat[w].empty()) run_chain(act[w], w ? p->idx_glob2 : p->idx_glob, (int)flat[w].size(), w);
   }
   for (int w = 0; w < 2; ++w)
     for (int id : flat[w]) p->has_basis[id] = 1;

@@ -4,6 +4,8 @@
 // l x l matrices, the r x r filter, norms) for all plans and (b) the large contractions too when the plan
 // runs on the fp32 engine (fp32 gradients, shapes the tensor-core kernels do not take).
 // Kernels are launched once per shape class; blockIdx.z selects the matrix through idx[] and the table.
+#include <algorithm>
+
 #include "sc_internal.cuh"
 
 namespace sc {
@@ -574,12 +576,19 @@ __global__ void __launch_bounds__(256) chol_kernel(const MatDev* tab, const int*
   __shared__ float invd[kMaxRank];
   __shared__ float piv_inv;
   const MatDev& md = tab[idx[blockIdx.x]];
-  const float* G = md.gram;
+  const float* G = md.gram;     // redirected to shared memory below when kSmem
   float* Rg = field<float>(md, offR);
   float* Rig = md.rinv;
   float* R = kSmem ? chol_smem : Rg;
   float* Ri = kSmem ? chol_smem + (size_t)lp * lp : Rig;
   const int t = threadIdx.x;
+  if (kSmem) {
+    // the Gram matrix comes into shared memory once (into the array that will hold the inverse, which is written only
+    // after the factor is complete), so that no column step waits for a global load
+    for (int e = t; e < lp * lp; e += 256) Ri[e] = md.gram[e];
+    G = Ri;
+    __syncthreads();
+  }
   for (int j = 0; j < lp; ++j) {
     const int i = t;
     float s = 0.f;
@@ -775,29 +784,49 @@ void launch_filter_weights(const MatDev* tab, const int* idx, int count, int rp,
 // =====================================================================================================
 // bf16 hi/lo splits of the basis: U ~= Uhi + Ulo (m x rp), V^T ~= Vthi + Vtlo (rp x n, transposed).
 // =====================================================================================================
+// blockIdx.y == 0: U (m x rp fp32) -> Uhi, Ulo (row stride rk; columns rp..rk-1 stay zero), four columns per thread.
+// blockIdx.y == 1: V (n x rp fp32) -> Vthi, Vtlo = the TRANSPOSE (rp x n) through 32 x 32 shared-memory tiles, so that
+// both the reads (along the rank index) and the writes (along n) are coalesced.
 __global__ void __launch_bounds__(256) split_basis_kernel(const MatDev* tab, const int* idx, int m, int n, int rp,
                                                           int rk) {
   const MatDev& md = tab[idx[blockIdx.z]];
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  const int64_t nu = (int64_t)m * rp, nv = (int64_t)n * rp;
-  // U is m x rp (fp32); the bf16 copies have row stride rk, columns rp..rk-1 stay zero
-  for (int64_t e = t0; e < nu; e += stride) {
-    const int64_t i = e / rp, k = e % rp;
-    split2(md.U[e], md.Uhi[i * rk + k], md.Ulo[i * rk + k]);
-  }
-  // V is n x rp; write the transpose rp x n (threads run along n for coalesced stores)
-  for (int64_t e = t0; e < nv; e += stride) {
-    const int64_t k = e / n, j = e % n;
-    split2(md.V[(size_t)j * rp + k], md.Vthi[e], md.Vtlo[e]);
+  if (blockIdx.y == 0) {
+    const int q = rp >> 2;                                     // rp is a multiple of 16
+    const int64_t nu4 = (int64_t)m * q;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < nu4; e += (int64_t)gridDim.x * blockDim.x) {
+      const int64_t i = e / q;
+      const int k = (int)(e - i * q) * 4;
+      const float4 u = *reinterpret_cast<const float4*>(md.U + i * rp + k);
+      bf16 h[4], l[4];
+      split2(u.x, h[0], l[0]); split2(u.y, h[1], l[1]); split2(u.z, h[2], l[2]); split2(u.w, h[3], l[3]);
+      *reinterpret_cast<uint2*>(md.Uhi + i * rk + k) = *reinterpret_cast<const uint2*>(h);
+      *reinterpret_cast<uint2*>(md.Ulo + i * rk + k) = *reinterpret_cast<const uint2*>(l);
+    }
+  } else {
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;    // 32 x 8 threads
+    const int ktiles = rp >> 5 ? (rp + 31) >> 5 : 1, jtiles = (n + 31) >> 5;
+    for (int t = blockIdx.x; t < ktiles * jtiles; t += gridDim.x) {
+      const int j0 = (t / ktiles) * 32, k0 = (t % ktiles) * 32;
+      __syncthreads();
+      for (int r = ty; r < 32; r += 8) {
+        const int j = j0 + r, k = k0 + tx;
+        tile[r][tx] = (j < n && k < rp) ? md.V[(size_t)j * rp + k] : 0.f;
+      }
+      __syncthreads();
+      for (int r = ty; r < 32; r += 8) {
+        const int k = k0 + r, j = j0 + tx;
+        if (k < rp && j < n) split2(tile[tx][r], md.Vthi[(size_t)k * n + j], md.Vtlo[(size_t)k * n + j]);
+      }
+    }
   }
 }
 
 void launch_split_basis(const MatDev* tab, const int* idx, int count, int m, int n, int rp, int rk, cudaStream_t s) {
   if (count <= 0 || rp <= 0) return;
-  int64_t tot = (int64_t)(m > n ? m : n) * rp;
-  int blocks = (int)((tot + 255) / 256 < 1184 ? (tot + 255) / 256 : 1184);
-  split_basis_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, m, n, rp, rk);
+  const int64_t work = std::max<int64_t>((int64_t)m * rp / 4, (int64_t)((n + 31) / 32) * ((rp + 31) / 32) * 256);
+  const int blocks = (int)std::min<int64_t>((work + 255) / 256, 592);
+  split_basis_kernel<<<dim3(blocks, 2, count), 256, 0, s>>>(tab, idx, m, n, rp, rk);
   ++g_kernel_launches;
 }
 

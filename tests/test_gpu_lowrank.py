@@ -31,7 +31,8 @@ def _dev(torch, arr, dtype):
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
-@pytest.mark.parametrize("m,n,rho", [(200, 136, 1), (330, 520, 4), (64, 2052, 2), (129, 1028, 8)])
+# the last two span more than one column range of phase A (4096 columns per block up to rank 4, 2048 above)
+@pytest.mark.parametrize("m,n,rho", [(200, 136, 1), (330, 520, 4), (64, 2052, 2), (129, 1028, 8), (72, 4104, 4), (40, 2056, 8)])
 def test_three_steps_with_error_feedback_match_the_oracle(torch, dtype, m, n, rho):
     import paper_2609_14339_b200 as sc
     Q = sc.lowrank_init_q(n, rho, seed=9)
