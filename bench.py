@@ -143,8 +143,7 @@ def _oracle_one_matrix(cfg, m, n, steps, warmup, with_svd=True):
         if with_svd and i % REFRESH_EVERY == 0:
             t0 = time.perf_counter()
             so.anchor_update(st, Ganc, hp, cfg["r"], mode="exact")
-            if i >= warmup or steps == 0:
-                t_refresh += time.perf_counter() - t0; n_refresh += 1
+            t_refresh += time.perf_counter() - t0; n_refresh += 1        # every arrival is timed, warm-up ones too
         t0 = time.perf_counter()
         Ws, ms, vs, _ = so.correct_and_step([st], [G], [W], [mm], [vv], 100 + i, hp)
         W, mm, vv = Ws[0], ms[0], vs[0]
@@ -159,8 +158,7 @@ def oracle_sample_run(cfg, steps, warmup):
     m, n = min(cfg["shapes"], key=lambda s: s[0] * s[1])
     t_total = 0.0
     steady, refresh = _oracle_one_matrix(cfg, m, n, steps, warmup)
-    n_refresh = sum(1 for i in range(warmup, warmup + steps) if i % REFRESH_EVERY == 0)
-    t_total = steady * steps + (refresh or 0.0) * n_refresh
+    t_total = steady * steps + (refresh or 0.0) * steps / REFRESH_EVERY        # one arrival every REFRESH_EVERY steps
     cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
     desc = ("one %dx%d matrix of the set (%d elements of %d), exact mode: Eq.1 + full fp64 SVD every %d steps, "
             "projection/filter/blend/AdamW every step; %d timed steps" % (m, n, m * n, 0, REFRESH_EVERY, steps))
@@ -734,7 +732,7 @@ def run_full_spectrum(args):
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": "full_spectrum_attention_%dlayers" % args.layers, "matrices": len(shapes), "elements": elems,
-                   "tokens": T, "keep": keep, "tau_p": tau, "sqrt_iters": 30, "inv_iters": 14,
+                   "tokens": T, "keep": keep, "tau_p": tau, "sqrt_iters": hp.fs_sqrt_iters, "inv_iters": hp.fs_inv_iters,
                    "l2": "256 MB buffer rewritten between timed iterations"},
         "gpu_launches": launches, "contraction_ms": gemm_ms, "adamw_ms": upd_ms, "anchor_refresh_ms": refresh_ms,
         "flops_executed_per_step": flops_exec, "flops_algorithmic_per_step": flops_alg,

@@ -115,8 +115,10 @@ typedef struct sc_hparams {
                               Gram matrix, then Newton-Schulz inverse), in fp64; every step is two dense tensor-core
                               contractions per matrix plus one elementwise AdamW pass. Needs tau_p > 0, bf16 gradients,
                               AdamW, no clipping, rows and cols multiples of 8 in [256, 8192]. */
-  int32_t fs_sqrt_iters;   /* full_spectrum: iterations of the square-root stage, 1..200 (default 30) */
-  int32_t fs_inv_iters;    /* full_spectrum: iterations of the inverse stage, 1..200 (default 14) */
+  int32_t fs_sqrt_iters;   /* full_spectrum: iterations of the square-root stage, 1..200 (default 24; directions with
+                              s_i below about 1e-3 of the largest are still under-weighted then, which only lowers d_i) */
+  int32_t fs_inv_iters;    /* full_spectrum: iterations of the inverse stage, 1..200 (default 12: enough for
+                              (s_max + tau_p) / tau_p up to a few hundred) */
   int32_t reserved;
 } sc_hparams;
 

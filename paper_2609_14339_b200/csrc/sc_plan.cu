@@ -353,7 +353,7 @@ sc_status sc_hparams_default(sc_hparams* hp) {
   hp->sketch_width = 0; hp->power_iters = 1; hp->engine = SC_ENGINE_AUTO; hp->collect_stats = 0; hp->seed = 0;
   hp->warm_start = 0; hp->warm_power_iters = 0;
   hp->optimizer = SC_OPT_ADAMW; hp->beta3 = 0.9999f; hp->mix_alpha = 5.f;
-  hp->full_spectrum = 0; hp->fs_sqrt_iters = 30; hp->fs_inv_iters = 14;
+  hp->full_spectrum = 0; hp->fs_sqrt_iters = 24; hp->fs_inv_iters = 12;
   return SC_OK;
 }
 

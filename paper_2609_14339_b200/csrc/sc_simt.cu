@@ -4,6 +4,8 @@
 // l x l matrices, the r x r filter, norms) for all plans and (b) the large contractions too when the plan
 // runs on the fp32 engine (fp32 gradients, shapes the tensor-core kernels do not take).
 // Kernels are launched once per shape class; blockIdx.z selects the matrix through idx[] and the table.
+#include <cooperative_groups.h>
+
 #include <algorithm>
 
 #include "sc_internal.cuh"
@@ -643,6 +645,90 @@ __global__ void __launch_bounds__(256) chol_kernel(const MatDev* tab, const int*
   }
 }
 
+// The same factorisation for 128 < lp <= 256, still on-chip: two full lp x lp arrays no longer fit in one SM's shared
+// memory, so the upper triangle is kept PACKED (lp (lp + 1) / 2 floats, 129 KB at lp = 256) and everything happens in
+// place: the Gram matrix is loaded into the packed array, row j of the factor overwrites row j of the Gram matrix (it
+// is the last use of that row), the factor is copied out, and then the packed array is inverted in place column by
+// column (x_j = -R^-1[0:j, 0:j] R[0:j, j] / r_jj uses only the already inverted leading block and column j itself).
+// One thread per column, lp <= 256 threads.
+__device__ __forceinline__ int tri_off(int j, int lp) { return j * lp - (j * (j - 1)) / 2; }   // start of packed row j
+
+__global__ void __launch_bounds__(256) chol_packed_kernel(const MatDev* tab, const int* idx, int lp, int offR) {
+  extern __shared__ __align__(16) float tri[];                 // packed upper triangle, row j: entries (j, j..lp-1)
+  __shared__ float invd[kMaxRank];
+  __shared__ float colj[kMaxRank];
+  __shared__ int roff[kMaxRank];                                // roff[k] + c = position of element (k, c), c >= k
+  __shared__ float piv_inv;
+  const MatDev& md = tab[idx[blockIdx.x]];
+  float* Rg = field<float>(md, offR);
+  float* Rig = md.rinv;
+  const int t = threadIdx.x;
+  if (t < lp) roff[t] = tri_off(t, lp) - t;
+  __syncthreads();
+  for (int e = t; e < lp * lp; e += 256) {                      // coalesced read of the Gram matrix, upper part kept
+    const int j = e / lp, i = e - j * lp;
+    if (i >= j) tri[roff[j] + i] = md.gram[e];
+  }
+  __syncthreads();
+  // factor: R[j][i] = (G[j][i] - sum_{k<j} R[k][j] R[k][i]) / r_jj, in place
+  for (int j = 0; j < lp; ++j) {
+    const int i = t;
+    float s = 0.f;
+    if (i >= j && i < lp) {
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+      int k = 0;
+      for (; k + 3 < j; k += 4) {
+        const int o0 = roff[k], o1 = roff[k + 1], o2 = roff[k + 2], o3 = roff[k + 3];
+        s0 = fmaf(tri[o0 + j], tri[o0 + i], s0); s1 = fmaf(tri[o1 + j], tri[o1 + i], s1);
+        s2 = fmaf(tri[o2 + j], tri[o2 + i], s2); s3 = fmaf(tri[o3 + j], tri[o3 + i], s3);
+      }
+      for (; k < j; ++k) { const int o = roff[k]; s0 = fmaf(tri[o + j], tri[o + i], s0); }
+      s = tri[roff[j] + i] - ((s0 + s1) + (s2 + s3));
+    }
+    if (i == j) {
+      const float gjj = tri[roff[j] + j];
+      const bool ok = (s > 1e-6f * gjj) && (gjj > 0.f);
+      const float rjj = ok ? sqrtf(s) : 0.f;
+      piv_inv = ok ? 1.f / rjj : 0.f;
+      invd[j] = piv_inv;
+    }
+    __syncthreads();
+    if (i == j) tri[roff[j] + j] = piv_inv > 0.f ? 1.f / piv_inv : 0.f;
+    if (i > j && i < lp) tri[roff[j] + i] = s * piv_inv;
+    __syncthreads();
+  }
+  // copy the factor out (full lp x lp, zeros below the diagonal)
+  for (int e = t; e < lp * lp; e += 256) {
+    const int j = e / lp, i = e - j * lp;
+    Rg[e] = i >= j ? tri[roff[j] + i] : 0.f;
+  }
+  __syncthreads();
+  // in-place inverse, column by column
+  for (int j = 0; j < lp; ++j) {
+    if (t < j) colj[t] = tri[roff[t] + j];                        // R[0:j, j], about to be overwritten
+    __syncthreads();
+    if (t < j) {
+      // x_t = -(sum_{k=t}^{j-1} Rinv[t][k] R[k][j]) / r_jj ; row t of the inverted block is packed row t, entries t..j-1
+      const int o = roff[t];
+      float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+      int k = t;
+      for (; k + 3 < j; k += 4) {
+        s0 = fmaf(tri[o + k], colj[k], s0); s1 = fmaf(tri[o + k + 1], colj[k + 1], s1);
+        s2 = fmaf(tri[o + k + 2], colj[k + 2], s2); s3 = fmaf(tri[o + k + 3], colj[k + 3], s3);
+      }
+      for (; k < j; ++k) s0 = fmaf(tri[o + k], colj[k], s0);
+      tri[o + j] = -((s0 + s1) + (s2 + s3)) * invd[j];
+    } else if (t == j) {
+      tri[roff[j] + j] = invd[j];
+    }
+    __syncthreads();
+  }
+  for (int e = t; e < lp * lp; e += 256) {
+    const int j = e / lp, i = e - j * lp;
+    Rig[e] = i >= j ? tri[roff[j] + i] : 0.f;
+  }
+}
+
 void launch_chol(const MatDev* tab, const int* idx, int count, int lp, int offR, cudaStream_t s) {
   if (count <= 0 || lp <= 0) return;
   if (lp <= 128) {
@@ -650,7 +736,9 @@ void launch_chol(const MatDev* tab, const int* idx, int count, int lp, int offR,
     cudaFuncSetAttribute(chol_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 128 * 128 * 4);
     chol_kernel<true><<<count, 256, smem, s>>>(tab, idx, lp, offR);
   } else {
-    chol_kernel<false><<<count, 256, 0, s>>>(tab, idx, lp, offR);
+    const size_t smem = ((size_t)lp * (lp + 1) / 2) * sizeof(float);
+    cudaFuncSetAttribute(chol_packed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (256 * 257 / 2) * 4);
+    chol_packed_kernel<<<count, 256, smem, s>>>(tab, idx, lp, offR);
   }
   ++g_kernel_launches;
 }
@@ -752,6 +840,124 @@ __global__ void __launch_bounds__(kJacobiThreads) jacobi_kernel(const MatDev* ta
   }
 }
 
+// The same SVD for 128 < lp <= 256, still on-chip: the two lp x lp work arrays (512 KB at lp = 256) are spread over the
+// shared memory of a CLUSTER of four blocks, lp / 4 columns of each array per block. A warp that rotates columns p and
+// q reaches them through distributed shared memory (plain loads and stores on addresses mapped into the owning block;
+// no multicast), rounds are separated by cluster barriers, and the "did anything rotate" flag lives in block 0.
+// Block 0 writes the results; the others wait in a final cluster barrier so that their shared memory stays alive.
+constexpr int kJacobiClusterThreads = 1024;     // 4 x 32 warps = one warp per column pair of a round at lp = 256
+
+__global__ void __cluster_dims__(4, 1, 1) __launch_bounds__(kJacobiClusterThreads)
+jacobi_cluster_kernel(const MatDev* tab, const int* idx, int lp, int rp, int rank, float tau_p) {
+  constexpr int kJacobiThreads = kJacobiClusterThreads;
+  namespace cg = cooperative_groups;
+  extern __shared__ __align__(16) float jc_smem[];
+  __shared__ float nrm[kMaxRank];
+  __shared__ int order[kMaxRank];
+  __shared__ int rotated;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int crank = (int)cluster.block_rank();
+  const MatDev& md = tab[idx[blockIdx.x >> 2]];
+  const int cols_per = lp >> 2;                        // lp is a multiple of 32
+  float* Kl = jc_smem;                                 // this block's columns of K = R^T ...
+  float* Jl = jc_smem + (size_t)cols_per * lp;         // ... and of the accumulated rotations
+  const float* R = md.racc;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarp = kJacobiThreads / 32;
+  for (int e = tid; e < cols_per * lp; e += kJacobiThreads) {
+    const int c = crank * cols_per + e / lp, i = e % lp;
+    Kl[e] = R[(size_t)c * lp + i];
+    Jl[e] = (c == i) ? 1.f : 0.f;
+  }
+  if (tid == 0) rotated = 0;
+  cluster.sync();
+  auto kcol = [&](int c) { return cluster.map_shared_rank(Kl + (size_t)(c % cols_per) * lp, c / cols_per); };
+  auto jcol = [&](int c) { return cluster.map_shared_rank(Jl + (size_t)(c % cols_per) * lp, c / cols_per); };
+  int* rot0 = cluster.map_shared_rank(&rotated, 0);
+  float* nrm0 = cluster.map_shared_rank(nrm, 0);
+  const int half = lp / 2, gw = crank * nwarp + warp, gwarps = 4 * nwarp;
+  for (int sweep = 0; sweep < 16; ++sweep) {
+    for (int rd = 0; rd < lp - 1; ++rd) {
+      for (int pi = gw; pi < half; pi += gwarps) {
+        int p, q;
+        if (pi == 0) { p = lp - 1; q = rd; }
+        else { p = (rd + pi) % (lp - 1); q = (rd - pi + (lp - 1)) % (lp - 1); }
+        float* kp = kcol(p); float* kq = kcol(q);
+        float* jp = jcol(p); float* jq = jcol(q);
+        // both columns of K and of J come into registers first (lp / 32 <= 8 elements per lane each): all the
+        // distributed-shared-memory loads of a pair are in flight together instead of one round trip per element
+        float x[8], y[8], u[8], w[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int i = lane + 32 * e;
+          const bool in = i < lp;
+          x[e] = in ? kp[i] : 0.f; y[e] = in ? kq[i] : 0.f;
+          u[e] = in ? jp[i] : 0.f; w[e] = in ? jq[i] : 0.f;
+        }
+        float a = 0.f, b = 0.f, c = 0.f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { a = fmaf(x[e], x[e], a); b = fmaf(y[e], y[e], b); c = fmaf(x[e], y[e], c); }
+        a = warp_sum(a); b = warp_sum(b); c = warp_sum(c);
+        const float lim = sqrtf(a) * sqrtf(b);
+        if (!(fabsf(c) > 1e-7f * lim) || lim == 0.f) continue;
+        if (fabsf(c) > 4e-6f * lim && lane == 0) *rot0 = 1;     // below this the fp32 dot product is noise
+        const float zeta = (b - a) / (2.f * c);
+        const float tt = copysignf(1.f, zeta) / (fabsf(zeta) + sqrtf(1.f + zeta * zeta));
+        const float cs = rsqrtf(1.f + tt * tt), sn = cs * tt;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const int i = lane + 32 * e;
+          if (i < lp) {
+            kp[i] = cs * x[e] - sn * y[e]; kq[i] = sn * x[e] + cs * y[e];
+            jp[i] = cs * u[e] - sn * w[e]; jq[i] = sn * u[e] + cs * w[e];
+          }
+        }
+      }
+      cluster.sync();
+    }
+    const int any = *rot0;          // the same value in every thread of the cluster: written before the barrier above
+    cluster.sync();                 // everyone has read it before block 0 clears it
+    if (!any) break;
+    if (crank == 0 && tid == 0) rotated = 0;
+    cluster.sync();
+  }
+  // column norms = singular values, into block 0
+  for (int j = warp; j < cols_per; j += nwarp) {
+    float a = 0.f;
+    for (int i = lane; i < lp; i += 32) { const float x = Kl[(size_t)j * lp + i]; a = fmaf(x, x, a); }
+    a = warp_sum(a);
+    if (lane == 0) nrm0[crank * cols_per + j] = sqrtf(a);
+  }
+  cluster.sync();
+  if (crank == 0) {
+    for (int j = tid; j < lp; j += kJacobiThreads) {      // rank of each column by counting (stable for ties)
+      int rk = 0;
+      const float sj = nrm[j];
+      for (int k = 0; k < lp; ++k) rk += (nrm[k] > sj) || (nrm[k] == sj && k < j);
+      order[rk] = j;
+    }
+    __syncthreads();
+    const float smax = nrm[order[0]];
+    for (int k = tid; k < rp; k += kJacobiThreads) {
+      float s = (k < rank && k < lp) ? nrm[order[k]] : 0.f;
+      if (!(s > 1e-7f * smax)) s = 0.f;
+      md.sv[k] = s;
+      md.d[k] = (s + tau_p > 0.f) ? s / (s + tau_p) : 0.f;
+    }
+    for (int e = tid; e < lp * rp; e += kJacobiThreads) {
+      const int i = e / rp, k = e % rp;
+      float u = 0.f, w = 0.f;
+      if (k < rank && k < lp) {
+        const int j = order[k];
+        const float s = nrm[j];
+        if (s > 1e-7f * smax) { u = kcol(j)[i] / s; w = jcol(j)[i]; }
+      }
+      md.ub[e] = u;
+      md.wb[e] = w;
+    }
+  }
+  cluster.sync();                   // nobody leaves while block 0 may still be reading its columns
+}
+
 void launch_jacobi(const MatDev* tab, const int* idx, int count, int lp, int rp, int rank, float tau_p,
                    cudaStream_t s) {
   if (count <= 0 || lp <= 0 || rp <= 0) return;
@@ -760,7 +966,9 @@ void launch_jacobi(const MatDev* tab, const int* idx, int count, int lp, int rp,
     cudaFuncSetAttribute(jacobi_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 128 * 128 * 4);
     jacobi_kernel<true><<<count, kJacobiThreads, smem, s>>>(tab, idx, lp, rp, rank, tau_p);
   } else {
-    jacobi_kernel<false><<<count, kJacobiThreads, 0, s>>>(tab, idx, lp, rp, rank, tau_p);
+    const size_t smem = (size_t)2 * (lp / 4) * lp * sizeof(float);
+    cudaFuncSetAttribute(jacobi_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 64 * 256 * 4);
+    jacobi_cluster_kernel<<<count * 4, kJacobiClusterThreads, smem, s>>>(tab, idx, lp, rp, rank, tau_p);
   }
   ++g_kernel_launches;
 }

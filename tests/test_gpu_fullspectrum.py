@@ -19,7 +19,7 @@ def torch():
     return torch
 
 
-def _run(torch, shapes, tau_p, n_anchor=2, tokens=192, planted=4, sqrt_iters=30, inv_iters=14, alpha=0.3, prescaled=True,
+def _run(torch, shapes, tau_p, n_anchor=2, tokens=192, planted=4, sqrt_iters=24, inv_iters=12, alpha=0.3, prescaled=True,
          keep=0.25):
     import paper_2609_14339_b200 as sc
     case = Case(shapes=shapes, rank=0, tokens=tokens, keep=keep, planted=planted, seed=7, tau_p=tau_p, n_anchor=n_anchor,
@@ -89,7 +89,7 @@ def test_fewer_iterations_only_under_weight(torch):
     """Directions whose square root has not converged get a smaller weight, never a larger one: the result moves
     towards alpha g, and the error against the exact operator falls as iterations are added."""
     errs = []
-    for it in (4, 10, 30):
+    for it in (4, 10, 24):
         _, out, _ = _run(torch, [(256, 384)], tau_p=60.0, sqrt_iters=it)
         errs.append(out[0]["gproj"])
     assert errs[0] > errs[1] > errs[2] and errs[2] < TOL, errs

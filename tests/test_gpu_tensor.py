@@ -241,3 +241,30 @@ def test_every_tile_of_every_matrix_is_updated_exactly_once(torch):
         assert float((v1[i] - v3[i]).double().norm() / v3[i].double().norm()) < 1e-5, i
         # element-wise as well: a tile applied twice or not at all moves dW by its whole size there
         assert float((dW1 - dW3).abs().max()) < 2e-2 * float(dW3.abs().max()), i
+
+
+@pytest.mark.parametrize("rank,tiles", [(96, 2), (128, 2), (128, 3), (256, 0), (200, 3)])
+@pytest.mark.parametrize("optimizer", [0, 1])
+def test_ranks_above_64_with_the_basis_panel_in_tensor_memory(torch, rank, tiles, optimizer, monkeypatch):
+    """Ranks above 64 keep the U panel of a work item in tensor memory (runs of `tiles` column tiles per item; the
+    library picks that path by itself for rank > 128 or large plans, here the run length is forced through its test
+    hook so that small matrices take it too). Ragged edges in both dimensions, several matrices, a last run that is
+    shorter than the others; AdamW and the dual-EMA optimizer."""
+    if tiles:
+        monkeypatch.setenv("SC_UT_TILES", str(tiles))
+    case = Case(shapes=[(520, 712), (520, 712), (264, 1160)], rank=rank, tokens=768, keep=0.25, planted=rank // 2, seed=6,
+                tau_p=120.0, optimizer=optimizer, beta3=0.99, mix_alpha=3.0)
+    inp = make_inputs(case)
+    g = GpuRun(case, inp, torch)
+    assert g.uses_tc and g.dev_status == 0
+    o = OracleRun(case, inp, "mirror")
+    eb = compare_basis(g, o)
+    assert max(eb["PU"], eb["PV"], eb["s"]) < TOL, eb
+    es = compare_step(g, o)
+    assert max(es["gproj"], es["m"], es["v"], es["dW"], es.get("ms", 0.0)) < TOL, es
+    # the same basis through the path that re-fetches U per tile: G_proj to rounding, everything else to 1e-6
+    monkeypatch.setenv("SC_NO_TMEM_U", "1")
+    g0 = GpuRun(case, inp, torch)
+    for i in range(len(case.shapes)):
+        assert rel(g.gproj[i], g0.gproj[i]) < 1e-6 and rel(g.W[i], g0.W[i]) < 1e-6
+        assert float(np.abs(g.gproj[i] - g0.gproj[i]).max()) < 1e-4 * float(np.abs(g0.gproj[i]).max())
