@@ -570,8 +570,8 @@ void launch_sketch_rowmajor(float* omega, int64_t rows, int width, uint64_t seed
 // A pivot that has cancelled to (numerically) nothing marks a column that lies in the span of the earlier
 // ones: that direction is dropped (its column of R^-1 is zero) instead of dividing by ~0.
 // =====================================================================================================
-// kSmem: the factor and its inverse are built in shared memory (2 lp^2 floats, lp <= 128) and copied out at the end;
-// otherwise they are built in place in global memory.
+// kSmem (the only form launched): the factor and its inverse are built in shared memory (2 lp^2 floats, lp <= 128) and
+// copied out at the end. Larger factors (lp <= 256) go through chol_packed_kernel below.
 template <bool kSmem>
 __global__ void __launch_bounds__(256) chol_kernel(const MatDev* tab, const int* idx, int lp, int offR) {
   extern __shared__ __align__(16) float chol_smem[];
@@ -755,7 +755,8 @@ constexpr int kJacobiThreads = 512;
 template <bool kSmem>
 __global__ void __launch_bounds__(kJacobiThreads) jacobi_kernel(const MatDev* tab, const int* idx, int lp, int rp,
                                                                 int rank, float tau_p) {
-  extern __shared__ __align__(16) float jac_smem[];   // kSmem: both l x l work arrays live here (lp <= 128)
+  extern __shared__ __align__(16) float jac_smem[];   // kSmem (the only form launched): both l x l work arrays live here
+                                                      // (lp <= 128); larger factors go through jacobi_cluster_kernel
   __shared__ float nrm[kMaxRank];
   __shared__ int order[kMaxRank];
   __shared__ int rotated;

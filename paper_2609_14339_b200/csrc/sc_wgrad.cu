@@ -269,9 +269,13 @@ struct TnEpilogue {
   float diag;
 };
 
+// GEN = false is the plain weight-gradient GEMM (one operand pair, bf16 or fp32 output): every generalisation below
+// folds away at compile time, so that path costs exactly what it did before the kernel was generalised.
+template <bool GEN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1)
-wgrad_pair_kernel(const __grid_constant__ TnMaps maps, int nseg, TnEpilogue epi, int tokens, int rows, int cols,
+wgrad_pair_kernel(const __grid_constant__ TnMaps maps, int nseg_arg, TnEpilogue epi, int tokens, int rows, int cols,
                   int n_fastest, unsigned* status) {
+  const int nseg = GEN ? nseg_arg : 1;
   void* __restrict__ G = epi.out;
   const int out_f32 = epi.out_mode == 1;
   const float scale = epi.scale;
@@ -311,17 +315,17 @@ wgrad_pair_kernel(const __grid_constant__ TnMaps maps, int nseg, TnEpilogue epi,
       bool dead = false;
       for (int tile = pair; tile < tiles && !dead; tile += n_pairs) {
         const int tm = n_fastest ? tile / tiles_n : tile % tiles_m, tn = n_fastest ? tile % tiles_n : tile / tiles_m;
-        for (int kk = 0; kk < kchunks * nseg; ++kk, ++it) {
-          const int seg = kk / kchunks, kc = kk - seg * kchunks;
+        for (int kk = 0, seg = 0, kc = 0; kk < kchunks * nseg; ++kk, ++it, ++kc) {
+          if (GEN && kc == kchunks) { kc = 0; ++seg; }
           const int s = it % kW2Stages;
           if (!mbar_wait(&bars->empty[s], ((it / kW2Stages) & 1) ^ 1, abort_flag)) { dead = true; break; }
           uint8_t* st = smem + (size_t)s * kW2StageBytes;
           if (rank == 0) mbar_expect_tx(&bars->full[s], 2 * kW2StageBytes);      // both blocks' bytes
           const uint32_t leader_bar = map_to_rank(smem_u32(&bars->full[s]), 0);
           for (int b = 0; b < 2; ++b)
-            tma_load_2d_pair(st + b * kWgBox, &maps.a[seg], leader_bar, tm * 256 + (int)rank * 128 + b * 64, kc * kWgBK);
+            tma_load_2d_pair(st + b * kWgBox, &maps.a[GEN ? seg : 0], leader_bar, tm * 256 + (int)rank * 128 + b * 64, kc * kWgBK);
           for (int b = 0; b < 2; ++b)
-            tma_load_2d_pair(st + kW2ABytes + b * kWgBox, &maps.b[seg], leader_bar, tn * 256 + (int)rank * 128 + b * 64,
+            tma_load_2d_pair(st + kW2ABytes + b * kWgBox, &maps.b[GEN ? seg : 0], leader_bar, tn * 256 + (int)rank * 128 + b * 64,
                              kc * kWgBK);
         }
       }
@@ -394,8 +398,11 @@ wgrad_pair_kernel(const __grid_constant__ TnMaps maps, int nseg, TnEpilogue epi,
         if (row < rows && col < cols) {
 #pragma unroll
           for (int j = 0; j < 16; ++j) v[j] *= scale;
-          if (epi.diag != 0.f && row >= col && row < col + 16) v[row - col] += epi.diag;
-          if (epi.out_mode == 2) {        // bf16 hi/lo pair: hi = rn(v), lo = rn(v - hi)
+          if (GEN && epi.diag != 0.f && row >= col && row < col + 16) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] += (col + j == row) ? epi.diag : 0.f;    // static indices: v stays in registers
+          }
+          if (GEN && epi.out_mode == 2) {        // bf16 hi/lo pair: hi = rn(v), lo = rn(v - hi)
             bf16* oh = static_cast<bf16*>(G) + (size_t)row * cols + col;
             bf16* ol = static_cast<bf16*>(epi.out_lo) + (size_t)row * cols + col;
 #pragma unroll
@@ -502,12 +509,12 @@ sc_status launch_tn_gemm(const void* const* A_segs, const void* const* B_segs, i
       cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 2)
     return SC_ERR_CUDA;
   const size_t smem2 = (size_t)kW2Stages * kW2StageBytes + sizeof(W2Bars) + 1024;
-  if (cudaFuncSetAttribute(wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
+  if (cudaFuncSetAttribute(wgrad_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
     return SC_ERR_CUDA;
   const long long tiles2 = ((M + 255) / 256) * ((N + 255) / 256);
   const int n_pairs = tiles2 < n_sm / 2 ? (int)tiles2 : n_sm / 2;
   const TnEpilogue epi{out, out_lo, out_mode, scale, diag};
-  wgrad_pair_kernel<<<2 * n_pairs, 192, smem2, s>>>(maps, nseg, epi, (int)K, (int)M, (int)N, M >= N ? 1 : 0, status);
+  wgrad_pair_kernel<true><<<2 * n_pairs, 192, smem2, s>>>(maps, nseg, epi, (int)K, (int)M, (int)N, M >= N ? 1 : 0, status);
   ++g_kernel_launches;
   return cudaGetLastError() == cudaSuccess ? SC_OK : SC_ERR_CUDA;
 }
@@ -553,14 +560,14 @@ extern "C" sc_status sc_masked_weight_grad(const void* dY_dev, const void* X_dev
   if (!pair_off && rows >= 256 && cols >= 256 && n_sm >= 2) {
     // pairs of SMs on 256 x 256 tiles (tcgen05 cta_group::2)
     const size_t smem2 = (size_t)kW2Stages * kW2StageBytes + sizeof(W2Bars) + 1024;
-    if (cudaFuncSetAttribute(wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
+    if (cudaFuncSetAttribute(wgrad_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
       return SC_ERR_CUDA;
     const int n_pairs = tiles2 < n_sm / 2 ? (int)tiles2 : n_sm / 2;
     TnMaps maps;
     maps.a[0] = map_dy; maps.b[0] = map_x;
     const TnEpilogue epi{G_dev, nullptr, out_dtype == SC_DTYPE_FP32 ? 1 : 0, scale, 0.f};
-    wgrad_pair_kernel<<<2 * n_pairs, 192, smem2, s>>>(maps, 1, epi, (int)tokens, (int)rows, (int)cols,
-                                                      rows >= cols ? 1 : 0, static_cast<unsigned*>(status_dev));
+    wgrad_pair_kernel<false><<<2 * n_pairs, 192, smem2, s>>>(maps, 1, epi, (int)tokens, (int)rows, (int)cols,
+                                                             rows >= cols ? 1 : 0, static_cast<unsigned*>(status_dev));
   } else {
     const long long tiles = ((rows + kWgBM - 1) / kWgBM) * ((cols + kWgBN - 1) / kWgBN);
     const int grid = tiles < n_sm ? (int)tiles : n_sm;
