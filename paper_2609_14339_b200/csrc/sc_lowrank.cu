@@ -63,22 +63,19 @@ __device__ __forceinline__ float4 load_g4(const void* G, size_t off) {
   return *reinterpret_cast<const float4*>(static_cast<const float*>(G) + off);
 }
 
-// Phase A. A warp owns ROWS rows at a time: M[i, :] = G[i, :] + E[i, :] (written back into E), P[i, :] = M[i, :] Q_prev.
-// Q_prev is staged chunk by chunk in shared memory, transposed (rho rows of kChunkA columns) so that a lane's four
-// consecutive columns are one conflict-free 128-bit read per factor; with several rows per warp each such read serves
-// all of them and more loads of the matrix are in flight per lane.
-template <int RHO, bool G_BF16, int ROWS>
+// Phase A. M[i, :] = G[i, :] + E[i, :] (written back into E), P[i, :] = M[i, :] Q_prev.
+// A persistent grid (a multiple of the SM count, so there is no partly filled last wave); warp w of block b owns rows
+// b * 8 + w, + 8 * gridDim.x, ... . The block walks over the columns in chunks of kChunkA: the chunk of Q_prev is staged
+// once in shared memory, transposed (rho rows of kChunkA columns) so that a lane's four consecutive columns are one
+// conflict-free 128-bit read per factor, then every warp runs that chunk of each of its rows and adds the chunk's
+// contribution to P (the same lane of the same warp every time, chunks in order: deterministic).
+template <int RHO, bool G_BF16>
 __global__ void __launch_bounds__(32 * kRowsPerBlockA)
 lowrank_mq_kernel(const void* __restrict__ G, float* __restrict__ E, const float* __restrict__ Qprev,
                   float* __restrict__ P, int rows, int cols) {
   __shared__ __align__(16) float Qs[RHO][kChunkA];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row0 = (blockIdx.x * kRowsPerBlockA + warp) * ROWS;
-  float acc[ROWS][RHO];
-#pragma unroll
-  for (int r = 0; r < ROWS; ++r)
-#pragma unroll
-    for (int k = 0; k < RHO; ++k) acc[r][k] = 0.f;
+  const int row_first = blockIdx.x * kRowsPerBlockA + warp, row_step = gridDim.x * kRowsPerBlockA;
   for (int c0 = 0; c0 < cols; c0 += kChunkA) {
     const int cw = min(kChunkA, cols - c0);
     __syncthreads();
@@ -87,41 +84,53 @@ lowrank_mq_kernel(const void* __restrict__ G, float* __restrict__ E, const float
       Qs[k][j] = Qprev[(size_t)(c0 + j) * RHO + k];
     }
     __syncthreads();
-    if (row0 >= rows) continue;
-#pragma unroll 2
-    for (int j = lane * 4; j < cw; j += 128) {                      // cols % 4 == 0, so a group of four is all in or out
-      float4 mv[ROWS];
+    for (int row = row_first; row < rows; row += row_step) {
+      float acc[RHO];
 #pragma unroll
-      for (int r = 0; r < ROWS; ++r) {
-        mv[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (row0 + r < rows) {
-          const size_t off = (size_t)(row0 + r) * cols + c0 + j;
-          mv[r] = load_g4<G_BF16>(G, off);
-          if (E) {
-            const float4 e4 = *reinterpret_cast<const float4*>(E + off);
-            mv[r].x += e4.x; mv[r].y += e4.y; mv[r].z += e4.z; mv[r].w += e4.w;
-            *reinterpret_cast<float4*>(E + off) = mv[r];
+      for (int k = 0; k < RHO; ++k) acc[k] = 0.f;
+      // Four column groups of 128 per trip, all loads first: the in-place write of M into E would otherwise pin every
+      // load of the next group behind the store of the previous one (same array, the compiler cannot tell them apart).
+      constexpr int kBatch = 4;
+      for (int j0 = lane * 4; j0 < cw; j0 += 128 * kBatch) {
+        float4 mv[kBatch];
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+          const int j = j0 + 128 * b;
+          mv[b] = j < cw ? load_g4<G_BF16>(G, (size_t)row * cols + c0 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (E) {
+          float4 ev[kBatch];
+#pragma unroll
+          for (int b = 0; b < kBatch; ++b) {
+            const int j = j0 + 128 * b;
+            ev[b] = j < cw ? *reinterpret_cast<const float4*>(E + (size_t)row * cols + c0 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+#pragma unroll
+          for (int b = 0; b < kBatch; ++b) {
+            const int j = j0 + 128 * b;
+            mv[b].x += ev[b].x; mv[b].y += ev[b].y; mv[b].z += ev[b].z; mv[b].w += ev[b].w;
+            if (j < cw) *reinterpret_cast<float4*>(E + (size_t)row * cols + c0 + j) = mv[b];
+          }
+        }
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+          const int j = j0 + 128 * b;
+          if (j >= cw) continue;
+#pragma unroll
+          for (int k = 0; k < RHO; ++k) {
+            const float4 q = *reinterpret_cast<const float4*>(&Qs[k][j]);
+            acc[k] = fmaf(mv[b].x, q.x, acc[k]); acc[k] = fmaf(mv[b].y, q.y, acc[k]);
+            acc[k] = fmaf(mv[b].z, q.z, acc[k]); acc[k] = fmaf(mv[b].w, q.w, acc[k]);
           }
         }
       }
 #pragma unroll
       for (int k = 0; k < RHO; ++k) {
-        const float4 q = *reinterpret_cast<const float4*>(&Qs[k][j]);
-#pragma unroll
-        for (int r = 0; r < ROWS; ++r) {
-          acc[r][k] = fmaf(mv[r].x, q.x, acc[r][k]); acc[r][k] = fmaf(mv[r].y, q.y, acc[r][k]);
-          acc[r][k] = fmaf(mv[r].z, q.z, acc[r][k]); acc[r][k] = fmaf(mv[r].w, q.w, acc[r][k]);
-        }
+        const float v = warp_sum(acc[k]);
+        if (lane == 0) P[(size_t)row * RHO + k] = (c0 == 0 ? 0.f : P[(size_t)row * RHO + k]) + v;
       }
     }
   }
-#pragma unroll
-  for (int r = 0; r < ROWS; ++r)
-#pragma unroll
-    for (int k = 0; k < RHO; ++k) {
-      const float v = warp_sum(acc[r][k]);
-      if (lane == 0 && row0 + r < rows) P[(size_t)(row0 + r) * RHO + k] = v;
-    }
 }
 
 // P_hat = orth(P) in one block: Cholesky QR twice. Each round: Gram matrix of the rows x rho panel (per-thread partial
@@ -279,30 +288,36 @@ lowrank_residual_kernel(float* __restrict__ E, const float* __restrict__ Phat, c
     for (int e = threadIdx.x; e < nr * RHO; e += blockDim.x) Ps[e / RHO][e % RHO] = Phat[(size_t)r0 * RHO + e];
     __syncthreads();
     if (!live) continue;
-#pragma unroll 4
-    for (int i = 0; i < nr; ++i) {
-      float* ptr = E + (size_t)(r0 + i) * cols + j;
-      float4 mv = *reinterpret_cast<const float4*>(ptr);
-      float lo[4] = {0.f, 0.f, 0.f, 0.f};
+    // four rows per trip, loads first (the in-place stores would otherwise hold the next row's load back)
+    for (int i0 = 0; i0 < nr; i0 += 4) {
+      float4 mv[4];
 #pragma unroll
-      for (int k = 0; k < RHO; ++k) {
-        const float p = Ps[i][k];
-        lo[0] = fmaf(p, q[0][k], lo[0]); lo[1] = fmaf(p, q[1][k], lo[1]);
-        lo[2] = fmaf(p, q[2][k], lo[2]); lo[3] = fmaf(p, q[3][k], lo[3]);
+      for (int b = 0; b < 4; ++b)
+        mv[b] = i0 + b < nr ? *reinterpret_cast<const float4*>(E + (size_t)(r0 + i0 + b) * cols + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        if (i0 + b >= nr) continue;
+        float lo[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int k = 0; k < RHO; ++k) {
+          const float p = Ps[i0 + b][k];
+          lo[0] = fmaf(p, q[0][k], lo[0]); lo[1] = fmaf(p, q[1][k], lo[1]);
+          lo[2] = fmaf(p, q[2][k], lo[2]); lo[3] = fmaf(p, q[3][k], lo[3]);
+        }
+        mv[b].x -= lo[0]; mv[b].y -= lo[1]; mv[b].z -= lo[2]; mv[b].w -= lo[3];
+        *reinterpret_cast<float4*>(E + (size_t)(r0 + i0 + b) * cols + j) = mv[b];
       }
-      mv.x -= lo[0]; mv.y -= lo[1]; mv.z -= lo[2]; mv.w -= lo[3];
-      *reinterpret_cast<float4*>(ptr) = mv;
     }
   }
 }
 
 template <int RHO>
 void launch_phase_a(const void* G, bool g_bf16, float* E, const float* Q, float* P, int rows, int cols, cudaStream_t s) {
-  // one row per warp: measured against four rows per warp (more loads in flight per lane, fewer streams) on
-  // 14336 x 4096: 0.18 ms against 0.25 ms
-  const int blocks = (rows + kRowsPerBlockA - 1) / kRowsPerBlockA;
-  if (g_bf16) lowrank_mq_kernel<RHO, true, 1><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
-  else lowrank_mq_kernel<RHO, false, 1><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
+  // Measured on 14336 x 4096: one row per warp at a time beats four (0.18 ms against 0.25 ms).
+  const int want = (rows + kRowsPerBlockA - 1) / kRowsPerBlockA;
+  const int blocks = want < 148 * 8 ? want : 148 * 8;          // eight blocks of 256 threads are resident per SM
+  if (g_bf16) lowrank_mq_kernel<RHO, true><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
+  else lowrank_mq_kernel<RHO, false><<<blocks, 32 * kRowsPerBlockA, 0, s>>>(G, E, Q, P, rows, cols);
 }
 template <int RHO>
 void launch_mtp(const void* M, bool m_bf16, const float* P, float* qpart, int rows, int cols, int slabs, int rps,
