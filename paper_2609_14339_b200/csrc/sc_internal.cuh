@@ -158,6 +158,7 @@ struct sc_plan {
   bool tensor_any = false;
   bool full = false;                  // full-spectrum soft filter (no rank cut)
   bool no_tmem_u = false;             // test hook (environment SC_NO_TMEM_U): ranks above 64 re-fetch U per tile instead
+  bool no_pair_project = false;       // test hook (environment SC_NO_PAIR_PROJECT): one block per 128-row tile instead
   int ut_tiles = 0;                   // test hook (environment SC_UT_TILES): tiles per item with U in tensor memory
   sc::FsState fs;
   int n_sm = 0;                       // SM count of the plan's device

@@ -395,6 +395,7 @@ sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int 
   p->keep = keep_ratio;
   p->n_sm = n_sm;
   p->no_tmem_u = getenv("SC_NO_TMEM_U") != nullptr;
+  p->no_pair_project = getenv("SC_NO_PAIR_PROJECT") != nullptr;
   p->ut_tiles = getenv("SC_UT_TILES") ? atoi(getenv("SC_UT_TILES")) : 0;
   if (p->ut_tiles < 0 || p->ut_tiles > 64) p->ut_tiles = 0;
   p->stream = reinterpret_cast<cudaStream_t>(stream);

@@ -16,7 +16,7 @@
 
 namespace sc {
 
-constexpr int kMapsPerMat = 27;
+constexpr int kMapsPerMat = 29;
 constexpr int kPerCallMaps = 7;   // the first seven are rebuilt whenever the caller's buffers move
 enum { MAP_G = 0,    // masked gradient, bf16, box 64 x 128 (MMA A operand of the projection)
        MAP_G32,      // masked gradient, bf16, box 32 x 128, 64-byte swizzle (streaming tile of the fused update)
@@ -32,7 +32,8 @@ enum { MAP_G = 0,    // masked gradient, bf16, box 64 x 128 (MMA A operand of th
        MAP_GANC32,               // anchor gradient, bf16, box 32 x 128, 64-byte swizzle (rebuilt per anchor call)
        MAP_M_F32,                // anchor momentum as plain fp32 (box 32 x 128): load and store of the fused EMA sweep
        MAP_U_MN, MAP_T,          // fp32 U (m x rp) and T (m x rp) as MN-major panels: X = U^T T on the tensor cores
-       MAP_SPARE };
+       MAP_SPARE,
+       MAP_VTHI_H, MAP_VTLO_H };   // V^T hi / lo with a box of rp / 2 rows: one block's half of the B operand of a pair
 constexpr int kTileBytes = 128 * 128;   // 128 rows x 64 bf16
 
 // =====================================================================================================
@@ -132,6 +133,142 @@ project_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, cons
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_d, tmem_cols);
+}
+
+// =====================================================================================================
+// The same projection on PAIRS of SMs (a cluster of two blocks, tcgen05.mma cta_group::2, M = 256): each block streams
+// its own 128 rows of G, but only HALF of every V^T tile (rp / 2 rows of the hi and of the lo part); the tensor cores of
+// both SMs read the two halves. With one block per tile every 16 KB tile of G came with a full hi + lo V^T tile out
+// of L2 and the kernel was bound by what TMA can bring into an SM (10.6 TB/s in all, half of it V^T); here the V^T
+// share is halved. Block 0 of a pair issues the MMAs; its barriers collect both blocks' bytes and its commits arrive in
+// both blocks. No multicast loads.
+// =====================================================================================================
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 2)
+project_pair_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx, const CUtensorMap* __restrict__ maps,
+                    int m, int n, int rp, int cps, int stages, uint32_t tmem_cols, unsigned* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int half_b = (rp / 2) * 128;                          // bytes of one block's half of V^T hi (or lo) per stage
+  const int stage_bytes = kTileBytes + 2 * half_b;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)stages * stage_bytes);
+  uint64_t* empty = full + stages;
+  uint64_t* accum = empty + stages;
+  uint64_t* drain = accum + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  volatile int* never_flag = abort_flag + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
+  const int row0 = (blockIdx.x >> 1) * 256 + (int)rank * 128;
+  const int nchunks = (n + 63) >> 6;
+  const int c0 = blockIdx.y * cps;
+  const int my_chunks = min(cps, nchunks - c0);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    mbar_init(accum, 1);
+    mbar_init(drain, 1);
+    *abort_flag = 0;
+    *never_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();            // the peer's barriers exist before anything is sent to them
+  tc_fence_after();
+  const uint32_t tmem_d = *tmem_slot;
+
+  if (warp == 0 && lane == 0) {
+    tensormap_acquire(mp + MAP_G); tensormap_acquire(mp + MAP_VTHI_H); tensormap_acquire(mp + MAP_VTLO_H);
+    int issued = 0;
+    bool dead = false;
+    for (int i = 0; i < my_chunks; ++i, ++issued) {
+      const int s = i % stages;
+      if (!mbar_wait(&empty[s], ((i / stages) & 1) ^ 1, abort_flag)) { dead = true; break; }
+      uint8_t* st = smem + (size_t)s * stage_bytes;
+      if (rank == 0) mbar_expect_tx(&full[s], 2u * (uint32_t)stage_bytes);      // both blocks' bytes
+      const uint32_t leader_bar = map_to_rank(smem_u32(&full[s]), 0);
+      const int x = (c0 + i) * 64;
+      tma_load_2d_pair(st, mp + MAP_G, leader_bar, x, row0);
+      tma_load_2d_pair(st + kTileBytes, mp + MAP_VTHI_H, leader_bar, x, (int)rank * (rp / 2));
+      tma_load_2d_pair(st + kTileBytes + half_b, mp + MAP_VTLO_H, leader_bar, x, (int)rank * (rp / 2));
+    }
+    if (dead) {
+      atomicOr(status, kDevTimeout);
+      *abort_flag = 1;
+      // the bytes of both blocks are counted on the leader's barriers: the leader waits (bounded) for the stages it
+      // armed, the other block idles for a grace period; both then meet in the cluster barrier at the end
+      if (rank == 0) {
+        for (int i = max(0, issued - stages); i < issued; ++i) mbar_wait(&full[i % stages], (i / stages) & 1, never_flag);
+      } else {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1 && lane == 0 && rank == 0) {
+    const uint32_t idesc = umma_idesc_bf16_pair(rp);
+    bool dead = false;
+    for (int i = 0; i < my_chunks; ++i) {
+      const int s = i % stages;
+      if (!mbar_wait(&full[s], (i / stages) & 1, abort_flag)) { dead = true; break; }
+      tc_fence_after();
+      const uint32_t a = smem_u32(smem + (size_t)s * stage_bytes);
+      const uint32_t bh = a + kTileBytes, bl = bh + half_b;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const uint64_t ad = umma_desc_k128(a + k * 32);
+        umma_bf16_pair(tmem_d, ad, umma_desc_k128(bh + k * 32), idesc, (i | k) != 0);
+        umma_bf16_pair(tmem_d, ad, umma_desc_k128(bl + k * 32), idesc, 1);
+      }
+      umma_commit_pair(&empty[s]);
+    }
+    if (!dead) {
+      umma_commit_pair(accum);
+    } else {
+      atomicOr(status, kDevTimeout);
+      *abort_flag = 1;
+      // MMAs already issued still read both blocks' shared memory: wait (bounded) until they are done
+      asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(drain)) : "memory");
+      mbar_wait(drain, 0, never_flag);
+    }
+  } else if (warp >= 2) {
+    const int q = warp & 3;
+    const int row = row0 + q * 32 + lane;
+    bool ok = my_chunks <= 0 || mbar_wait(accum, 0, abort_flag);
+    if (!ok && lane == 0) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
+    ok = __all_sync(0xffffffffu, ok) && !*abort_flag;
+    tc_fence_after();
+    if (ok) {
+      float* Trow = md.T + ((size_t)blockIdx.y * m + row) * rp;
+      for (int c = 0; c < rp; c += 16) {
+        float v[16];
+        if (my_chunks > 0) {
+          tmem_ld16(tmem_d + ((uint32_t)(q * 32) << 16) + c, v);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = 0.f;
+        }
+        if (row < m) {
+#pragma unroll
+          for (int j = 0; j < 16; j += 4)
+            *reinterpret_cast<float4*>(Trow + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();            // nothing of the peer is touched after this
+  if (warp == 1)
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols) : "memory");
 }
 
 // =====================================================================================================
@@ -972,6 +1109,7 @@ sc_status tc_init() {
   }
   // per device: the opt-in shared-memory sizes (cheap, so simply repeated for every plan)
   if (cudaFuncSetAttribute(project_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(project_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(fused_update_stream_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            StreamCfg<false>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
       cudaFuncSetAttribute(fused_update_stream_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -1037,6 +1175,8 @@ sc_status tc_encode_class(sc_plan* p, ShapeClass& c, bool static_part, bool per_
     if (static_part) {
       ok = ok && encode_bf16(mp + MAP_VTHI, md.Vthi, c.n, rp, c.n, rp);
       ok = ok && encode_bf16(mp + MAP_VTLO, md.Vtlo, c.n, rp, c.n, rp);
+      ok = ok && encode_bf16(mp + MAP_VTHI_H, md.Vthi, c.n, rp, c.n, rp / 2);
+      ok = ok && encode_bf16(mp + MAP_VTLO_H, md.Vtlo, c.n, rp, c.n, rp / 2);
       ok = ok && encode_bf16(mp + MAP_UHI, md.Uhi, rk, c.m, rk, 128);
       ok = ok && encode_bf16(mp + MAP_ULO, md.Ulo, rk, c.m, rk, 128);
       ok = ok && encode_bf16(mp + MAP_CTHI, md.Cthi, rk, c.n, rk, 128);
@@ -1090,6 +1230,17 @@ sc_status tc_launch_project(sc_plan* p, ShapeClass& c, const int* idx, int count
   const size_t smem = (size_t)stages * (kTileBytes + 2 * rp * 128) + 1024 + 256;
   uint32_t cols = 32;
   while ((int)cols < rp) cols <<= 1;
+  if (m >= 256 && !p->no_pair_project) {
+    // pairs of SMs on 256-row tiles, each block loading half of every V^T tile
+    const int stage_b = kTileBytes + rp * 128;
+    const int st2 = stages_for(stage_b, 6);
+    const size_t smem2 = (size_t)st2 * stage_b + 1024 + 256;
+    dim3 grid2(2 * ((m + 255) / 256), c.ksplit, count);
+    project_pair_kernel<<<grid2, 192, smem2, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), m, n,
+                                                          rp, cps, st2, cols, p->status_dev);
+    ++g_kernel_launches;
+    return cuda_ok(cudaGetLastError());
+  }
   dim3 grid((m + 127) / 128, c.ksplit, count);
   project_kernel<<<grid, 192, smem, p->stream>>>(p->dev_tab, idx, static_cast<const CUtensorMap*>(c.tmaps), m, n, rp,
                                                  cps, stages, cols, p->status_dev);
