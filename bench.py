@@ -31,6 +31,7 @@ BYTES_PER_ELEM_STEADY = 28.0      # read G (2) + read/write fp32 W, m, v (24) + 
 BYTES_PER_ELEM_UPDATE = 28.0      # what the fused update kernel itself moves per element (G is re-read here)
 TRAFFIC_PER_ELEM_UPDATE = 27.19   # dram read+write bytes per element of that kernel from one ncu capture of a
                                   # single 14336x4096 matrix; grows in proportion to the elements
+TRAFFIC_PER_ELEM_UPDATE_MIX = 35.20   # the same for the dual-EMA variant (36 algorithmic bytes per element)
 
 
 def parse_args():
@@ -423,7 +424,7 @@ def run_ours(args):
     upd_launches = max(prof["update"]["spans"] / nprof, 1)          # one launch per shape class and step
     roofline = {"bound": "hbm", "kernel": "fused_update_stream_kernel", "achieved": upd_gbs, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": upd_gbs / peaks["hbm_gbs"],
-                "traffic": None if mix else TRAFFIC_PER_ELEM_UPDATE * n_elems / upd_launches,
+                "traffic": (TRAFFIC_PER_ELEM_UPDATE_MIX if mix else TRAFFIC_PER_ELEM_UPDATE) * n_elems / upd_launches,
                 "peak_source": peaks["source"], "algorithmic_bytes_per_element": bytes_update,
                 "algorithmic_bytes_per_launch": bytes_update * n_elems / upd_launches,
                 "launches_per_step": upd_launches, "launch_ms": update_ms / upd_launches}

@@ -28,3 +28,16 @@ def test_other_ranks_of_the_reference_arm_do_no_work():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
                         "--warmup", "1"], capture_output=True, text=True, timeout=120, cwd=ROOT, env=env)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_per_shape_cpu_baseline_extrapolates_over_the_shape_counts():
+    """The cpu_baseline of the GPU arm: one matrix of each distinct shape, SVD measured where it fits the budget and
+    scaled by min(m, n)^2 max(m, n) elsewhere, multiplied by the counts."""
+    sys.path.insert(0, ROOT)
+    import bench
+    cfg = dict(layers=3, shapes=[(64, 96), (96, 64), (64, 96), (128, 160)], tokens=128, keep=0.5, k=2, r=4, dtype="bf16")
+    sec, cores, desc = bench.oracle_per_shape_run(cfg, cfg["layers"])
+    assert sec > 0 and cores >= 1 and "extrapolated" in desc
+    assert "(64, 96)" in desc and "(128, 160)" in desc
+    one, _ = bench._oracle_one_matrix(cfg, 64, 96, 1, 0)
+    assert sec > one                                   # the set costs more than one of its matrices

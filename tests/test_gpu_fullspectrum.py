@@ -105,6 +105,42 @@ def test_attention_kv_shape_full_size(torch):
     assert e["d"].max() > 0.5 and max(e["gproj"], e["m"], e["v"], e["dW"]) < TOL, e
 
 
+def test_attention_qo_shape_full_size(torch):
+    """One 4096 x 4096 matrix (the q / o projection of the 8B-shaped layer), as bench.py --full-spectrum launches it:
+    both soft projectors are 4096^2, every contraction runs 256 tiles of 256 x 256 over the 74 pairs of SMs."""
+    T = 1024
+    tau = 3.0 * 0.1 * np.sqrt(T) * (np.sqrt(4096) + np.sqrt(4096))
+    status, out, _ = _run(torch, [(4096, 4096)], tau_p=tau, n_anchor=1, tokens=T, planted=16, keep=0.1)
+    e = out[0]
+    print("full-spectrum 4096x4096", {k: v for k, v in e.items() if k != "d"}, "d range", e["d"].min(), e["d"].max())
+    assert e["d"].max() > 0.5 and max(e["gproj"], e["m"], e["v"], e["dW"]) < TOL, e
+
+
+def test_checkpoint_rebuilds_the_soft_projectors(torch):
+    """The checkpoint blob carries the anchor momentum only; an importing full-spectrum plan rebuilds P_U and P_V from
+    it, and a step afterwards is bit-identical to the exporting plan's."""
+    import paper_2609_14339_b200 as sc
+    shapes = [(256, 384), (256, 256)]
+    case = Case(shapes=shapes, rank=0, tokens=192, keep=0.25, planted=4, seed=9, tau_p=50.0)
+    inp = make_inputs(case)
+    hp = sc.Hparams.default(tau_p=50.0, lr=1e-2, full_spectrum=1)
+    a, b = sc.Plan(shapes, 0, 0.25, hp), sc.Plan(shapes, 0, 0.25, hp)
+    anc = [to_dev(inp["anchors"][i][0], "bf16", torch, "cuda:0") for i in range(2)]
+    a.anchor_update([anc[0], None], 3)                    # the second matrix has no anchor yet
+    b.state_import(a.state_export())
+    assert b.get_anchor_info() == (3, 1)
+    G = [to_dev(inp["G"][i], "bf16", torch, "cuda:0") for i in range(2)]
+    outs = []
+    for plan in (a, b):
+        W = [torch.from_numpy(inp["W"][i].copy()).cuda() for i in range(2)]
+        m = [torch.from_numpy(inp["m"][i].copy()).cuda() for i in range(2)]
+        v = [torch.from_numpy(inp["v"][i].copy()).cuda() for i in range(2)]
+        assert plan.correct_and_step(G, W, m, v, 100) == 0
+        torch.cuda.synchronize()
+        outs.append(W + m + v)
+    assert all(torch.equal(x, y) for x, y in zip(*outs))
+
+
 def test_rejects_unsupported_configurations(torch):
     import paper_2609_14339_b200 as sc
     hp = sc.Hparams.default(full_spectrum=1, tau_p=1.0)
