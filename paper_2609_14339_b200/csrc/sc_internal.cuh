@@ -45,7 +45,7 @@ struct MatDev {
   float* Ct;     // n x rp      C^T = V Xs^T, fp32
   bf16* Cthi;    // n x rk      bf16 split of C^T
   bf16* Ctlo;
-  float* xpart;  // kAtbMaxSplits x rp x rp   row-slice partials of X
+  float* xpart;  // split_m x rp x rp   row-slice partials of X
   float* sqpart; // kSqnormBlocks partial sums of ||G||^2
   float* stats;  // kStatsFloats
   // anchor-update scratch
@@ -158,6 +158,7 @@ struct sc_plan {
   bool tensor_any = false;
   bool full = false;                  // full-spectrum soft filter (no rank cut)
   bool no_tmem_u = false;             // test hook (environment SC_NO_TMEM_U): ranks above 64 re-fetch U per tile instead
+  bool no_fused_filter = false;       // test hook (environment SC_NO_FUSED_FILTER): filter and C^T as separate launches
   bool no_pair_project = false;       // test hook (environment SC_NO_PAIR_PROJECT): one block per 128-row tile instead
   int ut_tiles = 0;                   // test hook (environment SC_UT_TILES): tiles per item with U in tensor memory
   sc::FsState fs;
@@ -222,6 +223,9 @@ void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, i
 void launch_clip(const MatDev* tab, int n_mats, float max_norm, float* clip, cudaStream_t s);
 void launch_pad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, int cols_dst, cudaStream_t s);
 void launch_unpad_copy(float* dst, int ldd, const float* src, int lds, int rows, int cols, cudaStream_t s);
+bool filter_ct_supported(int rp);
+void launch_filter_ct(const MatDev* tab, const int* idx, int count, int rp, int rank, int n, int rk, float scale,
+                      float alpha, unsigned* status, cudaStream_t s);
 void launch_reduce_partials(const MatDev* tab, const int* idx, int count, int64_t numel, int ksplit, cudaStream_t s);
 
 // ---- tensor-core kernels (sc_tc.cu) -----------------------------------------------------------------------

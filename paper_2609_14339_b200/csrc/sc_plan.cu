@@ -396,6 +396,7 @@ sc_status sc_plan_create(sc_plan** out, const sc_shape* shapes, int n_mats, int 
   p->n_sm = n_sm;
   p->no_tmem_u = getenv("SC_NO_TMEM_U") != nullptr;
   p->no_pair_project = getenv("SC_NO_PAIR_PROJECT") != nullptr;
+  p->no_fused_filter = getenv("SC_NO_FUSED_FILTER") != nullptr;
   p->ut_tiles = getenv("SC_UT_TILES") ? atoi(getenv("SC_UT_TILES")) : 0;
   if (p->ut_tiles < 0 || p->ut_tiles > 64) p->ut_tiles = 0;
   p->stream = reinterpret_cast<cudaStream_t>(stream);
@@ -739,9 +740,12 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
       }
     }
     ProfScope ps(p, PROF_FILTER);
-    // X = U^T T as row-slice partials (the K-slice partials of T are added on the way in); xs_kernel adds them up
-    // (one block per matrix adds the slices inside xs_kernel unless that is too much for one block)
-    const bool sum_in_xs = (size_t)c.split_m * rp * rp <= (size_t)(1 << 16);
+    // X = U^T T as row-slice partials, added up in slice order: by a launch of its own, or inside xs_kernel when one
+    // block per matrix can do it
+    // few matrices: the filter and C^T in one launch (every block re-forms Xs, which only pays while there are few
+    // blocks); many matrices: the batched launches, whose launch latency is shared by the whole class
+    const bool one_launch = filter_ct_supported(rp) && (int64_t)cnt * ((n + 63) / 64) <= 1024 && !p->no_fused_filter;
+    const bool sum_in_xs = !one_launch && (size_t)c.split_m * rp * rp <= (size_t)(1 << 16);
     if (rp > 0 && c.tensor) {
       // plans with few matrices split K in the projection: add those partials of T up first (in place, slice 0)
       launch_reduce_partials(p->dev_tab, idx, cnt, (int64_t)m * rp, c.ksplit, s);
@@ -753,11 +757,15 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
                  !sum_in_xs);
     }
     if (want_norm) launch_sqnorm(p->dev_tab, idx, cnt, (int64_t)m * n, g_bf16, s);
-    launch_xs(p->dev_tab, idx, cnt, rp, p->rank, (rp > 0 && sum_in_xs) ? c.split_m : 0, scale, hp.alpha, p->status_dev, s);   // D X D
-    if (rp > 0) {
-      GemmArgs ga = gemm(p, idx, OFF(V), OFF(Xs), OFF(Ct), n, rp, rp, rp, rp, rp, 0, 1);             // C^T = V Xs^T
-      if (c.tensor) { ga.offHi = OFF(Cthi); ga.offLo = OFF(Ctlo); ga.ld_split = p->rk; }
-      launch_gemm(ga, cnt, s);
+    if (one_launch) {
+      launch_filter_ct(p->dev_tab, idx, cnt, rp, p->rank, n, p->rk, scale, hp.alpha, p->status_dev, s);   // D X D, C^T = V Xs^T
+    } else {
+      launch_xs(p->dev_tab, idx, cnt, rp, p->rank, (rp > 0 && sum_in_xs) ? c.split_m : 0, scale, hp.alpha, p->status_dev, s);   // D X D
+      if (rp > 0) {
+        GemmArgs ga = gemm(p, idx, OFF(V), OFF(Xs), OFF(Ct), n, rp, rp, rp, rp, rp, 0, 1);             // C^T = V Xs^T
+        if (c.tensor) { ga.offHi = OFF(Cthi); ga.offLo = OFF(Ctlo); ga.ld_split = p->rk; }
+        launch_gemm(ga, cnt, s);
+      }
     }
     return SC_OK;
   };

@@ -433,9 +433,39 @@ void launch_atb(const MatDev* tab, const int* idx, int count, int offA, int offB
   launch_sum_slices(tab, idx, count, offPart, offOut, ca * cb, nsplit, s);
 }
 
+// The same sum for many slices: 64 elements per block, the slices dealt to 16 groups of threads (group g adds slices
+// g, g + 16, ... in increasing order), the 16 group sums added in group order. Fixed order, so reproducible.
+__global__ void __launch_bounds__(1024) sum_slices_wide_kernel(const MatDev* tab, const int* idx, int offPart, int offOut,
+                                                              int numel, int nsplit) {
+  __shared__ float red[16][64];
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const float* part = field<const float>(md, offPart);
+  float* out = field<float>(md, offOut);
+  const int el = threadIdx.x & 63, g = threadIdx.x >> 6;
+  const int e = blockIdx.x * 64 + el;
+  float t = 0.f;
+  if (e < numel) {
+#pragma unroll 8
+    for (int s = g; s < nsplit; s += 16) t += part[(size_t)s * numel + e];
+  }
+  red[g][el] = t;
+  __syncthreads();
+  if (g == 0 && e < numel) {
+    float a = red[0][el];
+#pragma unroll
+    for (int k = 1; k < 16; ++k) a += red[k][el];
+    out[e] = a;
+  }
+}
+
 void launch_sum_slices(const MatDev* tab, const int* idx, int count, int offPart, int offOut, int numel, int nsplit,
                        cudaStream_t s) {
   if (count <= 0 || numel <= 0) return;
+  if (nsplit >= 32) {
+    sum_slices_wide_kernel<<<dim3((numel + 63) / 64, 1, count), 1024, 0, s>>>(tab, idx, offPart, offOut, numel, nsplit);
+    ++g_kernel_launches;
+    return;
+  }
   sum_slices_kernel<<<dim3((numel + 255) / 256 < 592 ? (numel + 255) / 256 : 592, 1, count), 256, 0, s>>>(
       tab, idx, offPart, offOut, numel, nsplit);
   ++g_kernel_launches;
@@ -1117,6 +1147,133 @@ void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, i
                unsigned* status, cudaStream_t s) {
   if (count <= 0) return;
   xs_kernel<<<count, 256, 0, s>>>(tab, idx, rp, rank, x_slices, scale, alpha, status);
+  ++g_kernel_launches;
+}
+
+// =====================================================================================================
+// The r x r filter and C^T = V Xs^T in one launch (padded rank up to 128). Every block forms Xs = coef * D X D in
+// shared memory from the summed X (16 to 64 KB out of L2) and multiplies its 64 rows of V by Xs^T; block 0 of a matrix
+// also writes Xs and the statistics, exactly as xs_kernel does. The sum over the rank index runs in increasing order
+// with one fmaf per term, like tsgemm_kernel, so C^T has the same bits as from the two separate launches.
+// CPT = rp / 16 columns of C^T per thread.
+// =====================================================================================================
+template <int CPT>
+__global__ void __launch_bounds__(256) filter_ct_kernel(const MatDev* tab, const int* idx, int rank, int n, int rk,
+                                                        float scale, float alpha, unsigned* status) {
+  constexpr int RP = 16 * CPT, XP = RP + 1, VP = RP + 4, RB = 64;
+  extern __shared__ __align__(16) float fct_smem[];
+  float* Vs = fct_smem;                  // [RB][VP]
+  float* Xs = fct_smem + RB * VP;        // [RP][XP]
+  __shared__ float red[5][8];
+  static_assert(kSqnormBlocks <= 256, "one partial of ||g||^2 per thread");
+  const MatDev& md = tab[idx[blockIdx.z]];
+  const bool lead = blockIdx.x == 0;
+  const int tid = threadIdx.x, row0 = blockIdx.x * RB;
+  for (int e = tid; e < RB * (RP / 4); e += 256) {
+    const int r = e / (RP / 4), q = e % (RP / 4);
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (row0 + r < n) v = *reinterpret_cast<const float4*>(md.V + (size_t)(row0 + r) * RP + 4 * q);
+    *reinterpret_cast<float4*>(Vs + r * VP + 4 * q) = v;
+  }
+  float sx = 0.f, s1 = 0.f, s2 = 0.f;
+  for (int e = tid; e < RP * RP; e += 256) {
+    const int i = e / RP, j = e % RP;
+    const float x = md.X[e] * scale;
+    const float dd = (i < rank && j < rank) ? md.d[i] * md.d[j] : 0.f;
+    const float xs = (1.f - alpha) * dd * x;
+    Xs[i * XP + j] = xs;
+    if (lead) {
+      md.Xs[e] = xs;
+      sx = fmaf(x, x, sx);
+      s1 = fmaf(dd * x, x, s1);
+      s2 = fmaf(dd * dd * x, x, s2);
+    }
+  }
+  if (lead) {
+    // ||g||^2 from its block partials and sum d^2, one term per thread; all five sums by warp, then in warp order
+    float gg = tid < kSqnormBlocks ? md.sqpart[tid] : 0.f;
+    float re = tid < rank ? md.d[tid] * md.d[tid] : 0.f;
+    sx = warp_sum(sx); s1 = warp_sum(s1); s2 = warp_sum(s2); gg = warp_sum(gg); re = warp_sum(re);
+    if ((tid & 31) == 0) {
+      const int w = tid >> 5;
+      red[0][w] = sx; red[1][w] = s1; red[2][w] = s2; red[3][w] = gg; red[4][w] = re;
+    }
+  }
+  __syncthreads();
+  if (lead && tid == 0) {
+    float tx = 0.f, t1 = 0.f, t2 = 0.f, gg = 0.f, re = 0.f;
+    for (int w = 0; w < 8; ++w) { tx += red[0][w]; t1 += red[1][w]; t2 += red[2][w]; gg += red[3][w]; re += red[4][w]; }
+    gg *= scale * scale;
+    md.stats[0] = gg;
+    md.stats[1] = tx;
+    md.stats[2] = alpha * alpha * gg + 2.f * alpha * (1.f - alpha) * t1 + (1.f - alpha) * (1.f - alpha) * t2;
+    md.stats[3] = re;
+    if (!isfinite(tx) || !isfinite(gg)) atomicOr(status, kDevNonfinite);
+  }
+  // rows ty + 16 i (i < 4), columns CPT tx .. CPT tx + CPT - 1
+  const int ty = tid >> 4, tx = tid & 15;
+  float acc[4][CPT];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) acc[i][j] = 0.f;
+#pragma unroll 4
+  for (int b = 0; b < RP; ++b) {
+    float xv[CPT], vv[4];
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) xv[j] = Xs[(tx * CPT + j) * XP + b];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) vv[i] = Vs[(ty + 16 * i) * VP + b];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) acc[i][j] = fmaf(vv[i], xv[j], acc[i][j]);
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int gr = row0 + ty + 16 * i;
+    if (gr >= n) continue;
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) {
+      const int gc = tx * CPT + j;
+      const float val = 1.f * acc[i][j];
+      md.Ct[(size_t)gr * RP + gc] = val;
+      if (md.Cthi) {
+        bf16 hi, lo;
+        split2(val, hi, lo);
+        md.Cthi[(size_t)gr * rk + gc] = hi;
+        md.Ctlo[(size_t)gr * rk + gc] = lo;
+      }
+    }
+  }
+}
+
+bool filter_ct_supported(int rp) { return rp >= 16 && rp <= 128 && rp % 16 == 0; }
+
+template <int CPT>
+static void launch_filter_ct_t(const MatDev* tab, const int* idx, int count, int rank, int n, int rk, float scale,
+                               float alpha, unsigned* status, cudaStream_t s) {
+  constexpr int RP = 16 * CPT;
+  constexpr size_t smem = ((size_t)64 * (RP + 4) + (size_t)RP * (RP + 1)) * sizeof(float);
+  static const cudaError_t attr =
+      cudaFuncSetAttribute(filter_ct_kernel<CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  (void)attr;
+  filter_ct_kernel<CPT><<<dim3((n + 63) / 64, 1, count), 256, smem, s>>>(tab, idx, rank, n, rk, scale, alpha, status);
+}
+
+void launch_filter_ct(const MatDev* tab, const int* idx, int count, int rp, int rank, int n, int rk, float scale,
+                      float alpha, unsigned* status, cudaStream_t s) {
+  if (count <= 0 || !filter_ct_supported(rp)) return;
+  switch (rp / 16) {
+    case 1: launch_filter_ct_t<1>(tab, idx, count, rank, n, rk, scale, alpha, status, s); break;
+    case 2: launch_filter_ct_t<2>(tab, idx, count, rank, n, rk, scale, alpha, status, s); break;
+    case 3: launch_filter_ct_t<3>(tab, idx, count, rank, n, rk, scale, alpha, status, s); break;
+    case 4: launch_filter_ct_t<4>(tab, idx, count, rank, n, rk, scale, alpha, status, s); break;
+    case 5: launch_filter_ct_t<5>(tab, idx, count, rank, n, rk, scale, alpha, status, s); break;
+    case 6: launch_filter_ct_t<6>(tab, idx, count, rank, n, rk, scale, alpha, status, s); break;
+    case 7: launch_filter_ct_t<7>(tab, idx, count, rank, n, rk, scale, alpha, status, s); break;
+    default: launch_filter_ct_t<8>(tab, idx, count, rank, n, rk, scale, alpha, status, s); break;
+  }
   ++g_kernel_launches;
 }
 
