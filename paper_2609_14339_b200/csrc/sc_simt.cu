@@ -1105,35 +1105,58 @@ void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, 
 // =====================================================================================================
 __global__ void __launch_bounds__(256) xs_kernel(const MatDev* tab, const int* idx, int rp, int rank, int x_slices,
                                                  float scale, float alpha, unsigned* status) {
-  __shared__ float red[3][8];
+  __shared__ float red[5][8];
   const MatDev& md = tab[idx[blockIdx.x]];
   float sx = 0.f, s1 = 0.f, s2 = 0.f;
-  for (int e = threadIdx.x; e < rp * rp; e += 256) {
-    const int i = e / rp, j = e % rp;
-    float xr;
+  const int numel = rp * rp;
+  // four elements per thread at a time, so that their loads (and the slices' loads) are in flight together
+  for (int e0 = threadIdx.x; e0 < numel; e0 += 4 * 256) {
+    float xr[4] = {0.f, 0.f, 0.f, 0.f};
     if (x_slices > 0) {                   // X = sum of the row-slice partials of U^T T, in slice order
-      xr = 0.f;
-      for (int sl = 0; sl < x_slices; ++sl) xr += md.xpart[(size_t)sl * rp * rp + e];
-      md.X[e] = xr;
-    } else {
-      xr = md.X[e];                       // already summed by a separate launch
+      for (int sl = 0; sl < x_slices; ++sl) {
+        const float* ps = md.xpart + (size_t)sl * numel;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int e = e0 + 256 * u;
+          if (e < numel) xr[u] += ps[e];
+        }
+      }
+    } else {                              // already summed by a separate launch
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int e = e0 + 256 * u;
+        if (e < numel) xr[u] = md.X[e];
+      }
     }
-    const float x = xr * scale;
-    const float dd = (i < rank && j < rank) ? md.d[i] * md.d[j] : 0.f;
-    md.Xs[e] = (1.f - alpha) * dd * x;
-    sx = fmaf(x, x, sx);
-    s1 = fmaf(dd * x, x, s1);
-    s2 = fmaf(dd * dd * x, x, s2);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int e = e0 + 256 * u;
+      if (e >= numel) break;
+      const int i = e / rp, j = e % rp;
+      if (x_slices > 0) md.X[e] = xr[u];
+      const float x = xr[u] * scale;
+      const float dd = (i < rank && j < rank) ? md.d[i] * md.d[j] : 0.f;
+      md.Xs[e] = (1.f - alpha) * dd * x;
+      sx = fmaf(x, x, sx);
+      s1 = fmaf(dd * x, x, s1);
+      s2 = fmaf(dd * dd * x, x, s2);
+    }
   }
-  sx = warp_sum(sx); s1 = warp_sum(s1); s2 = warp_sum(s2);
-  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = sx; red[1][threadIdx.x >> 5] = s1; red[2][threadIdx.x >> 5] = s2; }
+  // ||g||^2 from its block partials and sum d^2, one term per thread; all five sums by warp, then in warp order
+  const int tid = threadIdx.x;
+  float gg = tid < kSqnormBlocks ? md.sqpart[tid] : 0.f;
+  float re = tid < rank ? md.d[tid] * md.d[tid] : 0.f;
+  sx = warp_sum(sx); s1 = warp_sum(s1); s2 = warp_sum(s2); gg = warp_sum(gg); re = warp_sum(re);
+  if ((tid & 31) == 0) {
+    const int w = tid >> 5;
+    red[0][w] = sx; red[1][w] = s1; red[2][w] = s2; red[3][w] = gg; red[4][w] = re;
+  }
   __syncthreads();
   if (threadIdx.x == 0) {
-    float tx = 0.f, t1 = 0.f, t2 = 0.f, gg = 0.f, re = 0.f;
-    for (int w = 0; w < 8; ++w) { tx += red[0][w]; t1 += red[1][w]; t2 += red[2][w]; }
-    for (int b = 0; b < kSqnormBlocks; ++b) gg += md.sqpart[b];
+    float tx = 0.f, t1 = 0.f, t2 = 0.f;
+    gg = 0.f; re = 0.f;
+    for (int w = 0; w < 8; ++w) { tx += red[0][w]; t1 += red[1][w]; t2 += red[2][w]; gg += red[3][w]; re += red[4][w]; }
     gg *= scale * scale;
-    for (int k = 0; k < rank; ++k) re = fmaf(md.d[k], md.d[k], re);
     md.stats[0] = gg;
     md.stats[1] = tx;
     md.stats[2] = alpha * alpha * gg + 2.f * alpha * (1.f - alpha) * t1 + (1.f - alpha) * (1.f - alpha) * t2;
@@ -1169,24 +1192,54 @@ __global__ void __launch_bounds__(256) filter_ct_kernel(const MatDev* tab, const
   const MatDev& md = tab[idx[blockIdx.z]];
   const bool lead = blockIdx.x == 0;
   const int tid = threadIdx.x, row0 = blockIdx.x * RB;
-  for (int e = tid; e < RB * (RP / 4); e += 256) {
-    const int r = e / (RP / 4), q = e % (RP / 4);
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (row0 + r < n) v = *reinterpret_cast<const float4*>(md.V + (size_t)(row0 + r) * RP + 4 * q);
-    *reinterpret_cast<float4*>(Vs + r * VP + 4 * q) = v;
+  // every global load of a phase is issued before its first use (the kernel is a chain of load latencies otherwise)
+  __shared__ float ds[RP];
+  if (tid < RP) ds[tid] = tid < rank ? md.d[tid] : 0.f;
+  constexpr int NV = RB * (RP / 4) / 256;          // float4 loads of V per thread (= CPT)
+  float4 vreg[NV];
+#pragma unroll
+  for (int u = 0; u < NV; ++u) {
+    const int e = tid + 256 * u, r = e / (RP / 4), q = e % (RP / 4);
+    vreg[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (row0 + r < n) vreg[u] = *reinterpret_cast<const float4*>(md.V + (size_t)(row0 + r) * RP + 4 * q);
   }
+  constexpr int NX = RP * RP / 256;                // elements of X per thread (= CPT^2)
+  constexpr int XB = NX < 16 ? NX : 16;            // loaded in batches of up to 16
   float sx = 0.f, s1 = 0.f, s2 = 0.f;
-  for (int e = tid; e < RP * RP; e += 256) {
-    const int i = e / RP, j = e % RP;
-    const float x = md.X[e] * scale;
-    const float dd = (i < rank && j < rank) ? md.d[i] * md.d[j] : 0.f;
-    const float xs = (1.f - alpha) * dd * x;
-    Xs[i * XP + j] = xs;
-    if (lead) {
-      md.Xs[e] = xs;
-      sx = fmaf(x, x, sx);
-      s1 = fmaf(dd * x, x, s1);
-      s2 = fmaf(dd * dd * x, x, s2);
+  float xr[XB];
+#pragma unroll
+  for (int u = 0; u < XB; ++u) xr[u] = md.X[tid + 256 * u];
+#pragma unroll
+  for (int u = 0; u < NV; ++u) {
+    const int e = tid + 256 * u, r = e / (RP / 4), q = e % (RP / 4);
+    *reinterpret_cast<float4*>(Vs + r * VP + 4 * q) = vreg[u];
+  }
+  __syncthreads();                                 // ds
+  for (int b0 = 0; b0 < NX; b0 += XB) {
+    float xn[XB];
+    if (b0 + XB < NX) {
+#pragma unroll
+      for (int u = 0; u < XB; ++u) xn[u] = (b0 + XB + u < NX) ? md.X[tid + 256 * (b0 + XB + u)] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < XB; ++u) {
+      if (b0 + u >= NX) break;
+      const int e = tid + 256 * (b0 + u);
+      const int i = e / RP, j = e % RP;
+      const float x = xr[u] * scale;
+      const float dd = ds[i] * ds[j];              // zero beyond the rank
+      const float xs = (1.f - alpha) * dd * x;
+      Xs[i * XP + j] = xs;
+      if (lead) {
+        md.Xs[e] = xs;
+        sx = fmaf(x, x, sx);
+        s1 = fmaf(dd * x, x, s1);
+        s2 = fmaf(dd * dd * x, x, s2);
+      }
+    }
+    if (b0 + XB < NX) {
+#pragma unroll
+      for (int u = 0; u < XB; ++u) xr[u] = xn[u];
     }
   }
   if (lead) {
