@@ -1370,21 +1370,30 @@ void launch_unpad_copy(float* dst, int ldd, const float* src, int lds, int rows,
   launch_pad_copy(dst, ldd, src, lds, rows, cols, cols, s);
 }
 
-// Sum of split-K partials of T (fixed order): T[0] <- sum_s T[s].
-__global__ void reduce_partials_kernel(const MatDev* tab, const int* idx, int64_t numel, int ksplit) {
+// Sum of split-K partials of T (fixed order): T[0] <- sum_s T[s]. 128-bit accesses (numel is a multiple of 16), the
+// loads of all slices of an element issued together.
+__global__ void reduce_partials_kernel(const MatDev* tab, const int* idx, int64_t numel4, int ksplit) {
   const MatDev& md = tab[idx[blockIdx.z]];
+  float4* T4 = reinterpret_cast<float4*>(md.T);
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < numel; e += stride) {
-    float t = md.T[e];
-    for (int s = 1; s < ksplit; ++s) t += md.T[(size_t)s * numel + e];
-    md.T[e] = t;
+  for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < numel4; e += stride) {
+    float4 v[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s)
+      if (s < ksplit) v[s] = T4[(size_t)s * numel4 + e];
+    float4 t = v[0];
+#pragma unroll
+    for (int s = 1; s < 8; ++s)
+      if (s < ksplit) { t.x += v[s].x; t.y += v[s].y; t.z += v[s].z; t.w += v[s].w; }
+    T4[e] = t;
   }
 }
 
 void launch_reduce_partials(const MatDev* tab, const int* idx, int count, int64_t numel, int ksplit, cudaStream_t s) {
   if (count <= 0 || ksplit <= 1) return;
-  int blocks = (int)((numel + 255) / 256 < 592 ? (numel + 255) / 256 : 592);
-  reduce_partials_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, numel, ksplit);
+  const int64_t numel4 = numel / 4;      // rows x padded rank, the padded rank a multiple of 16
+  int blocks = (int)((numel4 + 255) / 256 < 1184 ? (numel4 + 255) / 256 : 1184);
+  reduce_partials_kernel<<<dim3(blocks, 1, count), 256, 0, s>>>(tab, idx, numel4, ksplit);
   ++g_kernel_launches;
 }
 
