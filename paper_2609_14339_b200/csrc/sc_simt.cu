@@ -1103,34 +1103,35 @@ void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, 
 // The r x r filter: Xs = coef * D X D (coef = (1-alpha)*scale), and the per-matrix statistics.
 //   stats[0] = ||g||^2, stats[1] = ||X||^2 (scaled), stats[2] = ||G_proj||^2 (closed form), stats[3] = sum d^2
 // =====================================================================================================
-__global__ void __launch_bounds__(256) xs_kernel(const MatDev* tab, const int* idx, int rp, int rank, int x_slices,
+__global__ void __launch_bounds__(1024) xs_kernel(const MatDev* tab, const int* idx, int rp, int rank, int x_slices,
                                                  float scale, float alpha, unsigned* status) {
-  __shared__ float red[5][8];
+  __shared__ float red[5][32];
+  const int nt = blockDim.x;             // 256 threads, 1024 above rank 128 (one block per matrix either way)
   const MatDev& md = tab[idx[blockIdx.x]];
   float sx = 0.f, s1 = 0.f, s2 = 0.f;
   const int numel = rp * rp;
   // four elements per thread at a time, so that their loads (and the slices' loads) are in flight together
-  for (int e0 = threadIdx.x; e0 < numel; e0 += 4 * 256) {
+  for (int e0 = threadIdx.x; e0 < numel; e0 += 4 * nt) {
     float xr[4] = {0.f, 0.f, 0.f, 0.f};
     if (x_slices > 0) {                   // X = sum of the row-slice partials of U^T T, in slice order
       for (int sl = 0; sl < x_slices; ++sl) {
         const float* ps = md.xpart + (size_t)sl * numel;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          const int e = e0 + 256 * u;
+          const int e = e0 + nt * u;
           if (e < numel) xr[u] += ps[e];
         }
       }
     } else {                              // already summed by a separate launch
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const int e = e0 + 256 * u;
+        const int e = e0 + nt * u;
         if (e < numel) xr[u] = md.X[e];
       }
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-      const int e = e0 + 256 * u;
+      const int e = e0 + nt * u;
       if (e >= numel) break;
       const int i = e / rp, j = e % rp;
       if (x_slices > 0) md.X[e] = xr[u];
@@ -1155,7 +1156,7 @@ __global__ void __launch_bounds__(256) xs_kernel(const MatDev* tab, const int* i
   if (threadIdx.x == 0) {
     float tx = 0.f, t1 = 0.f, t2 = 0.f;
     gg = 0.f; re = 0.f;
-    for (int w = 0; w < 8; ++w) { tx += red[0][w]; t1 += red[1][w]; t2 += red[2][w]; gg += red[3][w]; re += red[4][w]; }
+    for (int w = 0; w < nt / 32; ++w) { tx += red[0][w]; t1 += red[1][w]; t2 += red[2][w]; gg += red[3][w]; re += red[4][w]; }
     gg *= scale * scale;
     md.stats[0] = gg;
     md.stats[1] = tx;
@@ -1169,7 +1170,7 @@ __global__ void __launch_bounds__(256) xs_kernel(const MatDev* tab, const int* i
 void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, int x_slices, float scale, float alpha,
                unsigned* status, cudaStream_t s) {
   if (count <= 0) return;
-  xs_kernel<<<count, 256, 0, s>>>(tab, idx, rp, rank, x_slices, scale, alpha, status);
+  xs_kernel<<<count, rp > 128 ? 1024 : 256, 0, s>>>(tab, idx, rp, rank, x_slices, scale, alpha, status);
   ++g_kernel_launches;
 }
 
