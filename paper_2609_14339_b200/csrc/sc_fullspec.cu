@@ -28,60 +28,100 @@ inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 // ------------------------------------------------------------------------------------------ fp64 products
 // C (M x N, fp64) = alpha * op(A) op(B) + diag * I.  op(A) is M x K: A[i * lda + k], or A[k * lda + i] when TA.
 // op(B) is K x N: B[k * ldb + j], or B[j * ldb + k] when TB.  Inputs fp32 (the anchor momentum) or fp64.
-constexpr int DBM = 128, DBN = 64, DBK = 16;
+// 128 x 128 tile per block of 256 threads, 8 x 8 per thread as pairs of rows and columns interleaved across the tile (rows
+// 2 ty + {0, 1} + 32 i, columns 2 tx + {0, 1} + 32 j), so that every shared-memory read is a 16-byte one that the lanes
+// of a warp either share or read side by side. K advances 16 per stage; the next stage's global loads are in flight
+// while the current one multiplies, and land in the other half of the double buffer.
+constexpr int DBM = 128, DBN = 128, DBK = 16;
+constexpr int DPA = DBM + 2, DPB = DBN + 2;          // row pitch in doubles (even: 16-byte rows)
+constexpr size_t kDgemmSmem = (size_t)2 * DBK * (DPA + DPB) * sizeof(double);
 
 template <typename TIn, bool TA, bool TB>
 __global__ void __launch_bounds__(256)
 dgemm_kernel(const TIn* __restrict__ A, const TIn* __restrict__ B, double* __restrict__ C, int M, int N, int K, int lda,
              int ldb, int ldc, double alpha, double diag) {
-  __shared__ double As[DBK][DBM + 2];
-  __shared__ double Bs[DBK][DBN + 2];
+  extern __shared__ __align__(16) double dsm[];
+  double* As = dsm;                                  // [2][DBK][DPA]
+  double* Bs = dsm + 2 * DBK * DPA;                  // [2][DBK][DPB]
   const int row0 = blockIdx.y * DBM, col0 = blockIdx.x * DBN;
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
-  double acc[8][4];
+  constexpr int NA = DBM * DBK / 256, NB = DBN * DBK / 256;   // 8 and 8 elements per thread and stage
+  double ra[NA], rb[NB];
+  auto fetch = [&](int k0) {
 #pragma unroll
-  for (int i = 0; i < 8; ++i)
-#pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
-  for (int k0 = 0; k0 < K; k0 += DBK) {
-    for (int e = tid; e < DBM * DBK; e += 256) {
+    for (int u = 0; u < NA; ++u) {
+      const int e = tid + 256 * u;
       int r, k;
       if (!TA) { r = e / DBK; k = e % DBK; } else { k = e / DBM; r = e % DBM; }
       const int gr = row0 + r, gk = k0 + k;
-      double v = 0.0;
-      if (gr < M && gk < K) v = (double)(TA ? A[(size_t)gk * lda + gr] : A[(size_t)gr * lda + gk]);
-      As[k][r] = v;
+      ra[u] = (gr < M && gk < K) ? (double)(TA ? A[(size_t)gk * lda + gr] : A[(size_t)gr * lda + gk]) : 0.0;
     }
-    for (int e = tid; e < DBN * DBK; e += 256) {
+#pragma unroll
+    for (int u = 0; u < NB; ++u) {
+      const int e = tid + 256 * u;
       int c, k;
       if (!TB) { k = e / DBN; c = e % DBN; } else { c = e / DBK; k = e % DBK; }
       const int gc = col0 + c, gk = k0 + k;
-      double v = 0.0;
-      if (gc < N && gk < K) v = (double)(TB ? B[(size_t)gc * ldb + gk] : B[(size_t)gk * ldb + gc]);
-      Bs[k][c] = v;
+      rb[u] = (gc < N && gk < K) ? (double)(TB ? B[(size_t)gc * ldb + gk] : B[(size_t)gk * ldb + gc]) : 0.0;
     }
-    __syncthreads();
+  };
+  auto stash = [&](int buf) {
+    double* as = As + buf * DBK * DPA;
+    double* bs = Bs + buf * DBK * DPB;
+#pragma unroll
+    for (int u = 0; u < NA; ++u) {
+      const int e = tid + 256 * u;
+      int r, k;
+      if (!TA) { r = e / DBK; k = e % DBK; } else { k = e / DBM; r = e % DBM; }
+      as[k * DPA + r] = ra[u];
+    }
+#pragma unroll
+    for (int u = 0; u < NB; ++u) {
+      const int e = tid + 256 * u;
+      int c, k;
+      if (!TB) { k = e / DBN; c = e % DBN; } else { c = e / DBK; k = e % DBK; }
+      bs[k * DPB + c] = rb[u];
+    }
+  };
+  double acc[8][8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[i][j] = 0.0;
+  fetch(0);
+  stash(0);
+  __syncthreads();
+  const int nk = (K + DBK - 1) / DBK;
+  for (int t = 0; t < nk; ++t) {
+    const int buf = t & 1;
+    if (t + 1 < nk) fetch((t + 1) * DBK);
+    const double* as = As + buf * DBK * DPA + 2 * ty;
+    const double* bs = Bs + buf * DBK * DPB + 2 * tx;
 #pragma unroll
     for (int k = 0; k < DBK; ++k) {
-      double av[8], bv[4];
+      double av[8], bv[8];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) av[i] = As[k][ty * 8 + i];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) bv[j] = Bs[k][tx * 4 + j];
+      for (int i = 0; i < 4; ++i) {
+        const double2 a2 = *reinterpret_cast<const double2*>(as + k * DPA + 32 * i);
+        const double2 b2 = *reinterpret_cast<const double2*>(bs + k * DPB + 32 * i);
+        av[2 * i] = a2.x; av[2 * i + 1] = a2.y;
+        bv[2 * i] = b2.x; bv[2 * i + 1] = b2.y;
+      }
 #pragma unroll
       for (int i = 0; i < 8; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fma(av[i], bv[j], acc[i][j]);
+        for (int j = 0; j < 8; ++j) acc[i][j] = fma(av[i], bv[j], acc[i][j]);
     }
+    if (t + 1 < nk) stash(buf ^ 1);      // the other buffer: nobody reads it during this stage
     __syncthreads();
   }
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
-    const int gr = row0 + ty * 8 + i;
+    const int gr = row0 + 2 * ty + 32 * (i >> 1) + (i & 1);
     if (gr >= M) continue;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int gc = col0 + tx * 4 + j;
+    for (int j = 0; j < 8; ++j) {
+      const int gc = col0 + 2 * tx + 32 * (j >> 1) + (j & 1);
       if (gc < N) C[(size_t)gr * ldc + gc] = alpha * acc[i][j] + (gr == gc ? diag : 0.0);
     }
   }
@@ -90,8 +130,11 @@ dgemm_kernel(const TIn* __restrict__ A, const TIn* __restrict__ B, double* __res
 template <typename TIn, bool TA, bool TB>
 void dgemm(const TIn* A, const TIn* B, double* C, int M, int N, int K, int lda, int ldb, int ldc, double alpha,
            double diag, cudaStream_t s) {
+  static const cudaError_t attr = cudaFuncSetAttribute(dgemm_kernel<TIn, TA, TB>,
+                                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDgemmSmem);
+  (void)attr;
   dim3 grid((N + DBN - 1) / DBN, (M + DBM - 1) / DBM);
-  dgemm_kernel<TIn, TA, TB><<<grid, 256, 0, s>>>(A, B, C, M, N, K, lda, ldb, ldc, alpha, diag);
+  dgemm_kernel<TIn, TA, TB><<<grid, 256, kDgemmSmem, s>>>(A, B, C, M, N, K, lda, ldb, ldc, alpha, diag);
   ++g_kernel_launches;
 }
 
