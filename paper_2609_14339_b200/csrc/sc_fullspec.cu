@@ -39,7 +39,10 @@ constexpr size_t kDgemmSmem = (size_t)2 * DBK * (DPA + DPB) * sizeof(double);
 template <typename TIn, bool TA, bool TB>
 __global__ void __launch_bounds__(256)
 dgemm_kernel(const TIn* __restrict__ A, const TIn* __restrict__ B, double* __restrict__ C, int M, int N, int K, int lda,
-             int ldb, int ldc, double alpha, double diag) {
+             int ldb, int ldc, double alpha, double diag, int sym) {
+  // sym: the product is symmetric (a Gram matrix, or two commuting symmetric factors): only the tiles on and above the
+  // diagonal are computed and each is also written transposed
+  if (sym && blockIdx.x < blockIdx.y) return;
   extern __shared__ __align__(16) double dsm[];
   double* As = dsm;                                  // [2][DBK][DPA]
   double* Bs = dsm + 2 * DBK * DPA;                  // [2][DBK][DPB]
@@ -122,19 +125,23 @@ dgemm_kernel(const TIn* __restrict__ A, const TIn* __restrict__ B, double* __res
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int gc = col0 + 2 * tx + 32 * (j >> 1) + (j & 1);
-      if (gc < N) C[(size_t)gr * ldc + gc] = alpha * acc[i][j] + (gr == gc ? diag : 0.0);
+      if (gc >= N) continue;
+      const double v = alpha * acc[i][j] + (gr == gc ? diag : 0.0);
+      C[(size_t)gr * ldc + gc] = v;
+      if (sym && blockIdx.x != blockIdx.y) C[(size_t)gc * ldc + gr] = v;
     }
   }
 }
 
 template <typename TIn, bool TA, bool TB>
 void dgemm(const TIn* A, const TIn* B, double* C, int M, int N, int K, int lda, int ldb, int ldc, double alpha,
-           double diag, cudaStream_t s) {
+           double diag, cudaStream_t s, bool sym = false) {
   static const cudaError_t attr = cudaFuncSetAttribute(dgemm_kernel<TIn, TA, TB>,
                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDgemmSmem);
   (void)attr;
   dim3 grid((N + DBN - 1) / DBN, (M + DBM - 1) / DBM);
-  dgemm_kernel<TIn, TA, TB><<<grid, 256, kDgemmSmem, s>>>(A, B, C, M, N, K, lda, ldb, ldc, alpha, diag);
+  dgemm_kernel<TIn, TA, TB><<<grid, 256, kDgemmSmem, s>>>(A, B, C, M, N, K, lda, ldb, ldc, alpha, diag,
+                                                          sym && M == N ? 1 : 0);
   ++g_kernel_launches;
 }
 
@@ -278,16 +285,21 @@ static void fs_build_projector(sc_plan* p, const float* M, int m, int n, bool le
   double* normA = p->fs.scal; double* normY = p->fs.scal + 1;
   const int64_t numel = (int64_t)k * k;
   const int g = grid_for(numel);
-  if (left) dgemm<float, false, true>(M, M, A, k, k, n, n, n, k, 1.0, 0.0, s);      // M M^T
-  else dgemm<float, true, false>(M, M, A, k, k, m, n, n, k, 1.0, 0.0, s);           // M^T M
+  if (left) dgemm<float, false, true>(M, M, A, k, k, n, n, n, k, 1.0, 0.0, s, true);      // M M^T
+  else dgemm<float, true, false>(M, M, A, k, k, m, n, n, k, 1.0, 0.0, s, true);           // M^T M
   sqsum_part_kernel<<<kNormBlocks, 256, 0, s>>>(A, numel, p->fs.part);
   sqsum_final_kernel<<<1, 1, 0, s>>>(p->fs.part, kNormBlocks, normA);
   ns_init_kernel<<<g, 256, 0, s>>>(A, normA, Y, Z, k);
   g_kernel_launches += 3;
   // square root: T = (3 I - Z Y) / 2 ; Y <- Y T ; Z <- T Z.  A (no longer needed) is the second ping-pong buffer for Z.
+  // Y, Z and T are polynomials in the same symmetric matrix: they commute, so every product here is symmetric. Only the
+  // upper tiles of Z Y are computed (and of both products of the inverse iteration below). Y T and T Z are computed in
+  // full: a Gram matrix with a null space (more columns than rows) makes Z grow like 1.5^k there, and writing the upper
+  // tiles of Y T into the lower half mixes Y T with T Y, which feeds their rounding-level commutator back through that
+  // growth (measured: NaN after 24 iterations).
   double* Z2 = A;
   for (int it = 0; it < p->hp.fs_sqrt_iters; ++it) {
-    dgemm<double, false, false>(Z, Y, T, k, k, k, k, k, k, -0.5, 1.5, s);
+    dgemm<double, false, false>(Z, Y, T, k, k, k, k, k, k, -0.5, 1.5, s, true);
     dgemm<double, false, false>(Y, T, Y2, k, k, k, k, k, k, 1.0, 0.0, s);
     dgemm<double, false, false>(T, Z, Z2, k, k, k, k, k, k, 1.0, 0.0, s);
     std::swap(Y, Y2); std::swap(Z, Z2);
@@ -299,8 +311,8 @@ static void fs_build_projector(sc_plan* p, const float* M, int m, int n, bool le
   inv_init_kernel<<<g, 256, 0, s>>>(B, X, normA, normY, (double)p->hp.tau_p, k);
   g_kernel_launches += 3;
   for (int it = 0; it < p->hp.fs_inv_iters; ++it) {
-    dgemm<double, false, false>(B, X, R, k, k, k, k, k, k, -1.0, 2.0, s);
-    dgemm<double, false, false>(X, R, X2, k, k, k, k, k, k, 1.0, 0.0, s);
+    dgemm<double, false, false>(B, X, R, k, k, k, k, k, k, -1.0, 2.0, s, true);
+    dgemm<double, false, false>(X, R, X2, k, k, k, k, k, k, 1.0, 0.0, s, true);
     std::swap(X, X2);
   }
   soft_projector_out_kernel<<<g, 256, 0, s>>>(X, (double)p->hp.tau_p, k, hi, lo);
