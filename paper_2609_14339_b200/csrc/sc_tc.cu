@@ -671,17 +671,24 @@ constexpr int kUnitBf16 = 128 * kUnitW * 2;                  // 8 KB
 constexpr int kStreamStages = 3;                             // most stages any variant uses (sizes the barrier arrays)
 constexpr int kOpndU = 2 * kTileBytes;                       // U hi + lo, 128 rows x 64 bf16 each
 constexpr int kOpndC = 2 * (kTileN * 128);                   // C^T hi + lo, 64 rows x 64 bf16 each
-template <bool MIX>
+constexpr int kOpSlot = 16 * 1024;      // UT: one operand slot = a 128 x 64 bf16 tile of U (hi or lo), or C^T hi + lo (2 x 8 KB)
+constexpr int kMaxOpSlots = 6;
+template <bool MIX, bool UT = false>
 struct StreamCfg {
   static constexpr int kF32 = MIX ? 4 : 3;                              // fp32 arrays per unit: W, m, v (, slow m)
+  // Measured for UT on the 70B-shaped slice at rank 128 (update kernel against the HBM peak): three stages and three
+  // operand slots 0.894, the same with the store warp 0.904, two stages with six slots and the store warp 0.859, two
+  // stages with six slots without it 0.70 (one 14336 x 4096 matrix at rank 256: 0.81 / 0.81 / 0.83 / 0.64).
   static constexpr int kStages = MIX ? 2 : 3;
   static constexpr int kStageBytes = kF32 * kUnitF32 + kUnitBf16;      // 56 KB / 72 KB
-  static constexpr int kSmem = kStages * kStageBytes + kOpndU + kOpndC;
-  static constexpr int kStoreWarp = 10;                                 // MIX only
+  static constexpr int kOps = (UT && MIX) ? 4 : 3;                      // operand slots (UT); what fits beside the stages
+  static constexpr int kSmem = kStages * kStageBytes + (UT ? kOps * kOpSlot : kOpndU + kOpndC);
+  static constexpr bool kStoreWarpOn = MIX || UT;                       // a warp of its own sends the units out
+  static constexpr int kStoreWarp = 10;
 };
-// warps: 0 producer, 1 MMA, 2-9 consumers, then one store warp (MIX)
+// warps: 0 producer, 1 MMA, 2-9 consumers, then one store warp (MIX, UT)
 template <bool MIX, bool UT>
-constexpr int stream_threads() { return 320 + (MIX ? 32 : 0); }
+constexpr int stream_threads() { return 320 + ((MIX || UT) ? 32 : 0); }
 
 // Work items are handed out by an atomic counter: blocks do not run at the same speed (the slowest of a static split
 // finished 7% after the median), so each block's producer draws the next item when it needs one and passes the index
@@ -692,10 +699,10 @@ constexpr int kItemSlots = 8;
 struct StreamBars {
   uint64_t full[kStreamStages], empty[kStreamStages];
   uint64_t opnd_full, opnd_empty;
-  uint64_t op_full[3], op_empty[3];      // UT only: ring of three 16 KB operand slots
+  uint64_t op_full[kMaxOpSlots], op_empty[kMaxOpSlots];      // UT only: ring of 16 KB operand slots
   uint64_t acc_full[2], acc_empty[2];
   uint64_t item_ready[kItemSlots];
-  uint64_t store_ready[kStreamStages];   // MIX only: the consumers have finished a unit, the store warp may send it
+  uint64_t store_ready[kStreamStages];   // store-warp variants: the consumers have finished a unit, the store warp may send it
   int item_slot[kItemSlots];
   uint32_t tmem_slot;
   int abort_flag;
@@ -716,15 +723,15 @@ __device__ __forceinline__ void decode_item(const StreamGeom& g, int item, int& 
   ct1 = min(g.col_tiles, ct0 + g.tiles_per_chunk);
 }
 
-constexpr int kOpSlot = 16 * 1024;      // UT: one operand slot = a 128 x 64 bf16 tile of U (hi or lo), or C^T hi + lo (2 x 8 KB)
-
 template <bool MIX, bool UT>
 __global__ void __launch_bounds__(stream_threads<MIX, UT>(), 1)
 fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict__ idx,
                            const CUtensorMap* __restrict__ maps, StreamGeom g, StepScalars sc,
                            const float* __restrict__ clip_ptr, unsigned* status, unsigned* work_counter) {
-  constexpr int kStages = StreamCfg<MIX>::kStages, kStreamStageBytes = StreamCfg<MIX>::kStageBytes;
-  constexpr int kStreamSmem = StreamCfg<MIX>::kSmem, kF32 = StreamCfg<MIX>::kF32;
+  constexpr int kStages = StreamCfg<MIX, UT>::kStages, kStreamStageBytes = StreamCfg<MIX, UT>::kStageBytes;
+  constexpr int kStreamSmem = StreamCfg<MIX, UT>::kSmem, kF32 = StreamCfg<MIX, UT>::kF32;
+  constexpr int kOps = StreamCfg<MIX, UT>::kOps;
+  constexpr bool SW = StreamCfg<MIX, UT>::kStoreWarpOn;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* opnd = smem + kStages * kStreamStageBytes;
@@ -739,7 +746,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
     }
     mbar_init(&bars->opnd_full, 1);
     mbar_init(&bars->opnd_empty, 1);
-    for (int k = 0; k < 3; ++k) { mbar_init(&bars->op_full[k], 1); mbar_init(&bars->op_empty[k], 1); }
+    for (int k = 0; k < kMaxOpSlots; ++k) { mbar_init(&bars->op_full[k], 1); mbar_init(&bars->op_empty[k], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 8); }
     for (int k = 0; k < kItemSlots; ++k) mbar_init(&bars->item_ready[k], 1);
     bars->abort_flag = 0;
@@ -791,8 +798,8 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
             // dropped: no gain on the 70B-shaped set, slower on a single matrix.)
             const int n_u = ct == ct0 ? 2 * nch : 0;
             for (int j = 0; j < n_u + nch && !dead; ++j, ++op_it) {
-              const int sl = op_it % 3;
-              if (!mbar_wait(&bars->op_empty[sl], ((op_it / 3) & 1) ^ 1, abort_flag)) { dead = true; break; }
+              const int sl = op_it % kOps;
+              if (!mbar_wait(&bars->op_empty[sl], ((op_it / kOps) & 1) ^ 1, abort_flag)) { dead = true; break; }
               uint8_t* dst = opnd + sl * kOpSlot;
               mbar_expect_tx(&bars->op_full[sl], kOpSlot);
               if (j < n_u) {
@@ -841,7 +848,8 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
           mbar_wait(&bars->full[u % kStages], (u / kStages) & 1, &never);
         if (!UT && op_it > 0) mbar_wait(&bars->opnd_full, (op_it - 1) & 1, &never);
         if (UT)
-          for (uint32_t u = op_it > 3 ? op_it - 3 : 0; u < op_it; ++u) mbar_wait(&bars->op_full[u % 3], (u / 3) & 1, &never);
+          for (uint32_t u = op_it > (uint32_t)kOps ? op_it - kOps : 0; u < op_it; ++u)
+            mbar_wait(&bars->op_full[u % kOps], (u / kOps) & 1, &never);
       }
     }
     __syncwarp();
@@ -867,8 +875,8 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
             const uint32_t u_hi = tmem_base + 2 * kTileN, u_lo = u_hi + nch * 32;    // nch * 32 columns = rk / 2
             const int n_u = ct == ct0 ? 2 * nch : 0;
             for (int j = 0; j < n_u + nch && !dead; ++j, ++op_it) {
-              const int sl = op_it % 3;
-              if (!mbar_wait(&bars->op_full[sl], (op_it / 3) & 1, abort_flag)) { dead = true; break; }
+              const int sl = op_it % kOps;
+              if (!mbar_wait(&bars->op_full[sl], (op_it / kOps) & 1, abort_flag)) { dead = true; break; }
               tc_fence_after();
               const uint32_t sa = uh + sl * kOpSlot;
               if (j < n_u) {        // a U chunk: four K steps of 16 into tensor memory
@@ -927,7 +935,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
       decode_item(g, item, inst, rt, ct0, ct1);
       const MatDev& md = tab[idx[inst]];
       const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
-      if (!MIX && leader && inst != last_inst) {
+      if (!SW && leader && inst != last_inst) {
         tensormap_acquire(mp + MAP_W); tensormap_acquire(mp + MAP_M1); tensormap_acquire(mp + MAP_M2);
         tensormap_acquire(mp + MAP_WB);
       }
@@ -1003,7 +1011,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
           }
           fence_proxy_async();
           consumer_barrier();
-          if (MIX) {
+          if (SW) {
             if (leader) mbar_arrive(&bars->store_ready[s]);       // the store warp sends the unit and frees the stage
           } else if (leader) {
             tma_store_2d(mp + MAP_W, st, x, row0);
@@ -1023,9 +1031,9 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
       }
     }
     if (dead && lane == 0) { atomicOr(status, kDevTimeout); *abort_flag = 1; }
-    if (!MIX && leader) tma_store_wait_all();
-  } else if (MIX && warp == StreamCfg<MIX>::kStoreWarp) {
-    // -------------------------------------------------------------------- store warp (dual-EMA variant only)
+    if (!SW && leader) tma_store_wait_all();
+  } else if (SW && warp == StreamCfg<MIX, UT>::kStoreWarp) {
+    // -------------------------------------------------------------------- store warp (dual-EMA and UT variants)
     if (lane == 0) {
       uint32_t unit_it = 0;
       int last_inst = -1;
@@ -1040,7 +1048,8 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
         const CUtensorMap* mp = maps + (size_t)md.inst * kMapsPerMat;
         if (inst != last_inst) {
           tensormap_acquire(mp + MAP_W); tensormap_acquire(mp + MAP_M1); tensormap_acquire(mp + MAP_M2);
-          tensormap_acquire(mp + MAP_MS); tensormap_acquire(mp + MAP_WB);
+          if (MIX) tensormap_acquire(mp + MAP_MS);
+          tensormap_acquire(mp + MAP_WB);
           last_inst = inst;
         }
         const int row0 = rt * 128;
@@ -1055,7 +1064,7 @@ fused_update_stream_kernel(const MatDev* __restrict__ tab, const int* __restrict
             tma_store_2d(mp + MAP_W, st, x, row0);
             tma_store_2d(mp + MAP_M1, st + kUnitF32, x, row0);
             tma_store_2d(mp + MAP_M2, st + 2 * kUnitF32, x, row0);
-            tma_store_2d(mp + MAP_MS, st + 3 * kUnitF32, x, row0);
+            if (MIX) tma_store_2d(mp + MAP_MS, st + 3 * kUnitF32, x, row0);
             if (has_wb) tma_store_2d(mp + MAP_WB, st + kF32 * kUnitF32, x, row0);
             tma_store_commit();
             tma_store_wait_read<0>();          // the stage is free as soon as the stores have read it
@@ -1115,9 +1124,9 @@ sc_status tc_init() {
       cudaFuncSetAttribute(fused_update_stream_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            StreamCfg<true>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
       cudaFuncSetAttribute(fused_update_stream_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           StreamCfg<false>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
+                           StreamCfg<false, true>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
       cudaFuncSetAttribute(fused_update_stream_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           StreamCfg<true>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
+                           StreamCfg<true, true>::kSmem + (int)sizeof(StreamBars) + 1024) != cudaSuccess ||
       cudaFuncSetAttribute(ema_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(pass_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess ||
       cudaFuncSetAttribute(pass_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
@@ -1401,9 +1410,11 @@ sc_status tc_launch_epilogue(sc_plan* p, ShapeClass& c, const int* idx, int coun
 #define SC_LAUNCH_UPDATE(MIXV, UTV, SMEM)                                                                       \
   fused_update_stream_kernel<MIXV, UTV><<<grid, stream_threads<MIXV, UTV>(), SMEM, p->stream>>>(                \
       p->dev_tab, idx, maps, g, sc, p->clip_dev, p->status_dev, p->work_dev)
-  if (sc.mix && ut) SC_LAUNCH_UPDATE(true, true, smem_mix);
+  const size_t smem_mix_ut = StreamCfg<true, true>::kSmem + sizeof(StreamBars) + 1024;
+  const size_t smem_adam_ut = StreamCfg<false, true>::kSmem + sizeof(StreamBars) + 1024;
+  if (sc.mix && ut) SC_LAUNCH_UPDATE(true, true, smem_mix_ut);
   else if (sc.mix) SC_LAUNCH_UPDATE(true, false, smem_mix);
-  else if (ut) SC_LAUNCH_UPDATE(false, true, smem_adam);
+  else if (ut) SC_LAUNCH_UPDATE(false, true, smem_adam_ut);
   else SC_LAUNCH_UPDATE(false, false, smem_adam);
 #undef SC_LAUNCH_UPDATE
   ++g_kernel_launches;
