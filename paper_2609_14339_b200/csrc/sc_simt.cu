@@ -1106,7 +1106,7 @@ void launch_sqnorm(const MatDev* tab, const int* idx, int count, int64_t numel, 
 __global__ void __launch_bounds__(1024) xs_kernel(const MatDev* tab, const int* idx, int rp, int rank, int x_slices,
                                                  float scale, float alpha, unsigned* status) {
   __shared__ float red[5][32];
-  const int nt = blockDim.x;             // 256 threads, 1024 above rank 128 (one block per matrix either way)
+  const int nt = blockDim.x;             // 256 threads, 1024 from rank 64 on (one block per matrix either way)
   const MatDev& md = tab[idx[blockIdx.x]];
   float sx = 0.f, s1 = 0.f, s2 = 0.f;
   const int numel = rp * rp;
@@ -1170,7 +1170,7 @@ __global__ void __launch_bounds__(1024) xs_kernel(const MatDev* tab, const int* 
 void launch_xs(const MatDev* tab, const int* idx, int count, int rp, int rank, int x_slices, float scale, float alpha,
                unsigned* status, cudaStream_t s) {
   if (count <= 0) return;
-  xs_kernel<<<count, rp > 128 ? 1024 : 256, 0, s>>>(tab, idx, rp, rank, x_slices, scale, alpha, status);
+  xs_kernel<<<count, rp >= 64 ? 1024 : 256, 0, s>>>(tab, idx, rp, rank, x_slices, scale, alpha, status);
   ++g_kernel_launches;
 }
 
