@@ -198,6 +198,7 @@ struct GemmArgs {
   float alpha;
   float beta_c;            // C = alpha * acc + beta_c * C_old (0: plain store)
   int offHi, offLo, ld_split;   // when offHi != 0: also write the result as a bf16 hi/lo pair with this row stride
+  int split_only;               // with offHi: the fp32 result itself is not wanted (tsgemm_kernel only)
 };
 void launch_gemm(const GemmArgs& a, int count, cudaStream_t s);
 int atb_splits(int rows, int count);

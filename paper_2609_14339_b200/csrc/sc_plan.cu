@@ -763,7 +763,7 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
       launch_xs(p->dev_tab, idx, cnt, rp, p->rank, (rp > 0 && sum_in_xs) ? c.split_m : 0, scale, hp.alpha, p->status_dev, s);   // D X D
       if (rp > 0) {
         GemmArgs ga = gemm(p, idx, OFF(V), OFF(Xs), OFF(Ct), n, rp, rp, rp, rp, rp, 0, 1);             // C^T = V Xs^T
-        if (c.tensor) { ga.offHi = OFF(Cthi); ga.offLo = OFF(Ctlo); ga.ld_split = p->rk; }
+        if (c.tensor) { ga.offHi = OFF(Cthi); ga.offLo = OFF(Ctlo); ga.ld_split = p->rk; ga.split_only = 1; }
         launch_gemm(ga, cnt, s);
       }
     }

@@ -266,6 +266,8 @@ __global__ void __launch_bounds__(256, 2) tsgemm_kernel(GemmArgs a) {
   bf16* Clo = a.offHi ? field<bf16>(md, a.offLo) : nullptr;
   const int gc0 = col0 + tx * 4;
   const bool vec_c = ((reinterpret_cast<uintptr_t>(C) & 15) == 0) && (a.ldc % 4 == 0) && gc0 + 3 < a.N;
+  const bool vec_split = Chi && ((reinterpret_cast<uintptr_t>(Chi) & 7) == 0) && ((reinterpret_cast<uintptr_t>(Clo) & 7) == 0) &&
+                         (a.ld_split % 4 == 0);
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
     const int gr = row0 + i * 16 + ty;
@@ -274,7 +276,9 @@ __global__ void __launch_bounds__(256, 2) tsgemm_kernel(GemmArgs a) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) val[j] = a.alpha * acc[i][j];
     float* crow = C + (size_t)gr * a.ldc;
-    if (vec_c) {
+    if (Chi && a.split_only) {
+      // nobody reads the fp32 result (the tensor-core update takes the bf16 pair)
+    } else if (vec_c) {
       if (a.beta_c != 0.f) {
         const float4 o = *reinterpret_cast<const float4*>(crow + gc0);
         val[0] = fmaf(a.beta_c, o.x, val[0]); val[1] = fmaf(a.beta_c, o.y, val[1]);
@@ -290,13 +294,25 @@ __global__ void __launch_bounds__(256, 2) tsgemm_kernel(GemmArgs a) {
       }
     }
     if (Chi) {
+      bf16 hi[4], lo[4];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        if (gc0 + j >= a.N) continue;
-        bf16 hi, lo;
-        split2(val[j], hi, lo);
-        Chi[(size_t)gr * a.ld_split + gc0 + j] = hi;
-        Clo[(size_t)gr * a.ld_split + gc0 + j] = lo;
+      for (int j = 0; j < 4; ++j) split2(val[j], hi[j], lo[j]);
+      const size_t o = (size_t)gr * a.ld_split + gc0;
+      if (vec_split && gc0 + 3 < a.N) {            // four columns as one 8-byte store each
+        uint2 ph, pl;
+        ph.x = (uint32_t)__bfloat16_as_ushort(hi[0]) | ((uint32_t)__bfloat16_as_ushort(hi[1]) << 16);
+        ph.y = (uint32_t)__bfloat16_as_ushort(hi[2]) | ((uint32_t)__bfloat16_as_ushort(hi[3]) << 16);
+        pl.x = (uint32_t)__bfloat16_as_ushort(lo[0]) | ((uint32_t)__bfloat16_as_ushort(lo[1]) << 16);
+        pl.y = (uint32_t)__bfloat16_as_ushort(lo[2]) | ((uint32_t)__bfloat16_as_ushort(lo[3]) << 16);
+        *reinterpret_cast<uint2*>(Chi + o) = ph;
+        *reinterpret_cast<uint2*>(Clo + o) = pl;
+      } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          if (gc0 + j >= a.N) continue;
+          Chi[o + j] = hi[j];
+          Clo[o + j] = lo[j];
+        }
       }
     }
   }
