@@ -1303,17 +1303,29 @@ __global__ void __launch_bounds__(256) filter_ct_kernel(const MatDev* tab, const
   for (int i = 0; i < 4; ++i) {
     const int gr = row0 + ty + 16 * i;
     if (gr >= n) continue;
+    if (md.Cthi) {          // the tensor-core update takes the bf16 pair (nobody reads the fp32 copy then)
+      bf16 hi[CPT], lo[CPT];
 #pragma unroll
-    for (int j = 0; j < CPT; ++j) {
-      const int gc = tx * CPT + j;
-      const float val = 1.f * acc[i][j];
-      md.Ct[(size_t)gr * RP + gc] = val;
-      if (md.Cthi) {
-        bf16 hi, lo;
-        split2(val, hi, lo);
-        md.Cthi[(size_t)gr * rk + gc] = hi;
-        md.Ctlo[(size_t)gr * rk + gc] = lo;
+      for (int j = 0; j < CPT; ++j) split2(1.f * acc[i][j], hi[j], lo[j]);
+      const size_t o = (size_t)gr * rk + tx * CPT;
+      if (CPT % 4 == 0) {   // four columns as one 8-byte store (rk is a multiple of 64)
+#pragma unroll
+        for (int j = 0; j < CPT; j += 4) {
+          uint2 ph, pl;
+          ph.x = (uint32_t)__bfloat16_as_ushort(hi[j]) | ((uint32_t)__bfloat16_as_ushort(hi[j + 1]) << 16);
+          ph.y = (uint32_t)__bfloat16_as_ushort(hi[j + 2]) | ((uint32_t)__bfloat16_as_ushort(hi[j + 3]) << 16);
+          pl.x = (uint32_t)__bfloat16_as_ushort(lo[j]) | ((uint32_t)__bfloat16_as_ushort(lo[j + 1]) << 16);
+          pl.y = (uint32_t)__bfloat16_as_ushort(lo[j + 2]) | ((uint32_t)__bfloat16_as_ushort(lo[j + 3]) << 16);
+          *reinterpret_cast<uint2*>(md.Cthi + o + j) = ph;
+          *reinterpret_cast<uint2*>(md.Ctlo + o + j) = pl;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < CPT; ++j) { md.Cthi[o + j] = hi[j]; md.Ctlo[o + j] = lo[j]; }
       }
+    } else {
+#pragma unroll
+      for (int j = 0; j < CPT; ++j) md.Ct[(size_t)gr * RP + tx * CPT + j] = 1.f * acc[i][j];
     }
   }
 }
