@@ -58,6 +58,8 @@ def parse_args():
                     help="with --wgrad, --lowrank, --full-spectrum: time exactly --steps passes (profiler runs)")
     ap.add_argument("--wgrad", action="store_true",
                     help="time the masked weight gradients of one 8B-shaped layer (mask pass + tensor-core GEMM)")
+    ap.add_argument("--lowrank-streams", type=int, default=7,
+                    help="with --lowrank: streams the seven calls of a layer are spread over (1: one after the other)")
     ap.add_argument("--lowrank", action="store_true",
                     help="time the rank-4 gradient compressor with error feedback on the seven matrices of one 8B-shaped layer")
     ap.add_argument("--full-spectrum", action="store_true",
@@ -636,9 +638,30 @@ def run_lowrank(args):
     ws = [None] * len(shapes)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)      # larger than L2
 
+    # The matrices are independent and every call is a chain of short kernels, so the calls go out on a few streams
+    # (--lowrank-streams, forked from and joined to the current stream): one matrix's latency-bound phases run beside
+    # another's streaming ones.
+    n_streams = max(1, args.lowrank_streams)
+    side = [torch.cuda.Stream(device=device) for _ in range(n_streams)] if n_streams > 1 else []
+    fork = torch.cuda.Event()
+    joins = [torch.cuda.Event() for _ in side]
+
     def layer_pass():
-        for i in range(len(shapes)):
-            _, _, ws[i] = sc.lowrank_compress(G[i], Q[i], E=E[i], P=P[i], workspace=ws[i])
+        if not side:
+            for i in range(len(shapes)):
+                _, _, ws[i] = sc.lowrank_compress(G[i], Q[i], E=E[i], P=P[i], workspace=ws[i])
+            return
+        cur = torch.cuda.current_stream(device)
+        fork.record(cur)
+        order = sorted(range(len(shapes)), key=lambda i: -shapes[i][0] * shapes[i][1])     # largest first
+        for k, i in enumerate(order):
+            st = side[k % n_streams]
+            if k < n_streams:
+                st.wait_event(fork)
+            _, _, ws[i] = sc.lowrank_compress(G[i], Q[i], E=E[i], P=P[i], workspace=ws[i], stream=st)
+        for st, ev in zip(side, joins):
+            ev.record(st)
+            cur.wait_event(ev)
 
     for _ in range(max(args.warmup, 3)):
         layer_pass()
@@ -661,7 +684,7 @@ def run_lowrank(args):
         "metric": "low-rank gradient compressor with error feedback, one 8B-shaped layer (7 matrices), rank 4: gradient GB/s",
         "value": elems * 2 / (ms * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": 1, "steps": steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-        "data": "synthetic", "config": {"workload": "lowrank_llama8b_layer", "rho": rho, "elements": elems,
+        "data": "synthetic", "config": {"workload": "lowrank_llama8b_layer", "rho": rho, "elements": elems, "streams": n_streams,
                                         "l2": "256 MB buffer rewritten between timed iterations"},
         "gpu_launches": launches,
         "roofline": {"bound": "hbm", "kernel": "lowrank_mq_kernel + lowrank_mtp_kernel + lowrank_residual_kernel",
