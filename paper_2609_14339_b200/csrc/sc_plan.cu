@@ -777,7 +777,27 @@ static sc_status step_impl(sc_plan* p, const void* const* masked_grads, void* co
     return SC_OK;
   };
 
-  if (clip_on) {
+  // Device gradients, several shape classes: the projections and the short filter chains of the classes are independent,
+  // so each class runs them on its own stream (forked from and joined to the plan's stream, as in the anchor update)
+  // and one class's latency-bound chain runs beside another's projection; the updates follow on the plan's stream.
+  // Host gradients keep the class-by-class order, in which a class's update overlaps the next class's copy.
+  const bool fork = p->overlap_classes && !host_grads && p->classes.size() > 1 && rp > 0;
+  if (fork) {
+    cudaStream_t main_stream = p->stream;
+    if (cudaEventRecord(p->fork_ev, main_stream) != cudaSuccess) return SC_ERR_CUDA;
+    for (size_t ci = 0; ci < p->classes.size(); ++ci) {
+      cudaStream_t cs = p->class_streams[ci];
+      if (cudaStreamWaitEvent(cs, p->fork_ev, 0) != cudaSuccess) return SC_ERR_CUDA;
+      p->stream = cs; s = cs;
+      st = project(p->classes[ci]);
+      p->stream = main_stream; s = main_stream;
+      if (st != SC_OK) return st;
+      if (cudaEventRecord(p->join_evs[ci], cs) != cudaSuccess || cudaStreamWaitEvent(main_stream, p->join_evs[ci], 0) != cudaSuccess)
+        return SC_ERR_CUDA;
+    }
+    if (clip_on) launch_clip(p->dev_tab, p->n_mats, hp.max_grad_norm, p->clip_dev, s);
+    for (auto& c : p->classes) if ((st = update(c)) != SC_OK) return st;
+  } else if (clip_on) {
     for (auto& c : p->classes) if ((st = project(c)) != SC_OK) return st;
     launch_clip(p->dev_tab, p->n_mats, hp.max_grad_norm, p->clip_dev, s);
     for (auto& c : p->classes) if ((st = update(c)) != SC_OK) return st;
